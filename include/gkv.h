@@ -1,0 +1,178 @@
+/*
+ * gkv.h -- C ABI of the B200 (sm_100a) G-KV library: decode-time KV-cache eviction with a global
+ * attention score, and GQA decode attention over the compressed cache.
+ *
+ * Method (G-KV paper): Section 3 defines the eviction framework (compress every s generated
+ * tokens; the last w tokens are the observation window; keep the top-(b-w) scored tokens per KV
+ * head plus the window, so the cache returns to length b), Eq. 1 (window attention), the
+ * max-reduce over the query heads of a KV head, and Eq. 2 (local score S = window mean).
+ * Section 5 defines the global score F: S is divided by its per-head maximum and merged with the
+ * decayed history alpha*F_prev by Eq. 3 (max), Eq. 4 (average) or Eq. 5 (summation); rows
+ * without history and the first compression use the normalised S alone; the F of the retained
+ * rows is recorded for the next step.
+ *
+ * Conventions
+ *   - Every pointer named in gkv_buffers and every q/k/v/out/q_window/kept_idx argument of the
+ *     non-"_host" calls is a DEVICE pointer; the "_host" calls take HOST pointers (pinned memory
+ *     recommended). `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - The library owns no device memory: the caller allocates the buffers of gkv_query_sizes,
+ *     256-byte aligned, and keeps them alive until gkv_destroy. The context is host memory.
+ *   - All work is enqueued on the caller's stream; no call synchronises except
+ *     gkv_poll_device_status. Calls on one context must not overlap on the GPU (one stream, or
+ *     caller-side ordering).
+ *   - Every call returns a gkv_status; nothing is thrown across the boundary. Arguments are
+ *     validated before anything is launched; a failed call launches nothing.
+ *   - All sequences of the batch advance in lock step (one token per gkv_decode_attn call and
+ *     layer), so a layer has one cache length; the host keeps counters that mirror the device
+ *     copy.
+ *
+ * Layouts (d = head_dim = 128, C = budget + buffer rows per head, g = n_q_heads / n_kv_heads <= 8;
+ * query head i reads KV head i / g)
+ *   k, v     [n_layers][batch][n_kv_heads][C][d]  bf16      rows 0..len-1 valid
+ *   f        [n_layers][batch][n_kv_heads][C]     fp32      global score F of rows 0..n_hist-1
+ *   sacc     [n_layers][batch][n_kv_heads][C]     fp32      window sums: sum over the window's decode
+ *                                                            steps of max over the group of that
+ *                                                            step's attention weight (= w * S of Eq. 2)
+ *   pos      [n_layers][batch][n_kv_heads][C]     int32     original token position of each row
+ *                                                            (only with track_positions)
+ *   len      [2][n_layers][batch]                 int32     plane 0: cache length, plane 1: n_hist
+ *   q        [batch][n_q_heads][d]                bf16      (with layer = -1: [n_layers] in front)
+ *   k_new, v_new [batch][n_kv_heads][d]           bf16      (same)
+ *   out      [batch][n_q_heads][d]                bf16      (same)
+ *   q_window [batch][n_q_heads][w][d]             bf16      oldest window token first (same)
+ *   kept_idx [batch][n_kv_heads][b]               int32     (same)
+ */
+#ifndef GKV_H_
+#define GKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gkv_ctx gkv_ctx; /* opaque, host side, owns no device memory */
+
+typedef enum {
+    GKV_OK = 0,
+    GKV_ERR_INVALID_ARG = 1, /* NULL pointer, bad layer, inconsistent configuration            */
+    GKV_ERR_STATE = 2,       /* call not allowed in the current schedule state                 */
+    GKV_ERR_CAPACITY = 3,    /* the cache is full (len == C): evict before decoding further    */
+    GKV_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed                            */
+    GKV_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (latched status word)       */
+    GKV_ERR_UNSUPPORTED = 6  /* valid but not built (head_dim != 128, g > 8, ...)              */
+} gkv_status;
+
+/* Form of the global score (Section 5). LOCAL disables the history: F = normalised S. */
+typedef enum { GKV_MODE_MAX = 0, GKV_MODE_MEAN = 1, GKV_MODE_SUM = 2, GKV_MODE_LOCAL = 3 } gkv_mode;
+
+typedef struct {
+    int32_t n_layers, batch, n_q_heads, n_kv_heads, head_dim; /* head_dim must be 128           */
+    int32_t budget;   /* b: cache length after a compression (Section 3)                        */
+    int32_t buffer;   /* physical slack: C = budget + buffer rows per head                       */
+    int32_t window;   /* w: observation window, 1 <= w < b                                      */
+    int32_t interval; /* s: compress every s generated tokens, 1 <= s <= buffer, s >= w         */
+    float alpha;      /* memory decay rate of Eq. 3-5, in [0,1]; the paper uses 0.8             */
+    int32_t mode;     /* gkv_mode                                                               */
+    int32_t fuse_window_scores; /* 1: gkv_decode_attn adds each window token's group-max attention
+                                   row to sacc, and gkv_evict needs no q_window                 */
+    int32_t track_positions;    /* 1: pos carries original token positions through compaction   */
+} gkv_config;
+
+typedef struct { uint64_t k, v, f, sacc, pos, len, workspace, staging; } gkv_sizes; /* bytes      */
+typedef struct { void *k, *v, *f, *sacc, *pos, *len, *workspace, *staging; } gkv_buffers;
+
+/* Bytes of each caller-allocated device buffer for a configuration. `pos` is 0 without
+ * track_positions. `staging` is only needed by the "_host" calls (may be left NULL otherwise).
+ * Errors: INVALID_ARG (NULL, non-positive sizes, w >= b, s > buffer, s < w, alpha outside [0,1],
+ * n_q_heads not a multiple of n_kv_heads), UNSUPPORTED (head_dim != 128, g > 8, C > 4096). */
+gkv_status gkv_query_sizes(const gkv_config* cfg, gkv_sizes* out);
+
+/* Create a context over caller-owned device buffers and enqueue on `stream` the zeroing of k, v,
+ * f, sacc, pos, len and workspace (an empty cache: len = 0, no history). Encodes the TMA
+ * descriptors of k and v. The device current at this call is the context's device.
+ * Errors: as gkv_query_sizes; INVALID_ARG for a NULL or misaligned required buffer; CUDA. */
+gkv_status gkv_init(gkv_ctx** out, const gkv_config* cfg, const gkv_buffers* buffers, void* stream);
+
+/* Declare that the caller has filled the cache directly: rows 0..len-1 of k, v (and pos), the
+ * global scores of rows 0..n_hist-1 of f, and -- when window_scores_valid != 0 -- sacc holding the
+ * window sums of the last w tokens. Sets the host counters and enqueues the device copies.
+ * layer = -1 applies to all layers. since_evict is the number of tokens decoded since the last
+ * compression. Errors: INVALID_ARG (len > C, n_hist > len, bad layer). */
+gkv_status gkv_set_state(gkv_ctx* ctx, int32_t layer, int32_t len, int32_t n_hist, int32_t since_evict,
+                         int32_t window_scores_valid, void* stream);
+
+/* One decode step of attention (standard GQA attention over the compressed cache; the every-step
+ * part of the path whose cost Section 6.4 measures): append k_new, v_new at row len, then
+ * out[i] = sum_t softmax_t(q_i . K[i/g, t] / sqrt(d)) V[i/g, t] over t <= len (the new token
+ * included); len += 1. With fuse_window_scores, the last w steps before a scheduled compression
+ * also add max over the group of the final attention weights to sacc (this token's row of the
+ * group max that Eq. 2 averages). layer = -1 runs all layers in one launch with every tensor
+ * argument carrying a leading [n_layers] dimension.
+ * Errors: CAPACITY (len == C, nothing launched); STATE (fuse_window_scores and a compression is
+ * due: since_evict == interval); INVALID_ARG; CUDA. */
+gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const void* k_new,
+                           const void* v_new, void* out, void* stream);
+
+/* One compression step (Section 3 framework; Eq. 1-2 local score; Section 5 normalisation and
+ * Eq. 3-5 merge; top-(b-w) per KV head, equal scores resolved toward the lower position; kept
+ * rows in ascending position followed by the w window rows; K, V, F (and pos) compacted in
+ * place; len = b, n_hist = b-w, sacc = 0, since_evict = 0).
+ *   q_window == NULL : the local score is read from sacc (requires fuse_window_scores and
+ *                      since_evict == interval, or gkv_set_state(window_scores_valid = 1));
+ *   q_window != NULL : the local score is recomputed from the window queries and K (Eq. 1-2),
+ *                      each window token seeing the keys up to and including its own.
+ *   kept_idx_out     : optional; receives the pre-compaction row index of every kept row.
+ * If len <= b nothing is evicted: the call only resets since_evict and sacc.
+ * layer = -1 compresses all layers in one launch (leading [n_layers] dimension on the arguments).
+ * Errors: STATE (no valid window scores and no q_window; len < w), INVALID_ARG, CUDA. */
+gkv_status gkv_evict(gkv_ctx* ctx, int32_t layer, const void* q_window, int32_t* kept_idx_out,
+                     void* stream);
+
+/* The stages of gkv_evict as separate launches, for timing them one by one. They communicate
+ * through the workspace and must be called in order SCORE (only with q_window) -> MERGE ->
+ * SELECT -> COMPACT on one layer (or -1); after COMPACT the state equals that after gkv_evict.
+ * Results are identical to gkv_evict. Errors: as gkv_evict; STATE for an out-of-order stage. */
+typedef enum { GKV_STAGE_SCORE = 0, GKV_STAGE_MERGE = 1, GKV_STAGE_SELECT = 2, GKV_STAGE_COMPACT = 3 } gkv_stage;
+gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const void* q_window,
+                           int32_t* kept_idx_out, void* stream);
+
+/* Same operations with HOST buffers: inputs are copied to the staging buffer on `stream`, the
+ * kernels run, and the result is copied back, all asynchronously on `stream` (synchronise the
+ * stream before reading out / kept_idx_out). Require buffers.staging.
+ * Errors: as the device calls; INVALID_ARG when no staging buffer was given. */
+gkv_status gkv_decode_attn_host(gkv_ctx* ctx, int32_t layer, const void* q_host, const void* k_new_host,
+                                const void* v_new_host, void* out_host, void* stream);
+gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host,
+                          int32_t* kept_idx_out_host, void* stream);
+
+/* Host counters of one layer (no synchronisation): cache length, rows with history, tokens
+ * decoded since the last compression. Any output pointer may be NULL. */
+gkv_status gkv_get_state(const gkv_ctx* ctx, int32_t layer, int32_t* len, int32_t* n_hist,
+                         int32_t* since_evict);
+
+/* Number of kernels this context has launched so far (host counter). */
+int64_t gkv_launch_count(const gkv_ctx* ctx);
+
+/* Synchronises `stream` and returns GKV_ERR_TIMEOUT if any kernel latched an expired bounded
+ * wait since the last poll (the latch is then cleared), GKV_ERR_CUDA on a CUDA error, else OK. */
+gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream);
+
+/* Memory model of the paper's appendix "Memory Analysis": bytes of the full KV cache at
+ * seq_len tokens, of the compressed cache ((b + s) rows instead of seq_len), and of the score
+ * cache F (b - w entries per head), for `elem_bytes`-wide elements, over all layers and the
+ * whole batch. Pure host arithmetic. */
+typedef struct { uint64_t full_kv, compressed_kv, score_cache; } gkv_memory_model_t;
+gkv_status gkv_memory_model(const gkv_config* cfg, int64_t seq_len, int32_t elem_bytes,
+                            gkv_memory_model_t* out);
+
+const char* gkv_strerror(gkv_status status);
+
+/* Frees the host context only; device buffers stay with the caller. NULL is allowed. */
+void gkv_destroy(gkv_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GKV_H_ */

@@ -1,0 +1,513 @@
+// C-ABI entry points of the G-KV library: configuration checks, the host-side schedule state, the
+// workspace layout, TMA descriptor encoding and the kernel launches.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "gkv_common.cuh"
+#include "gkv_internal.h"
+
+using namespace gkv;
+
+namespace {
+
+constexpr int kMaxCapacity = 4096;
+constexpr uint64_t kAlign = 256;
+
+uint64_t align_up(uint64_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+gkv_status check_config(const gkv_config* c) {
+    if (!c) return GKV_ERR_INVALID_ARG;
+    if (c->n_layers <= 0 || c->batch <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0)
+        return GKV_ERR_INVALID_ARG;
+    if (c->budget <= 0 || c->buffer <= 0 || c->window <= 0 || c->interval <= 0) return GKV_ERR_INVALID_ARG;
+    if (c->window >= c->budget || c->interval > c->buffer || c->interval < c->window) return GKV_ERR_INVALID_ARG;
+    if (!(c->alpha >= 0.f && c->alpha <= 1.f)) return GKV_ERR_INVALID_ARG;
+    if (c->mode < GKV_MODE_MAX || c->mode > GKV_MODE_LOCAL) return GKV_ERR_INVALID_ARG;
+    if (c->n_q_heads % c->n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
+    if (c->head_dim != kHeadDim) return GKV_ERR_UNSUPPORTED;
+    if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return GKV_ERR_UNSUPPORTED;
+    if (c->budget + c->buffer > kMaxCapacity) return GKV_ERR_UNSUPPORTED;
+    const uint64_t rows = (uint64_t)c->n_layers * c->batch * c->n_kv_heads * (uint64_t)(c->budget + c->buffer);
+    if (rows >= (1ull << 31)) return GKV_ERR_UNSUPPORTED;  // TMA row coordinate is a signed 32-bit integer
+    return GKV_OK;
+}
+
+// Split factor of a decode launch over `units` units; 148 SMs assumed when no device is known.
+int splits_for(int units, int C, int sm_count) { return decode_pick_splits(units, C, sm_count > 0 ? sm_count : 148); }
+
+void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
+    const uint64_t L = c->n_layers, B = c->batch, H = c->n_kv_heads;
+    const uint64_t C = c->budget + c->buffer;
+    const uint64_t upl = B * H;
+    uint64_t off = 0;
+    w->status = off;    off = align_up(off + 64 * sizeof(int32_t));
+    w->seq_done = off;  off = align_up(off + L * B * sizeof(int32_t));
+    w->unit_done = off; off = align_up(off + L * upl * sizeof(int32_t));
+    // split-K scratch: sized for the larger of a one-layer launch and an all-layer launch
+    uint64_t part = 0, logits = 0;
+    const int cases[2] = {(int)upl, (int)(upl * L)};
+    for (int i = 0; i < 2; ++i) {
+        const int sp = splits_for(cases[i], (int)C, sm_count);
+        if (sp > 1) {
+            const uint64_t pb = (uint64_t)cases[i] * sp * (16 + kHeadDim * 8) * sizeof(float);
+            const uint64_t lb = (uint64_t)cases[i] * C * 8 * sizeof(float);
+            if (pb > part) part = pb;
+            if (lb > logits) logits = lb;
+        }
+    }
+    w->part = off;     off = align_up(off + part);
+    w->logits = off;   off = align_up(off + logits);
+    w->kept = off;     off = align_up(off + upl * c->budget * sizeof(int32_t));
+    w->fscratch = off; off = align_up(off + upl * C * sizeof(float));
+    w->total = off;
+}
+
+void fill_sizes(const gkv_config* c, int sm_count, gkv_sizes* s, WorkspaceLayout* wl) {
+    const uint64_t L = c->n_layers, B = c->batch, H = c->n_kv_heads, Hq = c->n_q_heads;
+    const uint64_t C = c->budget + c->buffer;
+    const uint64_t rows = L * B * H * C;
+    s->k = rows * kHeadDim * 2;
+    s->v = s->k;
+    s->f = rows * 4;
+    s->sacc = rows * 4;
+    s->pos = c->track_positions ? rows * 4 : 0;
+    s->len = 2 * L * B * 4;
+    WorkspaceLayout tmp;
+    layout_workspace(c, sm_count, &tmp);
+    s->workspace = tmp.total;
+    if (wl) *wl = tmp;
+    // staging for the host-buffer calls: q, k_new, v_new, out for all layers, or q_window + kept
+    const uint64_t dec = L * B * (Hq + 2 * H + Hq) * kHeadDim * 2;
+    const uint64_t evi = L * B * Hq * (uint64_t)c->window * kHeadDim * 2 + L * B * H * (uint64_t)c->budget * 4;
+    s->staging = align_up(dec > evi ? dec : evi) + 4 * kAlign;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D view of a K or V buffer: [rows][128] bf16, boxes of 64 rows x 64 elements, 128-byte swizzle.
+gkv_status encode_map(CUtensorMap* map, void* base, uint64_t rows) {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess || !sym)
+            return GKV_ERR_CUDA;
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTileKeys};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? GKV_OK : GKV_ERR_CUDA;
+}
+
+bool layer_ok(const gkv_ctx* ctx, int32_t layer) { return layer >= -1 && layer < ctx->cfg.n_layers; }
+void layer_range(const gkv_ctx* ctx, int32_t layer, int* l0, int* nl) {
+    if (layer < 0) { *l0 = 0; *nl = ctx->cfg.n_layers; }
+    else { *l0 = layer; *nl = 1; }
+}
+template <typename T>
+T* ws_ptr(const gkv_ctx* ctx, uint64_t off) { return reinterpret_cast<T*>(static_cast<uint8_t*>(ctx->buf.workspace) + off); }
+
+// All layers of a multi-layer call must be in the same schedule state.
+bool uniform(const std::vector<int32_t>& v, int l0, int nl) {
+    for (int i = 1; i < nl; ++i)
+        if (v[l0 + i] != v[l0]) return false;
+    return true;
+}
+
+EvictLaunch make_evict(gkv_ctx* ctx, int l0, int nl, int32_t* kept_out) {
+    EvictLaunch p;
+    const gkv_config& c = ctx->cfg;
+    p.k_cache = static_cast<__nv_bfloat16*>(ctx->buf.k);
+    p.v_cache = static_cast<__nv_bfloat16*>(ctx->buf.v);
+    p.f = static_cast<float*>(ctx->buf.f);
+    p.sacc = static_cast<float*>(ctx->buf.sacc);
+    p.pos = c.track_positions ? static_cast<int32_t*>(ctx->buf.pos) : nullptr;
+    p.len = static_cast<int32_t*>(ctx->buf.len);
+    p.seq_done = ws_ptr<int32_t>(ctx, ctx->ws.seq_done);
+    p.kept_out = kept_out;
+    p.kept_ws = ws_ptr<int32_t>(ctx, ctx->ws.kept);
+    p.f_ws = ws_ptr<float>(ctx, ctx->ws.fscratch);
+    p.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
+    p.layer0 = l0; p.n_layers = nl; p.L_total = c.n_layers; p.batch = c.batch; p.h_kv = c.n_kv_heads;
+    p.C = ctx->C; p.b = c.budget; p.w = c.window; p.alpha = c.alpha; p.mode = c.mode;
+    return p;
+}
+
+gkv_status launch_score_for(gkv_ctx* ctx, int l0, int nl, const void* q_window, cudaStream_t s) {
+    ScoreLaunch sp;
+    const gkv_config& c = ctx->cfg;
+    sp.q_win = static_cast<const __nv_bfloat16*>(q_window);
+    sp.sacc = static_cast<float*>(ctx->buf.sacc);
+    sp.len = static_cast<const int32_t*>(ctx->buf.len);
+    sp.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
+    sp.layer0 = l0; sp.n_layers = nl; sp.batch = c.batch; sp.h_q = c.n_q_heads; sp.h_kv = c.n_kv_heads;
+    sp.g = ctx->g; sp.C = ctx->C; sp.w = c.window;
+    sp.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
+    if (launch_score(sp, ctx->tm_k, s) != cudaSuccess) return GKV_ERR_CUDA;
+    ctx->launches += 1;
+    return GKV_OK;
+}
+
+// Shared validation of an eviction request. Returns GKV_OK with *noop set when len <= b.
+gkv_status evict_precheck(gkv_ctx* ctx, int32_t layer, bool need_window_sums, int* l0, int* nl, bool* noop) {
+    if (!ctx || !layer_ok(ctx, layer)) return GKV_ERR_INVALID_ARG;
+    layer_range(ctx, layer, l0, nl);
+    if (!uniform(ctx->len, *l0, *nl) || !uniform(ctx->n_hist, *l0, *nl) || !uniform(ctx->since_evict, *l0, *nl) ||
+        !uniform(ctx->sacc_valid, *l0, *nl))
+        return GKV_ERR_STATE;
+    const int len = ctx->len[*l0];
+    *noop = len <= ctx->cfg.budget;
+    if (*noop) return GKV_OK;
+    if (need_window_sums) {
+        const bool fused_ready = ctx->cfg.fuse_window_scores && ctx->since_evict[*l0] == ctx->cfg.interval;
+        if (!fused_ready && !ctx->sacc_valid[*l0]) return GKV_ERR_STATE;
+    }
+    return GKV_OK;
+}
+
+void after_evict(gkv_ctx* ctx, int l0, int nl, bool noop) {
+    for (int i = l0; i < l0 + nl; ++i) {
+        if (!noop) {
+            ctx->len[i] = ctx->cfg.budget;
+            ctx->n_hist[i] = ctx->cfg.budget - ctx->cfg.window;
+        }
+        ctx->since_evict[i] = 0;
+        ctx->sacc_valid[i] = 0;
+        ctx->stage_next[i] = 0;
+    }
+}
+
+gkv_status reset_sacc(gkv_ctx* ctx, int l0, int nl, cudaStream_t s) {
+    const size_t per_layer = (size_t)ctx->units_per_layer * ctx->C * sizeof(float);
+    if (cudaMemsetAsync(static_cast<uint8_t*>(ctx->buf.sacc) + l0 * per_layer, 0, nl * per_layer, s) != cudaSuccess)
+        return GKV_ERR_CUDA;
+    return GKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+gkv_status gkv_query_sizes(const gkv_config* cfg, gkv_sizes* out) {
+    if (!out) return GKV_ERR_INVALID_ARG;
+    const gkv_status st = check_config(cfg);
+    if (st != GKV_OK) return st;
+    int sm = 0, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+    (void)cudaGetLastError();  // no device (size queries on a CPU-only host) is not an error here
+    fill_sizes(cfg, sm, out, nullptr);
+    return GKV_OK;
+}
+
+gkv_status gkv_init(gkv_ctx** out, const gkv_config* cfg, const gkv_buffers* b, void* stream) {
+    if (!out || !b) return GKV_ERR_INVALID_ARG;
+    *out = nullptr;
+    gkv_status st = check_config(cfg);
+    if (st != GKV_OK) return st;
+    if (!b->k || !b->v || !b->f || !b->sacc || !b->len || !b->workspace) return GKV_ERR_INVALID_ARG;
+    if (cfg->track_positions && !b->pos) return GKV_ERR_INVALID_ARG;
+    const void* ptrs[] = {b->k, b->v, b->f, b->sacc, b->len, b->workspace, b->pos, b->staging};
+    for (const void* p : ptrs)
+        if (p && (reinterpret_cast<uintptr_t>(p) % kAlign) != 0) return GKV_ERR_INVALID_ARG;
+
+    gkv_ctx* ctx = new (std::nothrow) gkv_ctx();
+    if (!ctx) return GKV_ERR_CUDA;
+    ctx->cfg = *cfg;
+    ctx->buf = *b;
+    ctx->C = cfg->budget + cfg->buffer;
+    ctx->g = cfg->n_q_heads / cfg->n_kv_heads;
+    ctx->units_per_layer = cfg->batch * cfg->n_kv_heads;
+    ctx->launches = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    bool ok = cudaGetDevice(&ctx->device) == cudaSuccess &&
+              cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) == cudaSuccess;
+    if (ok) {
+        fill_sizes(cfg, ctx->sm_count, &ctx->sizes, &ctx->ws);
+        ok = cudaMemsetAsync(b->k, 0, ctx->sizes.k, s) == cudaSuccess &&
+             cudaMemsetAsync(b->v, 0, ctx->sizes.v, s) == cudaSuccess &&
+             cudaMemsetAsync(b->f, 0, ctx->sizes.f, s) == cudaSuccess &&
+             cudaMemsetAsync(b->sacc, 0, ctx->sizes.sacc, s) == cudaSuccess &&
+             cudaMemsetAsync(b->len, 0, ctx->sizes.len, s) == cudaSuccess &&
+             cudaMemsetAsync(b->workspace, 0, ctx->sizes.workspace, s) == cudaSuccess &&
+             (!cfg->track_positions || cudaMemsetAsync(b->pos, 0, ctx->sizes.pos, s) == cudaSuccess);
+    }
+    if (ok) ok = decode_kernel_setup() == cudaSuccess && score_kernel_setup() == cudaSuccess;
+    if (ok) {
+        const uint64_t rows = (uint64_t)cfg->n_layers * ctx->units_per_layer * ctx->C;
+        ok = encode_map(&ctx->tm_k, b->k, rows) == GKV_OK && encode_map(&ctx->tm_v, b->v, rows) == GKV_OK;
+    }
+    if (!ok) {
+        (void)cudaGetLastError();
+        delete ctx;
+        return GKV_ERR_CUDA;
+    }
+    ctx->len.assign(cfg->n_layers, 0);
+    ctx->n_hist.assign(cfg->n_layers, 0);
+    ctx->since_evict.assign(cfg->n_layers, 0);
+    ctx->sacc_valid.assign(cfg->n_layers, 0);
+    ctx->stage_next.assign(cfg->n_layers, 0);
+    *out = ctx;
+    return GKV_OK;
+}
+
+gkv_status gkv_set_state(gkv_ctx* ctx, int32_t layer, int32_t len, int32_t n_hist, int32_t since_evict,
+                         int32_t window_scores_valid, void* stream) {
+    if (!ctx || !layer_ok(ctx, layer)) return GKV_ERR_INVALID_ARG;
+    if (len < 0 || len > ctx->C || n_hist < 0 || n_hist > len || since_evict < 0) return GKV_ERR_INVALID_ARG;
+    int l0, nl;
+    layer_range(ctx, layer, &l0, &nl);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int B = ctx->cfg.batch, L = ctx->cfg.n_layers;
+    int32_t* dl = static_cast<int32_t*>(ctx->buf.len);
+    // a copy from pageable host memory has staged its source when the call returns, so `h` may be reused
+    std::vector<int32_t> h((size_t)nl * B);
+    for (auto& x : h) x = len;
+    if (cudaMemcpyAsync(dl + (size_t)l0 * B, h.data(), h.size() * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return GKV_ERR_CUDA;
+    for (auto& x : h) x = n_hist;
+    if (cudaMemcpyAsync(dl + (size_t)L * B + (size_t)l0 * B, h.data(), h.size() * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return GKV_ERR_CUDA;
+    for (int i = l0; i < l0 + nl; ++i) {
+        ctx->len[i] = len;
+        ctx->n_hist[i] = n_hist;
+        ctx->since_evict[i] = since_evict;
+        ctx->sacc_valid[i] = window_scores_valid ? 1 : 0;
+        ctx->stage_next[i] = 0;
+    }
+    return GKV_OK;
+}
+
+gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const void* k_new, const void* v_new,
+                           void* out, void* stream) {
+    if (!ctx || !layer_ok(ctx, layer) || !q || !k_new || !v_new || !out) return GKV_ERR_INVALID_ARG;
+    int l0, nl;
+    layer_range(ctx, layer, &l0, &nl);
+    if (!uniform(ctx->len, l0, nl) || !uniform(ctx->since_evict, l0, nl)) return GKV_ERR_STATE;
+    const gkv_config& c = ctx->cfg;
+    if (ctx->len[l0] >= ctx->C) return GKV_ERR_CAPACITY;
+    if (c.fuse_window_scores && ctx->since_evict[l0] >= c.interval) return GKV_ERR_STATE;
+
+    DecodeLaunch p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.k_cache = static_cast<__nv_bfloat16*>(ctx->buf.k);
+    p.v_cache = static_cast<__nv_bfloat16*>(ctx->buf.v);
+    p.sacc = static_cast<float*>(ctx->buf.sacc);
+    p.len = static_cast<int32_t*>(ctx->buf.len);
+    p.seq_done = ws_ptr<int32_t>(ctx, ctx->ws.seq_done);
+    p.unit_done = ws_ptr<int32_t>(ctx, ctx->ws.unit_done);
+    p.part = ws_ptr<float>(ctx, ctx->ws.part);
+    p.logits = ws_ptr<float>(ctx, ctx->ws.logits);
+    p.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
+    p.layer0 = l0; p.n_layers = nl; p.batch = c.batch; p.h_q = c.n_q_heads; p.h_kv = c.n_kv_heads;
+    p.g = ctx->g; p.C = ctx->C;
+    p.accum = (c.fuse_window_scores && ctx->since_evict[l0] >= c.interval - c.window) ? 1 : 0;
+    p.splits = decode_pick_splits(nl * ctx->units_per_layer, ctx->C, ctx->sm_count);
+    p.stages = decode_pick_stages(ctx->C, p.accum, p.splits, nullptr);
+    p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
+    if (launch_decode(p, ctx->tm_k, ctx->tm_v, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GKV_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    for (int i = l0; i < l0 + nl; ++i) {
+        ctx->len[i] += 1;
+        ctx->since_evict[i] += 1;
+        ctx->stage_next[i] = 0;
+        // window sums written by hand are stale once further tokens are decoded without accumulation
+        if (!p.accum) ctx->sacc_valid[i] = 0;
+    }
+    return GKV_OK;
+}
+
+gkv_status gkv_evict(gkv_ctx* ctx, int32_t layer, const void* q_window, int32_t* kept_idx_out, void* stream) {
+    int l0, nl;
+    bool noop;
+    gkv_status st = evict_precheck(ctx, layer, q_window == nullptr, &l0, &nl, &noop);
+    if (st != GKV_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (noop) {
+        st = reset_sacc(ctx, l0, nl, s);
+        if (st != GKV_OK) return st;
+        after_evict(ctx, l0, nl, true);
+        return GKV_OK;
+    }
+    if (q_window) {
+        st = launch_score_for(ctx, l0, nl, q_window, s);
+        if (st != GKV_OK) return st;
+    }
+    const EvictLaunch p = make_evict(ctx, l0, nl, kept_idx_out);
+    if (launch_evict_fused(p, s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GKV_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    after_evict(ctx, l0, nl, false);
+    return GKV_OK;
+}
+
+gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const void* q_window, int32_t* kept_idx_out,
+                           void* stream) {
+    int l0, nl;
+    bool noop;
+    if (stage < GKV_STAGE_SCORE || stage > GKV_STAGE_COMPACT) return GKV_ERR_INVALID_ARG;
+    gkv_status st = evict_precheck(ctx, layer, false, &l0, &nl, &noop);
+    if (st != GKV_OK) return st;
+    if (nl != 1) return GKV_ERR_UNSUPPORTED;  // the staged scratch holds one layer
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int& next = ctx->stage_next[l0];
+    if (noop) {
+        if (stage == GKV_STAGE_COMPACT) {
+            st = reset_sacc(ctx, l0, nl, s);
+            if (st != GKV_OK) return st;
+            after_evict(ctx, l0, nl, true);
+        }
+        return GKV_OK;
+    }
+    if (stage == GKV_STAGE_SCORE) {
+        if (!q_window || next != 0) return next != 0 ? GKV_ERR_STATE : GKV_ERR_INVALID_ARG;
+        st = launch_score_for(ctx, l0, nl, q_window, s);
+        if (st != GKV_OK) return st;
+        ctx->sacc_valid[l0] = 1;
+        next = GKV_STAGE_MERGE;
+        return GKV_OK;
+    }
+    const EvictLaunch p = make_evict(ctx, l0, nl, stage == GKV_STAGE_SELECT ? kept_idx_out : nullptr);
+    cudaError_t e;
+    if (stage == GKV_STAGE_MERGE) {
+        if (next != 0 && next != GKV_STAGE_MERGE) return GKV_ERR_STATE;
+        const bool fused_ready = ctx->cfg.fuse_window_scores && ctx->since_evict[l0] == ctx->cfg.interval;
+        if (!fused_ready && !ctx->sacc_valid[l0]) return GKV_ERR_STATE;
+        e = launch_evict_merge(p, s);
+        if (e == cudaSuccess) next = GKV_STAGE_SELECT;
+    } else if (stage == GKV_STAGE_SELECT) {
+        if (next != GKV_STAGE_SELECT) return GKV_ERR_STATE;
+        e = launch_evict_select(p, s);
+        if (e == cudaSuccess) next = GKV_STAGE_COMPACT;
+    } else {
+        if (next != GKV_STAGE_COMPACT) return GKV_ERR_STATE;
+        e = launch_evict_compact(p, ctx->sm_count, s);
+        if (e == cudaSuccess) after_evict(ctx, l0, nl, false);
+    }
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GKV_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    return GKV_OK;
+}
+
+gkv_status gkv_decode_attn_host(gkv_ctx* ctx, int32_t layer, const void* q_host, const void* k_new_host,
+                                const void* v_new_host, void* out_host, void* stream) {
+    if (!ctx || !layer_ok(ctx, layer) || !q_host || !k_new_host || !v_new_host || !out_host) return GKV_ERR_INVALID_ARG;
+    if (!ctx->buf.staging) return GKV_ERR_INVALID_ARG;
+    int l0, nl;
+    layer_range(ctx, layer, &l0, &nl);
+    const gkv_config& c = ctx->cfg;
+    if (ctx->len[l0] >= ctx->C) return GKV_ERR_CAPACITY;
+    const size_t qb = (size_t)nl * c.batch * c.n_q_heads * kHeadDim * 2;
+    const size_t kb = (size_t)nl * c.batch * c.n_kv_heads * kHeadDim * 2;
+    uint8_t* st = static_cast<uint8_t*>(ctx->buf.staging);
+    uint8_t *dq = st, *dk = st + align_up(qb), *dv = dk + align_up(kb), *dout = dv + align_up(kb);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return GKV_ERR_CUDA;
+    const gkv_status r = gkv_decode_attn(ctx, layer, dq, dk, dv, dout, stream);
+    if (r != GKV_OK) return r;
+    if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return GKV_ERR_CUDA;
+    return GKV_OK;
+}
+
+gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host, int32_t* kept_idx_out_host,
+                          void* stream) {
+    if (!ctx || !layer_ok(ctx, layer)) return GKV_ERR_INVALID_ARG;
+    if (!ctx->buf.staging) return GKV_ERR_INVALID_ARG;
+    int l0, nl;
+    layer_range(ctx, layer, &l0, &nl);
+    const gkv_config& c = ctx->cfg;
+    const size_t qb = (size_t)nl * c.batch * c.n_q_heads * c.window * kHeadDim * 2;
+    const size_t kb = (size_t)nl * c.batch * c.n_kv_heads * c.budget * 4;
+    uint8_t* st = static_cast<uint8_t*>(ctx->buf.staging);
+    uint8_t *dq = st, *dkept = st + align_up(qb);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (q_window_host && cudaMemcpyAsync(dq, q_window_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return GKV_ERR_CUDA;
+    const bool will_evict = ctx->len[l0] > c.budget;
+    const gkv_status r = gkv_evict(ctx, layer, q_window_host ? dq : nullptr,
+                                   kept_idx_out_host ? reinterpret_cast<int32_t*>(dkept) : nullptr, stream);
+    if (r != GKV_OK) return r;
+    if (kept_idx_out_host && will_evict &&
+        cudaMemcpyAsync(kept_idx_out_host, dkept, kb, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return GKV_ERR_CUDA;
+    return GKV_OK;
+}
+
+gkv_status gkv_get_state(const gkv_ctx* ctx, int32_t layer, int32_t* len, int32_t* n_hist, int32_t* since_evict) {
+    if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers) return GKV_ERR_INVALID_ARG;
+    if (len) *len = ctx->len[layer];
+    if (n_hist) *n_hist = ctx->n_hist[layer];
+    if (since_evict) *since_evict = ctx->since_evict[layer];
+    return GKV_OK;
+}
+
+int64_t gkv_launch_count(const gkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream) {
+    if (!ctx) return GKV_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t h[4] = {0, 0, 0, 0};
+    int32_t* d = ws_ptr<int32_t>(ctx, ctx->ws.status);
+    if (cudaMemcpyAsync(h, d, sizeof h, cudaMemcpyDeviceToHost, s) != cudaSuccess) return GKV_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return GKV_ERR_CUDA;
+    if (h[0] != 0) {
+        if (cudaMemsetAsync(d, 0, sizeof h, s) != cudaSuccess) return GKV_ERR_CUDA;
+        return GKV_ERR_TIMEOUT;
+    }
+    return GKV_OK;
+}
+
+gkv_status gkv_memory_model(const gkv_config* cfg, int64_t seq_len, int32_t elem_bytes, gkv_memory_model_t* out) {
+    if (!cfg || !out || seq_len <= 0 || elem_bytes <= 0) return GKV_ERR_INVALID_ARG;
+    if (cfg->n_layers <= 0 || cfg->batch <= 0 || cfg->n_kv_heads <= 0 || cfg->head_dim <= 0 || cfg->budget <= 0 ||
+        cfg->interval <= 0 || cfg->window < 0 || cfg->window >= cfg->budget)
+        return GKV_ERR_INVALID_ARG;
+    // K and V: layers x head_dim x kv_heads x tokens x elem_bytes x 2, times the batch
+    const uint64_t per_token = (uint64_t)cfg->n_layers * cfg->head_dim * cfg->n_kv_heads * elem_bytes * 2ull;
+    out->full_kv = per_token * (uint64_t)seq_len * cfg->batch;
+    out->compressed_kv = per_token * (uint64_t)(cfg->budget + cfg->interval) * cfg->batch;
+    out->score_cache = (uint64_t)cfg->n_layers * cfg->n_kv_heads * (uint64_t)(cfg->budget - cfg->window) *
+                       elem_bytes * cfg->batch;
+    return GKV_OK;
+}
+
+const char* gkv_strerror(gkv_status status) {
+    switch (status) {
+        case GKV_OK: return "ok";
+        case GKV_ERR_INVALID_ARG: return "invalid argument";
+        case GKV_ERR_STATE: return "call not allowed in the current schedule state";
+        case GKV_ERR_CAPACITY: return "cache full: evict before decoding further";
+        case GKV_ERR_CUDA: return "CUDA call failed";
+        case GKV_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case GKV_ERR_UNSUPPORTED: return "configuration not supported by this build";
+        default: return "unknown status";
+    }
+}
+
+void gkv_destroy(gkv_ctx* ctx) { delete ctx; }
+
+}  // extern "C"

@@ -1,0 +1,435 @@
+// GQA decode attention over the compressed cache, with the append of the current token and the
+// optional accumulation of the window score (the every-step half of the G-KV path).
+//
+// One CTA = one (unit, split), unit = (layer, sequence, KV head). A producer warp streams 64-key
+// K and V tiles (TMA, 128-byte swizzle) through a ring of stages; four consumer warps each own 16
+// keys of every tile and keep their own online-softmax state, so the main loop has no CTA-wide
+// barrier. Both products run on mma.sync m16n8k16 with the KEYS on the M side and the g <= 8 query
+// heads of the group on the N side (S^T = K Q^T, O^T = V^T P^T): no padded rows, each K/V byte
+// is read from shared memory exactly once, and the P^T operand comes from the S^T accumulator by
+// an 8x8 register transpose (movmatrix).
+#include "gkv_common.cuh"
+#include "gkv_internal.h"
+
+namespace gkv {
+
+constexpr int kConsumerWarps = 4;
+constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
+constexpr int kMaxStages = 6;
+constexpr int kPartFloats = 16 + kHeadDim * 8;  // M[8], L[8], acc[128][8]
+
+struct __align__(8) DecodeSmemTail {
+    uint64_t full_bar[kMaxStages];
+    uint64_t empty_bar[kMaxStages];
+    float m[kConsumerWarps][8];
+    float l[kConsumerWarps][8];
+    float fin_m[8];
+    float fin_l[8];
+    int abort_flag;
+    int issued;
+    int is_last;
+};
+
+__device__ __forceinline__ void latch_timeout(int32_t* status, int where) {
+    if (atomicCAS(status, 0, kStatusTimeout) == 0) {
+        status[1] = where;
+        status[2] = blockIdx.x;
+    }
+}
+
+__global__ void __launch_bounds__(kDecodeThreads)
+gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k,
+                  const __grid_constant__ CUtensorMap tm_v) {
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment for the swizzled TMA boxes
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int stages = p.stages;
+    uint8_t* stage_base = smem;
+    float* s_log = reinterpret_cast<float*>(smem + (size_t)stages * kStageBytes);  // [C][8] when accum && splits == 1
+    const size_t log_bytes = (p.accum && p.splits == 1) ? (size_t)((p.C + 63) & ~63) * 32 : 0;
+    DecodeSmemTail* tail = reinterpret_cast<DecodeSmemTail*>(smem + (size_t)stages * kStageBytes + log_bytes);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int unit_local = blockIdx.x / p.splits;
+    const int split = blockIdx.x - unit_local * p.splits;
+    const int head = unit_local % p.h_kv;
+    const int ls = unit_local / p.h_kv;              // layer_local * batch + seq
+    const int layer_local = ls / p.batch;
+    const int seq = ls - layer_local * p.batch;
+    const int layer = p.layer0 + layer_local;
+    const int lseq_global = layer * p.batch + seq;
+    const long unit = (long)lseq_global * p.h_kv + head;
+
+    const int len_old = p.len[lseq_global];
+    const int n = len_old + 1;                        // keys attended (current token included)
+    const int tiles_total = (n + kTileKeys - 1) / kTileKeys;
+    const int tps = (tiles_total + p.splits - 1) / p.splits;
+    const int t_begin = min(split * tps, tiles_total);
+    const int t_end = min(t_begin + tps, tiles_total);
+    const int row0 = (int)(unit * p.C);               // first cache row of this unit in the 2-D view
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(smem_u32(&tail->full_bar[s]), 1);
+            mbar_init(smem_u32(&tail->empty_bar[s]), kConsumerWarps);
+        }
+        tail->abort_flag = 0;
+        tail->issued = t_begin;
+        tail->is_last = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    // per-thread softmax / output state of a consumer warp (heads h0 = 2*(lane&3), h0+1)
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float acc[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            prefetch_tensormap(&tm_k);
+            prefetch_tensormap(&tm_v);
+            for (int it = t_begin; it < t_end; ++it) {
+                const int j = it - t_begin;
+                const int s = j % stages;
+                if (j >= stages) {
+                    if (!mbar_wait_bounded(smem_u32(&tail->empty_bar[s]), ((j / stages) - 1) & 1)) {
+                        latch_timeout(p.status, 1);
+                        tail->abort_flag = 1;
+                        break;
+                    }
+                }
+                if (*(volatile int*)&tail->abort_flag) break;
+                const uint32_t bar = smem_u32(&tail->full_bar[s]);
+                const uint32_t dst = smem_u32(stage_base + (size_t)s * kStageBytes);
+                const int y = row0 + it * kTileKeys;
+                mbar_arrive_expect_tx(bar, kStageBytes);
+                tma_load_2d(dst, &tm_k, 0, y, bar);
+                tma_load_2d(dst + kBoxBytes, &tm_k, 64, y, bar);
+                tma_load_2d(dst + kTileBytes, &tm_v, 0, y, bar);
+                tma_load_2d(dst + kTileBytes + kBoxBytes, &tm_v, 64, y, bar);
+                *(volatile int*)&tail->issued = it + 1;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumers
+        const int r_in = lane & 7, mat = lane >> 3;
+        const int hq = lane >> 2;                     // head whose Q row this lane holds (B operand)
+        // Q^T fragments: B[k = d][n = head], two packed bf16 pairs per 16-wide k step
+        uint32_t qf[8][2];
+        {
+            const __nv_bfloat16* qrow =
+                p.q + ((size_t)(layer_local * p.batch + seq) * p.h_q + (size_t)head * p.g + hq) * kHeadDim;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                if (hq < p.g) {
+                    qf[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + (lane & 3) * 2);
+                    qf[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + (lane & 3) * 2 + 8);
+                } else {
+                    qf[ks][0] = qf[ks][1] = 0u;
+                }
+            }
+        }
+        const int krow = warp * 16 + (mat & 1) * 8 + r_in;   // K ldmatrix: row this lane addresses
+        const int kch = mat >> 1;                             //   and which 16-byte chunk of the k step
+        const int vrow = warp * 16 + (mat >> 1) * 8 + r_in;   // V ldmatrix (transposed)
+        const int vch = mat & 1;
+
+        for (int it = t_begin; it < t_end; ++it) {
+            const int j = it - t_begin;
+            const int s = j % stages;
+            if (!mbar_wait_bounded(smem_u32(&tail->full_bar[s]), (j / stages) & 1)) {
+                latch_timeout(p.status, 2);
+                tail->abort_flag = 1;
+                break;
+            }
+            if (*(volatile int*)&tail->abort_flag) break;
+            uint8_t* kt = stage_base + (size_t)s * kStageBytes;
+            uint8_t* vt = kt + kTileBytes;
+            const int key0 = it * kTileKeys + warp * 16;
+            if (key0 < n) {
+                // append: the warp that owns row len_old overwrites it (in the tile and in the cache)
+                if (len_old >= key0 && len_old < key0 + 16) {
+                    const int lr = len_old - it * kTileKeys;          // row inside the tile
+                    const int c = lane & 15;
+                    const size_t src = ((size_t)(layer_local * p.batch + seq) * p.h_kv + head) * kHeadDim + c * 8;
+                    const size_t dstg = ((size_t)unit * p.C + len_old) * kHeadDim + c * 8;
+                    if (lane < 16) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(p.k_new + src);
+                        *reinterpret_cast<uint4*>(kt + tile_off(lr, c)) = x;
+                        *reinterpret_cast<uint4*>(p.k_cache + dstg) = x;
+                    } else {
+                        const uint4 x = *reinterpret_cast<const uint4*>(p.v_new + src);
+                        *reinterpret_cast<uint4*>(vt + tile_off(lr, c)) = x;
+                        *reinterpret_cast<uint4*>(p.v_cache + dstg) = x;
+                    }
+                    fence_proxy_async_smem();
+                }
+                // rows past the end of the cache may hold anything: zero the V rows so 0 * x stays 0
+                if (key0 + 16 > n) {
+                    const int first = n - it * kTileKeys;             // first invalid row of the tile
+                    for (int e = lane; e < (warp * 16 + 16 - first) * 16; e += 32) {
+                        const int lr = first + (e >> 4);
+                        *reinterpret_cast<uint4*>(vt + tile_off(lr, e & 15)) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+                __syncwarp();
+
+                // S^T[16 keys x 8 heads] = K_tile Q^T, two accumulators to halve the dependent chain
+                float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint32_t kaddr = smem_u32(kt);
+#pragma unroll
+                for (int ks = 0; ks < 8; ks += 2) {
+                    uint32_t a[4], a2[4];
+                    ldmatrix_x4(kaddr + tile_off(krow, ks * 2 + kch), a);
+                    ldmatrix_x4(kaddr + tile_off(krow, ks * 2 + 2 + kch), a2);
+                    mma_bf16_16816(sa, a, qf[ks][0], qf[ks][1]);
+                    mma_bf16_16816(sb, a2, qf[ks + 1][0], qf[ks + 1][1]);
+                }
+                const int key_a = key0 + (lane >> 2), key_b = key_a + 8;
+                float s0 = (sa[0] + sb[0]) * p.scale_log2, s1 = (sa[1] + sb[1]) * p.scale_log2;
+                float s2 = (sa[2] + sb[2]) * p.scale_log2, s3 = (sa[3] + sb[3]) * p.scale_log2;
+                if (key_a >= n) s0 = s1 = -INFINITY;
+                if (key_b >= n) s2 = s3 = -INFINITY;
+                if (p.accum) {
+                    const int h0 = (lane & 3) * 2;
+                    if (p.splits == 1) {
+                        if (key_a < n) *reinterpret_cast<float2*>(s_log + key_a * 8 + h0) = make_float2(s0, s1);
+                        if (key_b < n) *reinterpret_cast<float2*>(s_log + key_b * 8 + h0) = make_float2(s2, s3);
+                    } else {
+                        float* g_log = p.logits + (size_t)unit_local * p.C * 8;
+                        if (key_a < n) *reinterpret_cast<float2*>(g_log + key_a * 8 + h0) = make_float2(s0, s1);
+                        if (key_b < n) *reinterpret_cast<float2*>(g_log + key_b * 8 + h0) = make_float2(s2, s3);
+                    }
+                }
+                // tile maximum per head over the warp's 16 keys (lanes sharing lane & 3)
+                float t0 = fmaxf(s0, s2), t1 = fmaxf(s1, s3);
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) {
+                    t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, o));
+                    t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, o));
+                }
+                const float mn0 = fmaxf(m0, t0), mn1 = fmaxf(m1, t1);
+                const float sc0 = fast_exp2(m0 - mn0), sc1 = fast_exp2(m1 - mn1);
+                m0 = mn0; m1 = mn1;
+                const float p0 = fast_exp2(s0 - mn0), p1 = fast_exp2(s1 - mn1);
+                const float p2 = fast_exp2(s2 - mn0), p3 = fast_exp2(s3 - mn1);
+                l0 = l0 * sc0 + p0 + p2;
+                l1 = l1 * sc1 + p1 + p3;
+                if (__any_sync(0xffffffffu, (sc0 != 1.f) | (sc1 != 1.f))) {
+#pragma unroll
+                    for (int dt = 0; dt < 8; ++dt) {
+                        acc[dt][0] *= sc0; acc[dt][1] *= sc1; acc[dt][2] *= sc0; acc[dt][3] *= sc1;
+                    }
+                }
+                // P^T operand: transpose the two 8x8 (key x head) blocks in registers
+                const uint32_t b0 = movmatrix_trans(pack_bf16x2(p0, p1));
+                const uint32_t b1 = movmatrix_trans(pack_bf16x2(p2, p3));
+                const uint32_t vaddr = smem_u32(vt);
+#pragma unroll
+                for (int dt = 0; dt < 8; ++dt) {
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(vaddr + tile_off(vrow, dt * 2 + vch), a);
+                    mma_bf16_16816(acc[dt], a, b0, b1);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tail->empty_bar[s]));
+        }
+    }
+
+    __syncthreads();  // [A] every consumer is done with the stage buffers
+    if (*(volatile int*)&tail->abort_flag) {
+        // Give copies that are still in flight a bounded time to land before the CTA exits.
+        if (tid == 0) {
+            const int issued = *(volatile int*)&tail->issued;
+            for (int it = max(t_begin, issued - stages); it < issued; ++it) {
+                const int j = it - t_begin;
+                mbar_wait_bounded(smem_u32(&tail->full_bar[j % stages]), (j / stages) & 1);
+            }
+        }
+        return;
+    }
+
+    float* s_acc = reinterpret_cast<float*>(stage_base);  // [warp][128 dims][8 heads], aliases stage 0
+    if (warp < kConsumerWarps) {
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+            l0 += __shfl_xor_sync(0xffffffffu, l0, o);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+        }
+        const int h0 = (lane & 3) * 2;
+        if ((lane >> 2) == 0) {
+            tail->m[warp][h0] = m0; tail->m[warp][h0 + 1] = m1;
+            tail->l[warp][h0] = l0; tail->l[warp][h0 + 1] = l1;
+        }
+        float* dst = s_acc + warp * (kHeadDim * 8);
+#pragma unroll
+        for (int dt = 0; dt < 8; ++dt) {
+            const int dim = dt * 16 + (lane >> 2);
+            *reinterpret_cast<float2*>(dst + dim * 8 + h0) = make_float2(acc[dt][0], acc[dt][1]);
+            *reinterpret_cast<float2*>(dst + (dim + 8) * 8 + h0) = make_float2(acc[dt][2], acc[dt][3]);
+        }
+    }
+    __syncthreads();  // [B]
+
+    // CTA-level state: M, L per head and the merged accumulator column of this thread's dim
+    float o[8], M[8], L[8];
+    if (tid < kHeadDim) {
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+            float mm = tail->m[0][h];
+#pragma unroll
+            for (int w = 1; w < kConsumerWarps; ++w) mm = fmaxf(mm, tail->m[w][h]);
+            float ll = 0.f, oo = 0.f;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) {
+                const float wm = tail->m[w][h];
+                const float wgt = (wm == -INFINITY) ? 0.f : fast_exp2(wm - mm);
+                ll += wgt * tail->l[w][h];
+                oo += wgt * s_acc[w * (kHeadDim * 8) + tid * 8 + h];
+            }
+            M[h] = mm; L[h] = ll; o[h] = oo;
+        }
+    }
+
+    const int n_keys_all = n;
+    bool do_final = true;          // this CTA writes the output (always true without split)
+    if (p.splits > 1) {
+        float* mine = p.part + ((size_t)unit_local * p.splits + split) * kPartFloats;
+        if (tid < kHeadDim) {
+            if (tid < 8) { mine[tid] = M[tid]; mine[8 + tid] = L[tid]; }
+            float4* d4 = reinterpret_cast<float4*>(mine + 16 + tid * 8);
+            d4[0] = make_float4(o[0], o[1], o[2], o[3]);
+            d4[1] = make_float4(o[4], o[5], o[6], o[7]);
+        }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            const int prev = atomicAdd(&p.unit_done[unit], 1);
+            tail->is_last = (prev == p.splits - 1);
+            if (prev == p.splits - 1) p.unit_done[unit] = 0;   // self-reset for the next launch
+        }
+        __syncthreads();
+        do_final = tail->is_last != 0;
+        if (do_final) {
+            __threadfence();
+            if (tid < kHeadDim) {
+                const float* base = p.part + (size_t)unit_local * p.splits * kPartFloats;
+#pragma unroll
+                for (int h = 0; h < 8; ++h) {
+                    float mm = -INFINITY;
+                    for (int sp = 0; sp < p.splits; ++sp) mm = fmaxf(mm, __ldcg(base + sp * kPartFloats + h));
+                    float ll = 0.f, oo = 0.f;
+                    for (int sp = 0; sp < p.splits; ++sp) {
+                        const float wm = __ldcg(base + sp * kPartFloats + h);
+                        const float wgt = (wm == -INFINITY) ? 0.f : fast_exp2(wm - mm);
+                        ll += wgt * __ldcg(base + sp * kPartFloats + 8 + h);
+                        oo += wgt * __ldcg(base + sp * kPartFloats + 16 + tid * 8 + h);
+                    }
+                    M[h] = mm; L[h] = ll; o[h] = oo;
+                }
+            }
+        }
+    }
+
+    if (do_final) {
+        if (tid < kHeadDim) {
+            __nv_bfloat16* orow = p.out + ((size_t)(layer_local * p.batch + seq) * p.h_q + (size_t)head * p.g) * kHeadDim + tid;
+#pragma unroll
+            for (int h = 0; h < 8; ++h)
+                if (h < p.g) orow[(size_t)h * kHeadDim] = __float2bfloat16_rn(o[h] / L[h]);
+            if (tid < 8) { tail->fin_m[tid] = M[tid]; tail->fin_l[tid] = L[tid]; }
+        }
+        if (p.accum) {
+            __syncthreads();
+            // Sacc[t] += max over the group of the final weights = exp2(max_h (z_h[t] - M_h - log2 L_h))
+            float c[8];
+#pragma unroll
+            for (int h = 0; h < 8; ++h) c[h] = (h < p.g) ? tail->fin_m[h] + log2f(tail->fin_l[h]) : INFINITY;
+            float* sacc = p.sacc + (size_t)unit * p.C;
+            const float* g_log = p.logits + (size_t)unit_local * p.C * 8;
+            for (int t = tid; t < n_keys_all; t += kDecodeThreads) {
+                float4 x0, x1;
+                if (p.splits == 1) {
+                    x0 = *reinterpret_cast<const float4*>(s_log + t * 8);
+                    x1 = *reinterpret_cast<const float4*>(s_log + t * 8 + 4);
+                } else {
+                    x0 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8));
+                    x1 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8 + 4));
+                }
+                float v = x0.x - c[0];
+                v = fmaxf(v, x0.y - c[1]); v = fmaxf(v, x0.z - c[2]); v = fmaxf(v, x0.w - c[3]);
+                v = fmaxf(v, x1.x - c[4]); v = fmaxf(v, x1.y - c[5]); v = fmaxf(v, x1.z - c[6]);
+                v = fmaxf(v, x1.w - c[7]);
+                sacc[t] += fast_exp2(v);
+            }
+        }
+    }
+
+    // The last CTA of a (layer, sequence) publishes the new length.
+    __syncthreads();
+    if (tid == 0) {
+        const int per_seq = p.h_kv * p.splits;
+        const int prev = atomicAdd(&p.seq_done[lseq_global], 1);
+        if (prev == per_seq - 1) {
+            p.seq_done[lseq_global] = 0;
+            p.len[lseq_global] = n;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+static size_t decode_smem_bytes(int C, int accum, int splits, int stages) {
+    const size_t log_bytes = (accum && splits == 1) ? (size_t)((C + 63) & ~63) * 32 : 0;
+    return 1024 + (size_t)stages * kStageBytes + log_bytes + sizeof(DecodeSmemTail);
+}
+
+int decode_pick_splits(int units_in_launch, int C, int sm_count) {
+    const int max_tiles = (C + kTileKeys - 1) / kTileKeys;
+    const int want = 4 * sm_count;  // enough CTAs for two per SM, twice over
+    if (units_in_launch >= 2 * sm_count) return 1;
+    int s = (want + units_in_launch - 1) / units_in_launch;
+    if (s > max_tiles) s = max_tiles;
+    if (s > 32) s = 32;
+    if (s < 1) s = 1;
+    return s;
+}
+
+// Most bytes in flight per SM: stages per CTA x CTAs per SM, within 227 KB of shared memory.
+// Ties go to the earlier entry of the preference order (3 stages first).
+int decode_pick_stages(int C, int accum, int splits, size_t* smem_bytes) {
+    const size_t cap = 227 * 1024;
+    const int order[5] = {3, 4, 2, 5, 6};
+    int best = 2;
+    size_t best_flight = 0;
+    for (int i = 0; i < 5; ++i) {
+        const int st = order[i];
+        const size_t b = decode_smem_bytes(C, accum, splits, st);
+        if (b > cap) continue;
+        size_t ctas = cap / (b + 1024);  // 1 KB per-CTA reservation
+        if (ctas > 4) ctas = 4;
+        const size_t flight = ctas * (size_t)st;
+        if (flight > best_flight) {
+            best_flight = flight;
+            best = st;
+        }
+    }
+    if (smem_bytes) *smem_bytes = decode_smem_bytes(C, accum, splits, best);
+    return best;
+}
+
+cudaError_t decode_kernel_setup() {
+    return cudaFuncSetAttribute(gkv_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+}
+
+cudaError_t launch_decode(const DecodeLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v, cudaStream_t s) {
+    const size_t smem = decode_smem_bytes(p.C, p.accum, p.splits, p.stages);
+    const int grid = p.n_layers * p.batch * p.h_kv * p.splits;
+    gkv_decode_kernel<<<grid, kDecodeThreads, smem, s>>>(p, tm_k, tm_v);
+    return cudaGetLastError();
+}
+
+}  // namespace gkv

@@ -1,0 +1,362 @@
+// The compression step after scoring: max-normalise the local score, merge it with the decayed
+// history into the global score (Section 5, Eq. 3-5), select the top-(b-w) candidates per KV head
+// (ties toward the lower position), and compact K, V, F and pos in place.
+//
+// One CTA owns one unit (layer, sequence, KV head). All per-row score state of a unit (at most
+// C <= 4096 rows) lives in shared memory. The selection is a 4-pass radix select on the fp32 bit
+// patterns (scores are >= 0, so they order as unsigned integers) followed by one ordered scan that
+// assigns destinations. The compaction moves rows in ascending order, a group of rows fully loaded
+// into registers before any of them is stored: a row's destination never lies above its source,
+// so earlier groups can only overwrite rows that are already consumed.
+#include "gkv_common.cuh"
+#include "gkv_internal.h"
+
+namespace gkv {
+
+constexpr int kEvictThreads = 256;
+constexpr int kCompactUnroll = 4;
+
+struct EvictShared {
+    int hist[256];
+    int warp_sums[8];
+    float warp_max[8];
+    int digit, k_rem, first_evicted, is_last;
+};
+
+// inclusive prefix sum over the 256 threads of the CTA
+__device__ __forceinline__ int block_incl_scan(int v, int* warp_sums, int tid) {
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    if (lane == 31) warp_sums[warp] = v;
+    __syncthreads();
+    int base = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) base += (i < warp) ? warp_sums[i] : 0;
+    __syncthreads();
+    return v + base;
+}
+
+__device__ __forceinline__ float block_max(float v, float* warp_max, int tid) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if ((tid & 31) == 0) warp_max[tid >> 5] = v;
+    __syncthreads();
+    float r = warp_max[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) r = fmaxf(r, warp_max[i]);
+    __syncthreads();
+    return r;
+}
+
+// Section 5: S_hat = S / max S over the n_c candidates; F = merge(alpha * F_prev, S_hat) on the
+// n_h rows with history, F = S_hat elsewhere. `s_f` receives F for t < n_c.
+// `sums` holds w * S (the 1/w of Eq. 2 cancels in the normalisation).
+__device__ void merge_phase(const float* __restrict__ sums, const float* __restrict__ f_prev, float* s_f,
+                            int n_c, int n_h, float alpha, int mode, EvictShared* sh, int tid) {
+    float mx = 0.f;
+    for (int t = tid; t < n_c; t += kEvictThreads) {
+        const float s = sums[t];
+        s_f[t] = s;
+        mx = fmaxf(mx, s);
+    }
+    mx = block_max(mx, sh->warp_max, tid);
+    for (int t = tid; t < n_c; t += kEvictThreads) {
+        const float shat = (mx > 0.f) ? __fdiv_rn(s_f[t], mx) : 0.f;
+        float f = shat;
+        if (t < n_h && mode != GKV_MODE_LOCAL) {
+            const float fp = alpha * f_prev[t];
+            if (mode == GKV_MODE_MAX) f = fmaxf(fp, shat);
+            else if (mode == GKV_MODE_MEAN) f = fp + (1.f - alpha) * shat;
+            else f = fp + shat;
+        }
+        s_f[t] = f;
+    }
+    __syncthreads();
+}
+
+// Top-n_keep of s_f[0..n_c) with ties toward the lower index; kept rows ascending into s_kept,
+// followed by the w window rows n_c .. n_c+w-1. Returns (CTA-uniform) the first row that moves.
+__device__ int select_phase(const float* s_f, int* s_kept, int n_c, int n_keep, int w, EvictShared* sh, int tid) {
+    const uint32_t* bits = reinterpret_cast<const uint32_t*>(s_f);
+    uint32_t prefix = 0;
+    int k = n_keep;
+#pragma unroll 1
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        sh->hist[tid] = 0;
+        __syncthreads();
+        const uint32_t mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
+        for (int t = tid; t < n_c; t += kEvictThreads) {
+            const uint32_t x = bits[t];
+            if ((x & mask) == prefix) atomicAdd(&sh->hist[(x >> shift) & 255], 1);
+        }
+        __syncthreads();
+        // thread tid looks at digit 255 - tid; `ge` = number of matching elements with digit >= mine
+        const int mine = sh->hist[255 - tid];
+        const int ge = block_incl_scan(mine, sh->warp_sums, tid);
+        const int gt = ge - mine;
+        if (ge >= k && gt < k) {  // exactly one digit holds the k-th largest
+            sh->digit = 255 - tid;
+            sh->k_rem = k - gt;
+        }
+        __syncthreads();
+        prefix |= static_cast<uint32_t>(sh->digit) << shift;
+        k = sh->k_rem;
+    }
+    // prefix = bit pattern T of the n_keep-th largest score; take everything above it and the
+    // first k rows equal to it
+    const uint32_t T = prefix;
+    const int per = (n_c + kEvictThreads - 1) / kEvictThreads;
+    const int t0 = tid * per, t1 = min(t0 + per, n_c);
+    int gt = 0, eq = 0;
+    for (int t = t0; t < t1; ++t) {
+        const uint32_t x = bits[t];
+        gt += (x > T);
+        eq += (x == T);
+    }
+    if (tid == 0) sh->first_evicted = n_c;
+    const int packed = block_incl_scan(gt | (eq << 16), sh->warp_sums, tid);  // counts < 65536 each
+    int gt_before = (packed & 0xffff) - gt, eq_before = (packed >> 16) - eq;
+    int first_drop = n_c;
+    for (int t = t0; t < t1; ++t) {
+        const uint32_t x = bits[t];
+        if (x > T) {
+            s_kept[gt_before + min(eq_before, k)] = t;
+            ++gt_before;
+        } else if (x == T) {
+            if (eq_before < k) s_kept[gt_before + eq_before] = t;
+            else first_drop = min(first_drop, t);
+            ++eq_before;
+        } else {
+            first_drop = min(first_drop, t);
+        }
+    }
+    if (first_drop < n_c) atomicMin(&sh->first_evicted, first_drop);
+    for (int r = tid; r < w; r += kEvictThreads) s_kept[n_keep + r] = n_c + r;
+    __syncthreads();
+    return sh->first_evicted;
+}
+
+// Move the rows kept[r] -> r for r in [r_first, b) of one unit's K and V, restricted to the
+// 16-byte chunks [chunk0, chunk0 + cpr) of every row (cpr divides 16).
+__device__ void compact_phase(__nv_bfloat16* kbase, __nv_bfloat16* vbase, const int* kept, int b, int r_first,
+                              int chunk0, int cpr, int tid) {
+    const int rows_per_pass = kEvictThreads / cpr;
+    const int my_r = tid / cpr;
+    const int my_c = chunk0 + (tid - my_r * cpr);
+    uint4* k4 = reinterpret_cast<uint4*>(kbase);
+    uint4* v4 = reinterpret_cast<uint4*>(vbase);
+    for (int r0 = r_first; r0 < b; r0 += kCompactUnroll * rows_per_pass) {
+        uint4 kx[kCompactUnroll], vx[kCompactUnroll];
+        int src[kCompactUnroll];
+#pragma unroll
+        for (int u = 0; u < kCompactUnroll; ++u) {
+            const int r = r0 + u * rows_per_pass + my_r;
+            src[u] = (r < b) ? kept[r] : -1;
+            if (src[u] >= 0) {
+                kx[u] = k4[(size_t)src[u] * 16 + my_c];
+                vx[u] = v4[(size_t)src[u] * 16 + my_c];
+            }
+        }
+        __syncthreads();  // the whole group is in registers before any of its rows is overwritten
+#pragma unroll
+        for (int u = 0; u < kCompactUnroll; ++u) {
+            const int r = r0 + u * rows_per_pass + my_r;
+            if (src[u] >= 0) {
+                k4[(size_t)r * 16 + my_c] = kx[u];
+                v4[(size_t)r * 16 + my_c] = vx[u];
+            }
+        }
+    }
+}
+
+struct UnitIndex {
+    int unit_local, lseq_global;
+    long unit;
+};
+__device__ __forceinline__ UnitIndex unit_of(const EvictLaunch& p, int unit_local) {
+    UnitIndex u;
+    u.unit_local = unit_local;
+    const int ls = unit_local / p.h_kv;
+    const int head = unit_local - ls * p.h_kv;
+    u.lseq_global = p.layer0 * p.batch + ls;
+    u.unit = (long)u.lseq_global * p.h_kv + head;
+    return u;
+}
+
+// Record the per-row state after selection: compact F and pos, clear the window sums, export kept.
+__device__ void write_score_state(const EvictLaunch& p, const UnitIndex& u, const float* s_f, const int* s_kept,
+                                  int* s_pos, int n, int tid) {
+    const int n_keep = p.b - p.w;
+    float* f = p.f + (size_t)u.unit * p.C;
+    for (int r = tid; r < p.C; r += kEvictThreads) f[r] = (r < n_keep) ? s_f[s_kept[r]] : 0.f;
+    if (p.pos) {
+        int32_t* pos = p.pos + (size_t)u.unit * p.C;
+        for (int t = tid; t < n; t += kEvictThreads) s_pos[t] = pos[t];
+        __syncthreads();
+        for (int r = tid; r < p.b; r += kEvictThreads) pos[r] = s_pos[s_kept[r]];
+    }
+    float* sacc = p.sacc + (size_t)u.unit * p.C;
+    for (int t = tid; t < p.C; t += kEvictThreads) sacc[t] = 0.f;
+    if (p.kept_out) {
+        int32_t* ko = p.kept_out + (size_t)u.unit_local * p.b;
+        for (int r = tid; r < p.b; r += kEvictThreads) ko[r] = s_kept[r];
+    }
+}
+
+// The last CTA of a (layer, sequence) publishes len = b and n_hist = b - w.
+__device__ void publish_state(const EvictLaunch& p, const UnitIndex& u, int ctas_per_seq, EvictShared* sh, int tid) {
+    __syncthreads();
+    if (tid == 0) {
+        const int prev = atomicAdd(&p.seq_done[u.lseq_global], 1);
+        if (prev == ctas_per_seq - 1) {
+            p.seq_done[u.lseq_global] = 0;
+            p.len[u.lseq_global] = p.b;
+            p.len[(size_t)p.L_total * p.batch + u.lseq_global] = p.b - p.w;
+        }
+    }
+}
+
+__device__ __forceinline__ void carve(uint8_t* smem, const EvictLaunch& p, float** s_f, int** s_kept, int** s_pos,
+                                      EvictShared** sh) {
+    *sh = reinterpret_cast<EvictShared*>(smem);
+    *s_f = reinterpret_cast<float*>(smem + sizeof(EvictShared));
+    *s_kept = reinterpret_cast<int*>(*s_f + p.C);
+    *s_pos = *s_kept + p.b;
+}
+static size_t evict_smem_bytes(const EvictLaunch& p) {
+    return sizeof(EvictShared) + sizeof(float) * p.C + sizeof(int) * p.b + (p.pos ? sizeof(int) * p.C : 0);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Whole step in one launch: merge -> select -> score-state update -> K/V compaction.
+__global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const EvictLaunch p) {
+    extern __shared__ __align__(16) uint8_t evict_smem[];
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
+    const int tid = threadIdx.x;
+    const UnitIndex u = unit_of(p, blockIdx.x);
+    const int n = p.len[u.lseq_global];
+    const int n_h = p.len[(size_t)p.L_total * p.batch + u.lseq_global];
+    if (n <= p.b) {  // nothing to evict: only the window sums restart
+        float* sacc = p.sacc + (size_t)u.unit * p.C;
+        for (int t = tid; t < p.C; t += kEvictThreads) sacc[t] = 0.f;
+        return;
+    }
+    const int n_c = n - p.w;
+    merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
+    const int r_first = select_phase(s_f, s_kept, n_c, p.b - p.w, p.w, sh, tid);
+    write_score_state(p, u, s_f, s_kept, s_pos, n, tid);
+    compact_phase(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
+                  p.b, r_first, 0, 16, tid);
+    publish_state(p, u, p.h_kv, sh, tid);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same step as separate launches (timed one by one); they hand over through the workspace.
+__global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const EvictLaunch p) {
+    extern __shared__ __align__(16) uint8_t evict_smem[];
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
+    const int tid = threadIdx.x;
+    const UnitIndex u = unit_of(p, blockIdx.x);
+    const int n = p.len[u.lseq_global];
+    const int n_h = p.len[(size_t)p.L_total * p.batch + u.lseq_global];
+    if (n <= p.b) return;
+    const int n_c = n - p.w;
+    merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
+    float* out = p.f_ws + (size_t)u.unit_local * p.C;
+    for (int t = tid; t < n_c; t += kEvictThreads) out[t] = s_f[t];
+}
+
+__global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const EvictLaunch p) {
+    extern __shared__ __align__(16) uint8_t evict_smem[];
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
+    const int tid = threadIdx.x;
+    const UnitIndex u = unit_of(p, blockIdx.x);
+    const int n = p.len[u.lseq_global];
+    if (n <= p.b) {
+        float* sacc = p.sacc + (size_t)u.unit * p.C;
+        for (int t = tid; t < p.C; t += kEvictThreads) sacc[t] = 0.f;
+        return;
+    }
+    const int n_c = n - p.w;
+    const float* in = p.f_ws + (size_t)u.unit_local * p.C;
+    for (int t = tid; t < n_c; t += kEvictThreads) s_f[t] = in[t];
+    __syncthreads();
+    select_phase(s_f, s_kept, n_c, p.b - p.w, p.w, sh, tid);
+    write_score_state(p, u, s_f, s_kept, s_pos, n, tid);
+    int32_t* kw = p.kept_ws + (size_t)u.unit_local * p.b;
+    for (int r = tid; r < p.b; r += kEvictThreads) kw[r] = s_kept[r];
+}
+
+// grid = units x slices: each CTA moves one column slice of every row of its unit.
+__global__ void __launch_bounds__(kEvictThreads) gkv_evict_compact_kernel(const EvictLaunch p, int slices) {
+    extern __shared__ __align__(16) uint8_t evict_smem[];
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
+    const int tid = threadIdx.x;
+    const int unit_local = blockIdx.x / slices, slice = blockIdx.x - unit_local * slices;
+    const UnitIndex u = unit_of(p, unit_local);
+    const int n = p.len[u.lseq_global];
+    if (n <= p.b) return;
+    if (tid == 0) sh->first_evicted = p.b;
+    __syncthreads();
+    const int32_t* kw = p.kept_ws + (size_t)unit_local * p.b;
+    int first = p.b;
+    for (int r = tid; r < p.b; r += kEvictThreads) {
+        const int s = kw[r];
+        s_kept[r] = s;
+        if (s != r) first = min(first, r);
+    }
+    if (first < p.b) atomicMin(&sh->first_evicted, first);
+    __syncthreads();
+    const int cpr = 16 / slices;
+    compact_phase(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
+                  p.b, sh->first_evicted, slice * cpr, cpr, tid);
+    publish_state(p, u, p.h_kv * slices, sh, tid);
+}
+
+// ---------------------------------------------------------------------------------------------
+static cudaError_t ensure_smem(const void* fn, size_t bytes) {
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s) {
+    const size_t smem = evict_smem_bytes(p);
+    cudaError_t e = ensure_smem((const void*)gkv_evict_fused_kernel, smem);
+    if (e != cudaSuccess) return e;
+    gkv_evict_fused_kernel<<<p.n_layers * p.batch * p.h_kv, kEvictThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s) {
+    const size_t smem = evict_smem_bytes(p);
+    cudaError_t e = ensure_smem((const void*)gkv_evict_merge_kernel, smem);
+    if (e != cudaSuccess) return e;
+    gkv_evict_merge_kernel<<<p.n_layers * p.batch * p.h_kv, kEvictThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+cudaError_t launch_evict_select(const EvictLaunch& p, cudaStream_t s) {
+    const size_t smem = evict_smem_bytes(p);
+    cudaError_t e = ensure_smem((const void*)gkv_evict_select_kernel, smem);
+    if (e != cudaSuccess) return e;
+    gkv_evict_select_kernel<<<p.n_layers * p.batch * p.h_kv, kEvictThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+cudaError_t launch_evict_compact(const EvictLaunch& p, int sm_count, cudaStream_t s) {
+    const size_t smem = evict_smem_bytes(p);
+    cudaError_t e = ensure_smem((const void*)gkv_evict_compact_kernel, smem);
+    if (e != cudaSuccess) return e;
+    const int units = p.n_layers * p.batch * p.h_kv;
+    int slices = 1;
+    while (slices < 16 && units * slices < 4 * sm_count) slices <<= 1;  // column slices for small batches
+    gkv_evict_compact_kernel<<<units * slices, kEvictThreads, smem, s>>>(p, slices);
+    return cudaGetLastError();
+}
+
+}  // namespace gkv

@@ -1,0 +1,100 @@
+// Host-side internals of the G-KV library: the context, the workspace layout and the kernel
+// launchers that the C-ABI entry points call.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "gkv.h"
+
+namespace gkv {
+
+// Offsets (bytes) of the regions of the caller-allocated workspace.
+struct WorkspaceLayout {
+    uint64_t status;      // int32[64]   latched device status + diagnostics
+    uint64_t seq_done;    // int32[L*batch]         CTA completion counters per (layer, sequence)
+    uint64_t unit_done;   // int32[L*batch*h_kv]    split completion counters per unit
+    uint64_t part;        // split-K partials: per (unit, split) M[8], L[8], acc[128][8] fp32
+    uint64_t logits;      // split-K window steps: per unit C x 8 fp32 scaled logits
+    uint64_t kept;        // int32[units_per_layer * b]   kept lists of the staged eviction path
+    uint64_t fscratch;    // fp32[units_per_layer * C]    merged scores of the staged eviction path
+    uint64_t total;
+};
+
+struct DecodeLaunch {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16* out;
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    float* sacc;
+    int32_t* len;        // plane 0 of the len buffer
+    int32_t* seq_done;
+    int32_t* unit_done;
+    float* part;
+    float* logits;
+    int32_t* status;
+    int layer0, n_layers, batch, h_q, h_kv, g, C;
+    int splits, stages, accum;
+    float scale_log2;    // log2(e) / sqrt(d)
+};
+
+struct EvictLaunch {
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    float* f;
+    float* sacc;
+    int32_t* pos;        // may be NULL
+    int32_t* len;        // plane 0; plane 1 (n_hist) follows at len + L_total*batch
+    int32_t* seq_done;
+    int32_t* kept_out;   // may be NULL: [units in launch][b]
+    int32_t* kept_ws;    // staged path scratch
+    float* f_ws;         // staged path scratch
+    int32_t* status;
+    int layer0, n_layers, L_total, batch, h_kv, C, b, w;
+    float alpha;
+    int mode;
+};
+
+struct ScoreLaunch {
+    const __nv_bfloat16* q_win;  // [n_layers][batch][h_q][w][d]
+    float* sacc;                 // receives w * S
+    const int32_t* len;
+    int32_t* status;
+    int layer0, n_layers, batch, h_q, h_kv, g, C, w;
+    float scale_log2;
+};
+
+}  // namespace gkv
+
+struct gkv_ctx {
+    gkv_config cfg;
+    gkv_buffers buf;
+    gkv::WorkspaceLayout ws;
+    int C, g, units_per_layer;
+    int device, sm_count;
+    CUtensorMap tm_k, tm_v;
+    std::vector<int32_t> len, n_hist, since_evict, sacc_valid, stage_next;
+    int64_t launches;
+    gkv_sizes sizes;
+};
+
+namespace gkv {
+
+int decode_pick_splits(int units_in_launch, int C, int sm_count);
+int decode_pick_stages(int C, int accum, int splits, size_t* smem_bytes);
+cudaError_t launch_decode(const DecodeLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v, cudaStream_t s);
+cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s);
+cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s);
+cudaError_t launch_evict_select(const EvictLaunch& p, cudaStream_t s);
+cudaError_t launch_evict_compact(const EvictLaunch& p, int sm_count, cudaStream_t s);
+cudaError_t launch_score(const ScoreLaunch& p, const CUtensorMap& tm_k, cudaStream_t s);
+cudaError_t decode_kernel_setup();
+cudaError_t score_kernel_setup();
+
+}  // namespace gkv

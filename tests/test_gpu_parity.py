@@ -1,0 +1,321 @@
+"""GPU parity: the CUDA library (through the C ABI) against the fp64 oracle, element by element
+on the same seeded inputs. Sizes span several 64-key tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2512_00504_b200 as gkv
+from paper_2512_00504_b200 import synth
+
+from parity import (DECODE_ATOL, SCORE_ATOL, SCORE_RTOL, check_evict_against_oracle, oracle_mode, snapshot)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def load_case(cache, case, layer=0, window_scores=None):
+    """Fill one layer of the cache with an EvictionCase and declare the state."""
+    cache.k[layer].copy_(case.k)
+    cache.v[layer].copy_(case.v)
+    cache.f[layer].copy_(case.f_prev)
+    if cache.pos is not None:
+        cache.pos[layer].copy_(case.pos)
+    if window_scores is not None:
+        cache.sacc[layer].copy_(window_scores)
+    cache.set_state(layer, case.l, case.n_h, cache.cfg.interval, window_scores is not None)
+
+
+# ------------------------------------------------------------------------- decode attention
+@pytest.mark.parametrize("shape", [
+    dict(batch=1, h_q=8, h_kv=2, b=160, buffer=40, w=8, s=40),      # split-K path, C = 200 (ragged tiles)
+    dict(batch=2, h_q=28, h_kv=4, b=96, buffer=32, w=16, s=32),     # g = 7
+    dict(batch=80, h_q=16, h_kv=4, b=130, buffer=30, w=8, s=30),    # 320 units: one CTA per unit, no split
+])
+def test_decode_attention_matches_oracle(shape):
+    cfg = gkv.make_config(n_layers=1, **shape, fuse_window_scores=False)
+    cache = gkv.GKVCache(cfg, DEV)
+    B, Hq, H, C = shape["batch"], shape["h_q"], shape["h_kv"], cache.C
+    gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 7)
+    rnd = lambda *s: torch.randn(*s, generator=gen, device=DEV).to(torch.bfloat16)
+    # prefill rows directly, then decode across tile boundaries and up to the last row
+    for start in (0, 60, C - 5):
+        cache.k[0, :, :, :start] = rnd(B, H, start, 128)
+        cache.v[0, :, :, :start] = rnd(B, H, start, 128)
+        cache.set_state(0, start, 0, 0)
+        K, V = synth.bits(cache.k[0]), synth.bits(cache.v[0])
+        out = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device=DEV)
+        for t in range(start, min(start + 6, C)):
+            q, kn, vn = rnd(B, Hq, 128), rnd(B, H, 128), rnd(B, H, 128)
+            cache.decode_attn(0, q, kn, vn, out)
+            K[:, :, t], V[:, :, t] = synth.bits(kn), synth.bits(vn)
+            sel = np.arange(B) if B <= 4 else np.array([0, 1, B // 2, B - 1])
+            ref = oracle.decode_batch(synth.bits(q)[sel], K[sel], V[sel], t + 1)
+            got = out.float().cpu().numpy()[sel]
+            assert np.abs(got - ref).max() < DECODE_ATOL, (start, t)
+            assert cache.state(0)[0] == t + 1
+        # the appended rows landed in the cache, bit for bit
+        assert (synth.bits(cache.k[0]) == K).all() and (synth.bits(cache.v[0]) == V).all()
+        assert int(cache.len[0].min()) == int(cache.len[0].max()) == min(start + 6, C)
+    cache.poll()
+    with pytest.raises(gkv.GKVError) as e:   # cache full
+        cache.decode_attn(0, q, kn, vn, out)
+    assert e.value.status == gkv.GKV_ERR_CAPACITY
+
+
+@pytest.mark.parametrize("shape", [
+    dict(batch=1, h_q=8, h_kv=2, b=150, buffer=50, w=16, s=50),     # split-K + window accumulation
+    dict(batch=75, h_q=28, h_kv=4, b=100, buffer=40, w=8, s=40),    # 300 units, shared-memory logits
+])
+def test_window_accumulation_matches_recomputed_local_score(shape):
+    """Fused window sums from w decode steps vs Eq. 1-2 recomputed by the oracle from the stored
+    window queries; and the recompute kernel vs the same."""
+    cfg = gkv.make_config(n_layers=1, **shape, fuse_window_scores=True)
+    cache = gkv.GKVCache(cfg, DEV)
+    B, Hq, H, C, w, s, b = shape["batch"], shape["h_q"], shape["h_kv"], cache.C, shape["w"], shape["s"], shape["b"]
+    gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 8)
+    rnd = lambda *sh: torch.randn(*sh, generator=gen, device=DEV).to(torch.bfloat16)
+    start = C - w
+    cache.k[0, :, :, :start] = rnd(B, H, start, 128)
+    cache.v[0, :, :, :start] = rnd(B, H, start, 128)
+    cache.set_state(0, start, 0, s - w)
+    qs = []
+    out = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device=DEV)
+    for t in range(w):
+        q, kn, vn = rnd(B, Hq, 128), rnd(B, H, 128), rnd(B, H, 128)
+        cache.decode_attn(0, q, kn, vn, out)
+        qs.append(q)
+    assert cache.state(0) == (C, 0, s)
+    q_win = torch.stack(qs, dim=2).contiguous()           # [B][Hq][w][d], oldest first
+    sel = list(range(B)) if B <= 4 else [0, B // 2, B - 1]
+    K = synth.bits(cache.k[0])
+    sacc = cache.sacc[0].cpu().numpy()
+    for n in sel:
+        S = oracle.window_mean(oracle.group_max(oracle.window_attention(synth.bits(q_win[n]), K[n], C), H))
+        np.testing.assert_allclose(sacc[n][:, :C] / w, S, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+    # the recompute kernel (score stage) must give the same sums
+    fused = cache.sacc[0].clone()
+    cache.evict_stage(0, gkv.GKV_STAGE_SCORE, q_win)
+    torch.cuda.synchronize()
+    cache.poll()
+    re = cache.sacc[0].cpu().numpy()
+    for n in sel:
+        S = oracle.window_mean(oracle.group_max(oracle.window_attention(synth.bits(q_win[n]), K[n], C), H))
+        np.testing.assert_allclose(re[n][:, :C] / w, S, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+    np.testing.assert_allclose(re, fused.cpu().numpy(), rtol=2 * SCORE_RTOL, atol=2 * SCORE_ATOL)
+    with pytest.raises(gkv.GKVError) as e:   # the cache is full and a compression is due
+        cache.decode_attn(0, q, kn, vn, out)
+    assert e.value.status == gkv.GKV_ERR_CAPACITY
+
+
+# ------------------------------------------------------------------------- eviction step
+def run_single_eviction(shape, seed, mode=gkv.GKV_MODE_MAX, alpha=0.8, n_h=None, l=None, recompute=True,
+                        track=True, staged=False, n_planted=8):
+    cfg = gkv.make_config(n_layers=1, **shape, alpha=alpha, mode=mode, fuse_window_scores=False, track_positions=track)
+    cache = gkv.GKVCache(cfg, DEV)
+    kw = {k: shape[k] for k in ("batch", "h_q", "h_kv", "b", "buffer", "w")}
+    case = synth.eviction_case(seed, **kw, l=l, n_h=n_h, n_planted=n_planted, device=DEV)
+    B, H, b = shape["batch"], shape["h_kv"], shape["b"]
+    sums = None
+    if not recompute:
+        # window sums computed by the oracle, stored as the fp32 state the kernel reads
+        S = np.stack([oracle.window_mean(oracle.group_max(
+            oracle.window_attention(synth.bits(case.q_win[n]), synth.bits(case.k[n]), case.l), H)) for n in range(B)])
+        sums = torch.zeros((B, H, cache.C), dtype=torch.float32, device=DEV)
+        sums[:, :, : case.l] = torch.from_numpy(S * shape["w"]).float().to(DEV)
+    load_case(cache, case, 0, sums)
+    seqs = list(range(B)) if B <= 4 else [0, B // 3, B - 1]
+    snap = snapshot(cache, 0, seqs)
+    kept = torch.full((B, H, b), -1, dtype=torch.int32, device=DEV)
+    qw = case.q_win if recompute else None
+    if staged:
+        if recompute:
+            cache.evict_stage(0, gkv.GKV_STAGE_SCORE, qw)
+        cache.evict_stage(0, gkv.GKV_STAGE_MERGE)
+        cache.evict_stage(0, gkv.GKV_STAGE_SELECT, None, kept)
+        cache.evict_stage(0, gkv.GKV_STAGE_COMPACT)
+    else:
+        cache.evict(0, qw, kept)
+    cache.poll()
+    assert cache.state(0) == (b, b - shape["w"], 0)
+    assert int(cache.len[0].min()) == int(cache.len[0].max()) == b
+    assert int(cache.len[1].min()) == int(cache.len[1].max()) == b - shape["w"]
+    assert float(cache.sacc.abs().max()) == 0.0          # window sums restart
+    kept_np = kept.cpu().numpy()[seqs]
+    q_bits = [synth.bits(case.q_win[n]) for n in seqs] if recompute else None
+    swaps = check_evict_against_oracle(cache, 0, seqs, snap, kept_np, l=case.l, n_h=case.n_h, q_win=q_bits)
+    return cache, case, kept.cpu().numpy(), swaps
+
+
+CONFIG0 = {k: v for k, v in synth.CONFIGS[0].items() if k != "n_layers" and k != "d"}
+
+
+@pytest.mark.parametrize("seed", [synth.BASE_SEED, synth.BASE_SEED + 1, synth.BASE_SEED + 2])
+def test_evict_config0_recompute(seed):
+    """Configuration 0: 8 q / 2 kv heads, l = 640, b = 512, w = 16, history on 496 rows."""
+    cache, case, kept, swaps = run_single_eviction(CONFIG0, seed)
+    assert swaps <= 2
+    for j in range(2):   # planted heavy hitters have ~e^4 times the weight of other keys: F = 1-ish, always kept
+        assert set(case.planted[0, j].tolist()) <= set(kept[0, j].tolist()) or cache.cfg.mode != gkv.GKV_MODE_LOCAL
+
+
+@pytest.mark.parametrize("mode", [gkv.GKV_MODE_MAX, gkv.GKV_MODE_MEAN, gkv.GKV_MODE_SUM, gkv.GKV_MODE_LOCAL])
+@pytest.mark.parametrize("recompute", [True, False])
+def test_evict_all_forms(mode, recompute):
+    shape = dict(batch=3, h_q=28, h_kv=4, b=200, buffer=56, w=16, s=56)   # g = 7, C = 256
+    run_single_eviction(shape, synth.BASE_SEED + 3 + mode, mode=mode, recompute=recompute)
+
+
+def test_evict_first_step_and_short_cache():
+    shape = dict(batch=2, h_q=16, h_kv=4, b=100, buffer=60, w=12, s=60)   # C = 160, ragged
+    run_single_eviction(shape, synth.BASE_SEED + 9, n_h=0)                # first compression: no history
+    run_single_eviction(shape, synth.BASE_SEED + 10, l=101)               # evicts exactly one row
+    run_single_eviction(shape, synth.BASE_SEED + 11, l=131, n_h=50, alpha=0.0)
+
+
+def test_evict_large_window_and_group8():
+    shape = dict(batch=2, h_q=64, h_kv=8, b=320, buffer=64, w=64, s=64)   # g = 8, w = 64: two CTAs per unit
+    run_single_eviction(shape, synth.BASE_SEED + 12)
+    shape = dict(batch=2, h_q=32, h_kv=8, b=256, buffer=128, w=64, s=128)  # g = 4, w = 64
+    run_single_eviction(shape, synth.BASE_SEED + 13)
+    shape = dict(batch=1, h_q=3, h_kv=1, b=70, buffer=20, w=5, s=20)       # g = 3, odd window
+    run_single_eviction(shape, synth.BASE_SEED + 14)
+
+
+def test_evict_staged_equals_fused():
+    shape = dict(batch=5, h_q=16, h_kv=4, b=300, buffer=84, w=16, s=84)
+    for recompute in (True, False):
+        c1, _, kept1, _ = run_single_eviction(shape, synth.BASE_SEED + 20, recompute=recompute, staged=False)
+        c2, _, kept2, _ = run_single_eviction(shape, synth.BASE_SEED + 20, recompute=recompute, staged=True)
+        assert (kept1 == kept2).all()
+        b = shape["b"]
+        assert torch.equal(c1.k[:, :, :, :b], c2.k[:, :, :, :b]) and torch.equal(c1.v[:, :, :, :b], c2.v[:, :, :, :b])
+        assert torch.equal(c1.f, c2.f) and torch.equal(c1.pos[:, :, :, :b], c2.pos[:, :, :, :b])
+
+
+def test_evict_exact_ties_break_toward_lower_position():
+    """Quantised scores make the arithmetic exact in fp32, so the kept lists must equal the
+    oracle's bit for bit, including the tie rule."""
+    shape = dict(batch=2, h_q=8, h_kv=2, b=96, buffer=32, w=8, s=32)
+    cfg = gkv.make_config(n_layers=1, **shape, alpha=0.5, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True)
+    cache = gkv.GKVCache(cfg, DEV)
+    C, b, w = 128, 96, 8
+    rng = np.random.default_rng(5)
+    sums = rng.integers(0, 5, size=(2, 2, C)).astype(np.float32)
+    sums[:, :, 7] = 4.0                                       # the maximum (a power of two) is present
+    f_prev = (rng.integers(0, 9, size=(2, 2, C)) / 8.0).astype(np.float32)
+    case = synth.eviction_case(1, batch=2, h_q=8, h_kv=2, b=b, buffer=32, w=w, device=DEV)
+    case.f_prev = torch.from_numpy(f_prev).to(DEV)
+    load_case(cache, case, 0, torch.from_numpy(sums).to(DEV))
+    snap = snapshot(cache, 0, [0, 1])
+    kept = torch.empty((2, 2, b), dtype=torch.int32, device=DEV)
+    cache.evict(0, None, kept)
+    cache.poll()
+    ref = oracle.evict_batch(None, sums, snap["K"], snap["V"], f_prev, h_q=8, l=C, n_h=case.n_h, b=b, w=w,
+                             alpha=0.5, mode=oracle.MODE_MAX, want_kv=True)
+    assert (kept.cpu().numpy() == ref["kept"]).all()
+    assert (synth.bits(cache.k[0])[:, :, :b] == ref["K"][:, :, :b]).all()
+    np.testing.assert_array_equal(cache.f[0].cpu().numpy()[:, :, : b - w], ref["F_state"][:, :, : b - w].astype(np.float32))
+
+
+def test_evict_noop_and_state_errors():
+    shape = dict(batch=1, h_q=8, h_kv=2, b=96, buffer=32, w=8, s=32)
+    cfg = gkv.make_config(n_layers=2, **shape, fuse_window_scores=True)
+    cache = gkv.GKVCache(cfg, DEV)
+    cache.sacc.fill_(1.0)
+    cache.k.normal_()
+    before = cache.k.clone()
+    cache.set_state(-1, 90, 0, 32)
+    cache.evict(-1)                                           # len <= b: nothing moves, sums restart
+    assert torch.equal(cache.k, before) and float(cache.sacc.abs().max()) == 0.0
+    assert cache.state(0) == (90, 0, 0) and cache.state(1) == (90, 0, 0)
+    cache.set_state(-1, 120, 0, 5)                            # mid-interval: no window sums yet
+    with pytest.raises(gkv.GKVError) as e:
+        cache.evict(-1)
+    assert e.value.status == gkv.GKV_ERR_STATE
+    with pytest.raises(gkv.GKVError) as e:
+        cache.evict(5)
+    assert e.value.status == gkv.GKV_ERR_INVALID_ARG
+    with pytest.raises(gkv.GKVError) as e:
+        cache.evict_stage(0, gkv.GKV_STAGE_SELECT)            # out of order
+    assert e.value.status == gkv.GKV_ERR_STATE
+    cache.set_state(-1, 100, 0, 32)                           # a compression is due: no decode in fused mode
+    x = torch.zeros((2, 1, 8, 128), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(gkv.GKVError) as e:
+        cache.decode_attn(-1, x, x[:, :, :2].contiguous(), x[:, :, :2].contiguous(), x.clone())
+    assert e.value.status == gkv.GKV_ERR_STATE
+    cache.poll()
+
+
+# ------------------------------------------------------------------------- multi-step loop
+def test_decode_eviction_loop_stepwise_parity():
+    """Configuration-1-shaped loop (28 q / 4 kv heads, drifting queries, planted keys), shortened:
+    at every compression the oracle steps from the GPU's own pre-eviction state."""
+    shape = dict(n_layers=2, batch=2, h_q=28, h_kv=4, b=128, buffer=32, w=16, s=32)
+    cfg = gkv.make_config(**shape, fuse_window_scores=True, track_positions=False)
+    cache = gkv.GKVCache(cfg, DEV)
+    stream = synth.DecodeStream(synth.BASE_SEED + 1, n_layers=2, batch=2, h_q=28, h_kv=4, b=128, s=32, device=DEV)
+    out = torch.empty((2, 2, 28, 128), dtype=torch.bfloat16, device=DEV)
+    kept = torch.empty((2, 2, 4, 128), dtype=torch.int32, device=DEV)
+    real = 0
+    for t in range(32 * 9):
+        q, kn, vn = stream.step()
+        cache.decode_attn(-1, q, kn, vn, out)
+        if t % 37 == 0:   # spot-check the attention output against the oracle on the live cache
+            n = cache.state(0)[0]
+            ref = oracle.decode_batch(synth.bits(q[1]), synth.bits(cache.k[1]), synth.bits(cache.v[1]), n)
+            assert np.abs(out[1].float().cpu().numpy() - ref).max() < DECODE_ATOL
+        if (t + 1) % 32 == 0:
+            l, n_h, _ = cache.state(0)
+            snaps = [snapshot(cache, layer, [0, 1]) for layer in range(2)]
+            cache.evict(-1, None, kept)
+            if l > 128:
+                real += 1
+                for layer in range(2):
+                    check_evict_against_oracle(cache, layer, [0, 1], snaps[layer], kept[layer].cpu().numpy(),
+                                               l=l, n_h=n_h)
+            assert cache.state(1) == (min(l, 128), 112 if l > 128 else 0, 0)
+    cache.poll()
+    assert real == 5
+
+
+# ------------------------------------------------------------------------- full-size, sampled
+def test_full_size_config2_sampled():
+    """Configuration 2 at full size (28 layers x batch 32, 28 q / 4 kv, b = 1024, w = 32), in the
+    launch configuration the benchmark times: one decode window and one eviction, sampled units."""
+    shape = {k: v for k, v in synth.CONFIGS[2].items() if k != "steps"}
+    cfg = gkv.make_config(**shape, fuse_window_scores=True)
+    cache = gkv.GKVCache(cfg, DEV)
+    L, B, Hq, H, C, w, b, s = 28, 32, 28, 4, 1152, 32, 1024, 128
+    gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 2)
+    cache.k.copy_(torch.randn(cache.k.shape, generator=gen, device=DEV).to(torch.bfloat16))
+    cache.v.copy_(torch.randn(cache.v.shape, generator=gen, device=DEV).to(torch.bfloat16))
+    cache.f.copy_(torch.rand(cache.f.shape, generator=gen, device=DEV))
+    cache.set_state(-1, C - w, b - w, s - w)
+    out = torch.empty((L, B, Hq, 128), dtype=torch.bfloat16, device=DEV)
+    qs = []
+    for t in range(w):
+        q = torch.randn((L, B, Hq, 128), generator=gen, device=DEV).to(torch.bfloat16)
+        kn = torch.randn((L, B, H, 128), generator=gen, device=DEV).to(torch.bfloat16)
+        vn = torch.randn((L, B, H, 128), generator=gen, device=DEV).to(torch.bfloat16)
+        cache.decode_attn(-1, q, kn, vn, out)
+        qs.append(q)
+    sample = [(0, 0), (13, 17), (27, 31)]
+    for layer, seq in sample:   # last decode step's output and the window sums
+        ref = oracle.decode_attention(synth.bits(qs[-1][layer, seq]), synth.bits(cache.k[layer, seq]),
+                                      synth.bits(cache.v[layer, seq]), C)
+        assert np.abs(out[layer, seq].float().cpu().numpy() - ref).max() < DECODE_ATOL
+        qw = synth.bits(torch.stack([x[layer, seq] for x in qs], dim=1).contiguous())
+        S = oracle.window_mean(oracle.group_max(oracle.window_attention(qw, synth.bits(cache.k[layer, seq]), C), H))
+        np.testing.assert_allclose(cache.sacc[layer, seq].cpu().numpy() / w, S, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+    snaps = {ls: snapshot(cache, ls[0], [ls[1]]) for ls in sample}
+    kept = torch.empty((L, B, H, b), dtype=torch.int32, device=DEV)
+    cache.evict(-1, None, kept)
+    cache.poll()
+    for layer, seq in sample:
+        check_evict_against_oracle(cache, layer, [seq], snaps[(layer, seq)], kept[layer, seq:seq + 1].cpu().numpy(),
+                                   l=C, n_h=b - w)
+    # properties that hold for every unit
+    kk = kept.cpu().numpy()
+    assert (np.diff(kk, axis=-1) > 0).all() and (kk[..., b - w:] == np.arange(C - w, C)).all()
+    assert int(cache.len[0].min()) == int(cache.len[0].max()) == b

@@ -1,0 +1,105 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every symbol the header declares, and
+its host logic (configuration checks, size calculator, memory model) behaves. No kernel runs."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+import paper_2512_00504_b200 as gkv
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    gkv.build_library()
+
+
+def test_every_declared_symbol_is_exported():
+    header = (ROOT / "include" / "gkv.h").read_text()
+    # function declarations: a return type, then gkv_xxx( at the start of a declaration
+    names = set(re.findall(r"^(?:gkv_status|const char\*|void|int64_t)\s+(gkv_\w+)\s*\(", header, flags=re.M))
+    assert {"gkv_init", "gkv_decode_attn", "gkv_evict", "gkv_query_sizes", "gkv_destroy"} <= names
+    lib = ctypes.CDLL(str(gkv.LIB_PATH))
+    for name in sorted(names):
+        assert hasattr(lib, name), f"{name} declared in gkv.h but not exported"
+
+
+def test_strerror_and_null_handling():
+    assert gkv.gkv_strerror(gkv.GKV_OK) == "ok"
+    assert "full" in gkv.gkv_strerror(gkv.GKV_ERR_CAPACITY)
+    lib = gkv.lib()
+    assert lib.gkv_query_sizes(None, None) == gkv.GKV_ERR_INVALID_ARG
+    assert lib.gkv_evict(None, 0, None, None, None) == gkv.GKV_ERR_INVALID_ARG
+    assert lib.gkv_decode_attn(None, 0, None, None, None, None, None) == gkv.GKV_ERR_INVALID_ARG
+    assert lib.gkv_get_state(None, 0, None, None, None) == gkv.GKV_ERR_INVALID_ARG
+    assert lib.gkv_launch_count(None) == 0
+    lib.gkv_destroy(None)
+
+
+def base(**over):
+    kw = dict(n_layers=2, batch=3, h_q=8, h_kv=2, b=512, buffer=128, w=16, s=128)
+    kw.update(over)
+    return gkv.make_config(**kw)
+
+
+@pytest.mark.parametrize("over,status", [
+    (dict(w=512), gkv.GKV_ERR_INVALID_ARG),          # window must be smaller than the budget
+    (dict(s=129), gkv.GKV_ERR_INVALID_ARG),          # interval beyond the physical slack
+    (dict(s=8), gkv.GKV_ERR_INVALID_ARG),            # interval shorter than the window
+    (dict(alpha=1.5), gkv.GKV_ERR_INVALID_ARG),
+    (dict(h_q=9), gkv.GKV_ERR_INVALID_ARG),          # not a multiple of the KV heads
+    (dict(batch=0), gkv.GKV_ERR_INVALID_ARG),
+    (dict(mode=7), gkv.GKV_ERR_INVALID_ARG),
+    (dict(d=64), gkv.GKV_ERR_UNSUPPORTED),
+    (dict(h_q=32), gkv.GKV_ERR_UNSUPPORTED),         # g = 16 > 8
+    (dict(b=4000, buffer=200, s=128), gkv.GKV_ERR_UNSUPPORTED),
+])
+def test_config_validation(over, status):
+    with pytest.raises(gkv.GKVError) as e:
+        gkv.gkv_query_sizes(base(**over))
+    assert e.value.status == status
+
+
+def test_query_sizes_layout():
+    cfg = base(track_positions=True)
+    s = gkv.gkv_query_sizes(cfg)
+    rows = 2 * 3 * 2 * 640
+    assert s.k == s.v == rows * 128 * 2
+    assert s.f == s.sacc == s.pos == rows * 4
+    assert s.len == 2 * 2 * 3 * 4
+    assert s.workspace > 0 and s.workspace % 256 == 0 and s.staging > 0
+    assert gkv.gkv_query_sizes(base()).pos == 0
+    # the benchmark's 7B-shaped configuration: 28 layers x batch 32 x 4 KV heads x 1152 rows
+    big = gkv.gkv_query_sizes(gkv.make_config(n_layers=28, batch=32, h_q=28, h_kv=4, b=1024, buffer=128, w=32, s=128))
+    assert big.k == 28 * 32 * 4 * 1152 * 256
+    # the 32B-shaped stress configuration keeps ~77 GB of K+V resident
+    huge = gkv.gkv_query_sizes(gkv.make_config(n_layers=64, batch=128, h_q=64, h_kv=8, b=2048, buffer=256, w=64, s=256))
+    assert abs((huge.k + huge.v) / 1e9 - 77.3) < 0.1
+
+
+def test_memory_model_reproduces_the_papers_appendix():
+    """Appendix "Memory Analysis": 28 layers, d = 128, 2 KV heads, bf16, 16k tokens -> ~0.44 GB per
+    sequence and 56 GB at batch 128; with s = 128 and b = 512 / 1024 / 2048 the compressed cache
+    takes 2.18 / 3.93 / 7.43 GB (savings 96.1 / 92.9 / 86.7 %); the score cache is ~1/(2d) of the
+    KV cache, ~27 MB at b = 2048."""
+    GB = 2.0 ** 30
+    one = gkv.make_config(n_layers=28, batch=1, h_q=28, h_kv=2, b=512, buffer=128, w=16, s=128)
+    m = gkv.gkv_memory_model(one, 16384, 2)
+    assert abs(m.full_kv / GB - 0.4375) < 1e-9 and round(m.full_kv / GB, 2) == 0.44
+    for b, gb, saving in ((512, 2.18, 96.1), (1024, 3.93, 92.9), (2048, 7.43, 86.7)):
+        cfg = gkv.make_config(n_layers=28, batch=128, h_q=28, h_kv=2, b=b, buffer=128, w=16, s=128)
+        m = gkv.gkv_memory_model(cfg, 16384, 2)
+        assert m.full_kv / GB == 56.0
+        # the paper truncates rather than rounds its GB figures (2.1875 -> 2.18, 3.9375 -> 3.93, 7.4375 -> 7.43)
+        assert int(m.compressed_kv / GB * 100) / 100 == gb
+        # the printed savings mix rounding and truncation (92.97 % is printed as 92.9 %): allow 0.1
+        assert abs(100 * (1 - m.compressed_kv / m.full_kv) - saving) < 0.1
+        # score cache / compressed-to-b KV cache = (b - w) / (b * d * 2)
+        kv_at_b = m.compressed_kv * b / (b + 128)
+        assert abs(m.score_cache / kv_at_b - (b - 16) / (b * 128 * 2)) < 1e-12
+    assert 26.0 < m.score_cache / 2 ** 20 < 28.5      # "around 27 MB" at b = 2048
+    assert abs(kv_at_b / GB - 7.0) < 0.01             # "approximately 7 GB"
+    with pytest.raises(gkv.GKVError):
+        gkv.gkv_memory_model(one, 0, 2)
