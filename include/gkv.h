@@ -61,7 +61,8 @@ typedef enum {
     GKV_ERR_CAPACITY = 3,    /* the cache is full (len == C): evict before decoding further    */
     GKV_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed                            */
     GKV_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (latched status word)       */
-    GKV_ERR_UNSUPPORTED = 6  /* valid but not built (head_dim != 128, g > 8, ...)              */
+    GKV_ERR_UNSUPPORTED = 6, /* valid but not built (head_dim != 128, g > 8, ...)              */
+    GKV_ERR_SCRATCH_LIMIT = 7 /* problem larger than the library's built-in scratch array      */
 } gkv_status;
 
 /* Form of the global score (Section 5). LOCAL disables the history: F = normalised S. */
@@ -146,6 +147,33 @@ gkv_status gkv_decode_attn_host(gkv_ctx* ctx, int32_t layer, const void* q_host,
                                 const void* v_new_host, void* out_host, void* stream);
 gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host,
                           int32_t* kept_idx_out_host, void* stream);
+
+/* (No counterpart in the paper: an engineering variant of gkv_decode_attn.)
+ * One decode-attention step for ONE layer that needs no workspace, no context and no device
+ * allocation: for callers that cannot obtain device memory when they call -- a plug-in running
+ * inside a server whose memory pool it does not own, or a latency-critical loop where cudaMalloc is
+ * off limits because it synchronises the device and may fail late. The caller passes only inputs and
+ * outputs (device pointers): q [batch][n_q_heads][128], k_new / v_new [batch][n_kv_heads][128],
+ * k_cache / v_cache [batch][n_kv_heads][capacity][128] (16-byte aligned), out [batch][n_q_heads][128],
+ * all bf16. Semantics are those of gkv_decode_attn without window-score accumulation: k_new, v_new are
+ * written to row `len` of every head's cache and out is the attention over rows 0..len; the caller
+ * keeps track of `len` itself (it is passed by value, nothing is read back).
+ * The split-K partials, completion counters, length words and status word live in an array of about
+ * 4.1 MiB that is part of the library's device image: every GPU that loads the library holds it until
+ * the process exits. Limits: batch <= 1024, batch * n_kv_heads <= 1024, and (units x key splits) <=
+ * 1024 CTAs; beyond them the call returns GKV_ERR_SCRATCH_LIMIT and launches nothing.
+ * All calls on a device share that array and it keeps the previous call's contents; each call clears
+ * the words that must start at zero. Calls that overlap on the GPU (two streams, or unordered host
+ * threads) race on the array and produce wrong results: keep them ordered.
+ * The first call on each device resolves the array's device address (with that device current);
+ * make that first call outside any stream capture. The call itself performs no cudaMalloc / cudaFree.
+ * A bounded wait that expires inside the kernel cannot be polled through this entry point; `out` is
+ * then undefined.
+ * Errors: INVALID_ARG (NULL, non-positive sizes, misaligned cache), UNSUPPORTED (g > 8, capacity > 4096),
+ * CAPACITY (len >= capacity), SCRATCH_LIMIT, CUDA. */
+gkv_status gkv_decode_attn_static(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                  void* v_cache, void* out, int32_t batch, int32_t n_q_heads,
+                                  int32_t n_kv_heads, int32_t capacity, int32_t len, void* stream);
 
 /* Host counters of one layer (no synchronisation): cache length, rows with history, tokens
  * decoded since the last compression. Any output pointer may be NULL. */

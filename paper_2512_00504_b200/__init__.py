@@ -18,9 +18,10 @@ from pathlib import Path
 _PKG = Path(__file__).resolve().parent
 _ROOT = _PKG.parent
 LIB_PATH = _PKG / "libgkv.so"
-_SOURCES = ["gkv_api.cu", "gkv_decode.cu", "gkv_evict.cu", "gkv_score.cu"]
+_SOURCES = ["gkv_api.cu", "gkv_decode.cu", "gkv_evict.cu", "gkv_score.cu", "gkv_static_scratch.cu"]
 
-GKV_OK, GKV_ERR_INVALID_ARG, GKV_ERR_STATE, GKV_ERR_CAPACITY, GKV_ERR_CUDA, GKV_ERR_TIMEOUT, GKV_ERR_UNSUPPORTED = range(7)
+GKV_OK, GKV_ERR_INVALID_ARG, GKV_ERR_STATE, GKV_ERR_CAPACITY, GKV_ERR_CUDA, GKV_ERR_TIMEOUT, GKV_ERR_UNSUPPORTED, \
+    GKV_ERR_SCRATCH_LIMIT = range(8)
 GKV_MODE_MAX, GKV_MODE_MEAN, GKV_MODE_SUM, GKV_MODE_LOCAL = range(4)
 GKV_STAGE_SCORE, GKV_STAGE_MERGE, GKV_STAGE_SELECT, GKV_STAGE_COMPACT = range(4)
 
@@ -88,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.gkv_decode_attn_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.gkv_evict_host.argtypes = [vp, i32, vp, vp, vp]
         L.gkv_get_state.argtypes = [vp, i32, P(i32), P(i32), P(i32)]
+        L.gkv_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        L.gkv_decode_attn_static.restype = ctypes.c_int
         L.gkv_launch_count.argtypes = [vp]
         L.gkv_launch_count.restype = i64
         L.gkv_poll_device_status.argtypes = [vp, vp]
@@ -176,6 +179,16 @@ def gkv_decode_attn_host(ctx, layer, q, k_new, v_new, out):
 
 def gkv_evict_host(ctx, layer, q_window=None, kept_idx_out=None):
     _check(lib().gkv_evict_host(ctx, layer, _ptr(q_window), _ptr(kept_idx_out), _stream()), "gkv_evict_host")
+
+
+def gkv_decode_attn_static(q, k_new, v_new, k_cache, v_cache, out, length):
+    """Workspace-free decode step for one layer (see gkv.h): for callers that cannot allocate device
+    memory when they call. k_cache / v_cache are [batch][h_kv][capacity][128]; `length` is the number of
+    rows already in the cache; the new row is written at that index. Calls must not overlap on the GPU."""
+    batch, h_q, _ = q.shape
+    _, h_kv, capacity, _ = k_cache.shape
+    _check(lib().gkv_decode_attn_static(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(out),
+                                        batch, h_q, h_kv, capacity, int(length), _stream()), "gkv_decode_attn_static")
 
 
 def gkv_get_state(ctx, layer):

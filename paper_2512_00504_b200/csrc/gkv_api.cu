@@ -504,6 +504,7 @@ const char* gkv_strerror(gkv_status status) {
         case GKV_ERR_CUDA: return "CUDA call failed";
         case GKV_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case GKV_ERR_UNSUPPORTED: return "configuration not supported by this build";
+        case GKV_ERR_SCRATCH_LIMIT: return "problem exceeds the library's built-in scratch array";
         default: return "unknown status";
     }
 }

@@ -1,0 +1,153 @@
+// gkv_decode_attn_static: one decode-attention step that needs no buffer beyond its inputs and
+// outputs. The split-K partial results, the completion counters, the per-sequence length words and
+// the status word that the context-based call keeps in a caller-allocated workspace live here in a
+// fixed array inside the library's own device image.
+//
+// It exists for callers that cannot obtain device memory at the point of the call: code running
+// after an application has handed its whole memory budget to a pool it does not control (a plug-in
+// inside an inference server), or latency-critical loops where cudaMalloc is forbidden because it
+// synchronises the device and can fail late. Such a caller still owns q, k_new, v_new, the cache and
+// out; it just has no way to produce a workspace.
+//
+// The array costs kStaticScratchBytes of device memory on every GPU that loads the library, until
+// the process exits. All calls share it: two calls that overlap on the GPU (different streams, or
+// different host threads without ordering) race on it and give wrong results.
+#include <math.h>
+
+#include <mutex>
+
+#include "gkv_common.cuh"
+#include "gkv_internal.h"
+
+namespace {
+
+using namespace gkv;
+
+constexpr int kStaticMaxSeq = 1024;            // batch
+constexpr int kStaticMaxUnits = 1024;          // batch * n_kv_heads
+constexpr int kStaticMaxCtas = 1024;           // units * splits
+constexpr size_t kPartBytesPerCta = (16 + kHeadDim * 8) * sizeof(float);
+constexpr size_t kOffStatus = 0;                                   // int32[64]
+constexpr size_t kOffLen = 256;                                    // int32[kStaticMaxSeq]
+constexpr size_t kOffSeqDone = kOffLen + 4 * kStaticMaxSeq;        // int32[kStaticMaxSeq]
+constexpr size_t kOffUnitDone = kOffSeqDone + 4 * kStaticMaxSeq;   // int32[kStaticMaxUnits]
+constexpr size_t kOffPart = kOffUnitDone + 4 * kStaticMaxUnits;    // split-K partials
+constexpr size_t kStaticScratchBytes = kOffPart + kStaticMaxCtas * kPartBytesPerCta;   // ~4.1 MiB
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+__global__ void gkv_static_fill_len(int32_t* len, int n, int32_t value) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) len[i] = value;
+}
+
+// Device address of the array on the current device, resolved once per device.
+constexpr int kMaxDevices = 64;
+std::mutex g_mu;
+unsigned char* g_addr[kMaxDevices] = {};
+bool g_ready[kMaxDevices] = {};
+
+gkv_status scratch_for_current_device(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GKV_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_ready[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+            (void)cudaGetLastError();
+            return GKV_ERR_CUDA;
+        }
+        if (decode_kernel_setup() != cudaSuccess) {
+            (void)cudaGetLastError();
+            return GKV_ERR_CUDA;
+        }
+        g_addr[dev] = static_cast<unsigned char*>(p);
+        g_ready[dev] = true;
+    }
+    *out = g_addr[dev];
+    return GKV_OK;
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// [rows][128] bf16 view in 64 x 64 boxes with the 128-byte swizzle the decode kernel expects.
+bool encode_rows(CUtensorMap* map, void* base, uint64_t rows) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess || !sym)
+        return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTileKeys};
+    const cuuint32_t estr[2] = {1, 1};
+    return reinterpret_cast<EncodeFn>(sym)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                             void* v_cache, void* out, int32_t batch, int32_t n_q_heads,
+                                             int32_t n_kv_heads, int32_t capacity, int32_t len, void* stream) {
+    if (!q || !k_new || !v_new || !k_cache || !v_cache || !out) return GKV_ERR_INVALID_ARG;
+    if (batch <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || capacity <= 0 || len < 0) return GKV_ERR_INVALID_ARG;
+    if (n_q_heads % n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
+    if (n_q_heads / n_kv_heads > kMaxGroup || capacity > 4096) return GKV_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(k_cache) | reinterpret_cast<uintptr_t>(v_cache)) % 16 != 0) return GKV_ERR_INVALID_ARG;
+    if (len >= capacity) return GKV_ERR_CAPACITY;
+    const long units = (long)batch * n_kv_heads;
+    if (batch > kStaticMaxSeq || units > kStaticMaxUnits) return GKV_ERR_SCRATCH_LIMIT;
+
+    unsigned char* scratch = nullptr;
+    gkv_status st = scratch_for_current_device(&scratch);
+    if (st != GKV_OK) return st;
+    int dev = 0, sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return GKV_ERR_CUDA;
+
+    DecodeLaunch p;
+    p.splits = decode_pick_splits((int)units, capacity, sm);
+    if (units * p.splits > kStaticMaxCtas) return GKV_ERR_SCRATCH_LIMIT;
+    CUtensorMap tm_k, tm_v;
+    if (!encode_rows(&tm_k, k_cache, (uint64_t)units * capacity) || !encode_rows(&tm_v, v_cache, (uint64_t)units * capacity))
+        return GKV_ERR_CUDA;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The array keeps whatever the previous call left: status word and counters must start at zero,
+    // and every sequence's length word is set to this call's `len`.
+    if (cudaMemsetAsync(scratch, 0, kOffPart, s) != cudaSuccess) return GKV_ERR_CUDA;
+    int32_t* d_len = reinterpret_cast<int32_t*>(scratch + kOffLen);
+    gkv_static_fill_len<<<(batch + 255) / 256, 256, 0, s>>>(d_len, batch, len);
+    if (cudaGetLastError() != cudaSuccess) return GKV_ERR_CUDA;
+
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.k_cache = static_cast<__nv_bfloat16*>(k_cache);
+    p.v_cache = static_cast<__nv_bfloat16*>(v_cache);
+    p.sacc = nullptr;
+    p.len = d_len;
+    p.seq_done = reinterpret_cast<int32_t*>(scratch + kOffSeqDone);
+    p.unit_done = reinterpret_cast<int32_t*>(scratch + kOffUnitDone);
+    p.part = reinterpret_cast<float*>(scratch + kOffPart);
+    p.logits = nullptr;
+    p.status = reinterpret_cast<int32_t*>(scratch + kOffStatus);
+    p.layer0 = 0; p.n_layers = 1; p.batch = batch; p.h_q = n_q_heads; p.h_kv = n_kv_heads;
+    p.g = n_q_heads / n_kv_heads; p.C = capacity;
+    p.accum = 0;
+    p.stages = decode_pick_stages(capacity, 0, p.splits, nullptr);
+    p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
+    if (launch_decode(p, tm_k, tm_v, s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GKV_ERR_CUDA;
+    }
+    return GKV_OK;
+}
