@@ -28,9 +28,11 @@ sys.path.insert(0, str(ROOT))
 METRIC = "decode tok/s over the compressed cache incl. eviction (attention + eviction only)"
 UNIT = "tok/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
-# capture summarised in profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {"cfg2": None, "cfg1": None, "cfg4": None}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
+# summarised in profiles/decode_kernel_cfg2.md: measured on a 4-layer stack (512 units) as 1.041 x the
+# algorithmic bytes of the captured launch, scaled to the full 3584-unit launch at the period's
+# average length (traffic grows in proportion to units). None where no capture exists.
+NCU_TRAFFIC_BYTES = {"cfg2": 1.041 * 2.022e9, "cfg1": None, "cfg4": None}
 
 
 def workload_shape(name: str) -> dict:
@@ -152,6 +154,8 @@ def run_ours(args) -> dict:
     gkv.build_library()
 
     sh = workload_shape(args.workload)
+    if args.layers > 0:
+        sh["n_layers"] = args.layers   # reduced stack for profiler captures; not a benchmark number
     L, B, Hq, H, d, b, w, s = (sh[k] for k in ("n_layers", "batch", "h_q", "h_kv", "d", "b", "w", "s"))
     C = b + sh["buffer"]
     cfg = gkv.make_config(**sh, alpha=0.8, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True)
@@ -277,7 +281,8 @@ def run_ours(args) -> dict:
         "metric": METRIC, "value": summ["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": summ["ms_per_step"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": describe(args.workload, sh), "tokens_per_step": B * s,
+        "config": {"workload": describe(args.workload, sh) + (" [REDUCED LAYER COUNT: profiling only]" if args.layers > 0 else ""),
+                   "tokens_per_step": B * s,
                    "l2": "inputs larger than L2: every launch streams the whole resident cache "
                          f"({2 * units * C * d * 2 / 1e9:.2f} GB K+V)",
                    "input_ring": ring, "replicas": world},
@@ -368,6 +373,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg4"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiler captures only)")
     ap.add_argument("--ring", type=int, default=0, help="distinct per-step inputs kept on the device (0 = one period)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=20.0)

@@ -8,6 +8,8 @@
 // heads of the group on the N side (S^T = K Q^T, O^T = V^T P^T): no padded rows, each K/V byte
 // is read from shared memory exactly once, and the P^T operand comes from the S^T accumulator by
 // an 8x8 register transpose (movmatrix).
+#include <stdlib.h>
+
 #include "gkv_common.cuh"
 #include "gkv_internal.h"
 
@@ -398,24 +400,27 @@ int decode_pick_splits(int units_in_launch, int C, int sm_count) {
     return s;
 }
 
-// Most bytes in flight per SM: stages per CTA x CTAs per SM, within 227 KB of shared memory.
-// Ties go to the earlier entry of the preference order (3 stages first).
+// Resident CTAs per SM matter more than ring depth: with four consumer warps per CTA the per-warp
+// dependent chain (ldmatrix -> mma -> shuffles -> exp2 -> mma) needs >= 8-12 warps per SM to hide, so take
+// the stage count that allows the most CTAs per SM (up to 3), then the deepest ring that still fits.
 int decode_pick_stages(int C, int accum, int splits, size_t* smem_bytes) {
     const size_t cap = 227 * 1024;
-    const int order[5] = {3, 4, 2, 5, 6};
-    int best = 2;
-    size_t best_flight = 0;
-    for (int i = 0; i < 5; ++i) {
-        const int st = order[i];
+    int best = 2, best_score = -1;
+    for (int st = 2; st <= kMaxStages; ++st) {
         const size_t b = decode_smem_bytes(C, accum, splits, st);
-        if (b > cap) continue;
-        size_t ctas = cap / (b + 1024);  // 1 KB per-CTA reservation
-        if (ctas > 4) ctas = 4;
-        const size_t flight = ctas * (size_t)st;
-        if (flight > best_flight) {
-            best_flight = flight;
+        if (b > cap) break;
+        int ctas = (int)(cap / (b + 1024));  // 1 KB per-CTA reservation
+        if (ctas > 3) ctas = 3;
+        const int score = ctas * 100 + st;
+        if (score > best_score) {
+            best_score = score;
             best = st;
         }
+    }
+    // tuning knobs for experiments: GKV_DECODE_STAGES (plain steps), GKV_DECODE_STAGES_WINDOW (window steps)
+    if (const char* e = getenv(accum ? "GKV_DECODE_STAGES_WINDOW" : "GKV_DECODE_STAGES")) {
+        const int st = atoi(e);
+        if (st >= 2 && st <= kMaxStages && decode_smem_bytes(C, accum, splits, st) <= cap) best = st;
     }
     if (smem_bytes) *smem_bytes = decode_smem_bytes(C, accum, splits, best);
     return best;
