@@ -30,6 +30,7 @@ struct __align__(8) DecodeSmemTail {
     int abort_flag;
     int issued;
     int is_last;
+    uint32_t tmem_base;
 };
 
 __device__ __forceinline__ void latch_timeout(int32_t* status, int where) {
@@ -39,6 +40,14 @@ __device__ __forceinline__ void latch_timeout(int32_t* status, int where) {
     }
 }
 
+// Shared memory for the unit's window sums on window steps without key split.
+__host__ __device__ constexpr size_t decode_sum_bytes(int C, int accum_mode) {
+    return accum_mode == 1 ? (size_t)((C + 63) & ~63) * sizeof(float) : 0;
+}
+
+// ACCUM = 0: plain step. ACCUM = 1: window step, one CTA per unit, logits parked in TMEM.
+// ACCUM = 2: window step with the keys split over several CTAs, logits in the workspace.
+template <int ACCUM>
 __global__ void __launch_bounds__(kDecodeThreads)
 gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v) {
@@ -47,9 +56,14 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int stages = p.stages;
     uint8_t* stage_base = smem;
-    float* s_log = reinterpret_cast<float*>(smem + (size_t)stages * kStageBytes);  // [C][8] when accum && splits == 1
-    const size_t log_bytes = (p.accum && p.splits == 1) ? (size_t)((p.C + 63) & ~63) * 32 : 0;
-    DecodeSmemTail* tail = reinterpret_cast<DecodeSmemTail*>(smem + (size_t)stages * kStageBytes + log_bytes);
+    float* s_sum = reinterpret_cast<float*>(smem + (size_t)stages * kStageBytes);   // [C] window sums, ACCUM == 1 only
+    DecodeSmemTail* tail = reinterpret_cast<DecodeSmemTail*>(smem + (size_t)stages * kStageBytes + decode_sum_bytes(p.C, ACCUM));
+    // Window steps without key split keep the scaled logits [key][head] on chip until the row's
+    // normaliser is final. They live in tensor memory, not shared memory: a consumer thread parks
+    // the 4 values it owns of every tile in 4 columns of its own TMEM lane and reads them back
+    // itself in the epilogue, so shared memory (and with it the number of resident CTAs) is the
+    // same as on plain steps.
+    constexpr bool use_tmem = ACCUM == 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int unit_local = blockIdx.x / p.splits;
@@ -80,7 +94,23 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
         tail->is_last = 0;
         fence_mbar_init();
     }
+    if (use_tmem && warp == kConsumerWarps) {   // whole warp; p.tmem_cols x resident CTAs <= 512, so this never waits
+        tmem_alloc(smem_u32(&tail->tmem_base), (uint32_t)p.tmem_cols);
+        tmem_relinquish_alloc_permit();
+        tmem_fence_before_sync();
+    }
     __syncthreads();
+    if (use_tmem) tmem_fence_after_sync();
+    const uint32_t tmem_warp = use_tmem ? (*(volatile uint32_t*)&tail->tmem_base + ((uint32_t)(warp & 3) << 21)) : 0u;
+
+    // Window steps: the unit's current window sums start their way into shared memory now and are
+    // needed only in the epilogue; the updated sums go back with plain coalesced stores. (One
+    // atomic per key is measurably slower: the L2 atomic units saturate at ~4 M reductions a launch.)
+    if (ACCUM == 1 && warp < kConsumerWarps) {
+        const float* gsum = p.sacc + (size_t)unit * p.C;
+        for (int t = tid; t < n; t += kConsumerWarps * 32) cp_async_4(smem_u32(s_sum + t), gsum + t);
+        cp_async_commit();
+    }
 
     // per-thread softmax / output state of a consumer warp (heads h0 = 2*(lane&3), h0+1)
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
@@ -195,11 +225,10 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
                 float s2 = (sa[2] + sb[2]) * p.scale_log2, s3 = (sa[3] + sb[3]) * p.scale_log2;
                 if (key_a >= n) s0 = s1 = -INFINITY;
                 if (key_b >= n) s2 = s3 = -INFINITY;
-                if (p.accum) {
+                if (ACCUM != 0) {
                     const int h0 = (lane & 3) * 2;
-                    if (p.splits == 1) {
-                        if (key_a < n) *reinterpret_cast<float2*>(s_log + key_a * 8 + h0) = make_float2(s0, s1);
-                        if (key_b < n) *reinterpret_cast<float2*>(s_log + key_b * 8 + h0) = make_float2(s2, s3);
+                    if (ACCUM == 1) {
+                        tmem_st4(tmem_warp + 4u * (uint32_t)it, s0, s1, s2, s3);
                     } else {
                         float* g_log = p.logits + (size_t)unit_local * p.C * 8;
                         if (key_a < n) *reinterpret_cast<float2*>(g_log + key_a * 8 + h0) = make_float2(s0, s1);
@@ -242,6 +271,10 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
         }
     }
 
+    if (use_tmem && warp < kConsumerWarps) {
+        tmem_wait_st();
+        tmem_fence_before_sync();
+    }
     __syncthreads();  // [A] every consumer is done with the stage buffers
     if (*(volatile int*)&tail->abort_flag) {
         // Give copies that are still in flight a bounded time to land before the CTA exits.
@@ -251,6 +284,12 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
                 const int j = it - t_begin;
                 mbar_wait_bounded(smem_u32(&tail->full_bar[j % stages]), (j / stages) & 1);
             }
+        }
+        if (ACCUM == 1) cp_async_wait_all();
+        if (use_tmem && warp == kConsumerWarps) {
+            __syncwarp();
+            tmem_fence_after_sync();
+            tmem_dealloc(*(volatile uint32_t*)&tail->tmem_base, (uint32_t)p.tmem_cols);
         }
         return;
     }
@@ -345,34 +384,62 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
                 if (h < p.g) orow[(size_t)h * kHeadDim] = __float2bfloat16_rn(o[h] / L[h]);
             if (tid < 8) { tail->fin_m[tid] = M[tid]; tail->fin_l[tid] = L[tid]; }
         }
-        if (p.accum) {
+        if (ACCUM != 0) {
+            if (ACCUM == 1) cp_async_wait_all();
             __syncthreads();
-            // Sacc[t] += max over the group of the final weights = exp2(max_h (z_h[t] - M_h - log2 L_h))
-            float c[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) c[h] = (h < p.g) ? tail->fin_m[h] + log2f(tail->fin_l[h]) : INFINITY;
+            // Sacc[t] += max over the group of the final weights = exp2(max_h (z_h[t] - M_h - log2 L_h)).
             float* sacc = p.sacc + (size_t)unit * p.C;
-            const float* g_log = p.logits + (size_t)unit_local * p.C * 8;
-            for (int t = tid; t < n_keys_all; t += kDecodeThreads) {
-                float4 x0, x1;
-                if (p.splits == 1) {
-                    x0 = *reinterpret_cast<const float4*>(s_log + t * 8);
-                    x1 = *reinterpret_cast<const float4*>(s_log + t * 8 + 4);
-                } else {
-                    x0 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8));
-                    x1 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8 + 4));
+            if (ACCUM == 1) {
+                if (warp < kConsumerWarps) {
+                    const int h0 = (lane & 3) * 2;
+                    const float c0 = (h0 < p.g) ? tail->fin_m[h0] + log2f(tail->fin_l[h0]) : INFINITY;
+                    const float c1 = (h0 + 1 < p.g) ? tail->fin_m[h0 + 1] + log2f(tail->fin_l[h0 + 1]) : INFINITY;
+                    // four tiles per TMEM access; columns past the last tile are allocated but never written
+                    // and are ignored (key >= n); each key of the unit is owned by exactly one thread
+                    for (int it4 = 0; it4 < tiles_total; it4 += 4) {
+                        float z[16];
+                        tmem_ld16(tmem_warp + 4u * (uint32_t)it4, z);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            float va = fmaxf(z[4 * u] - c0, z[4 * u + 1] - c1), vb = fmaxf(z[4 * u + 2] - c0, z[4 * u + 3] - c1);
+                            va = fmaxf(va, __shfl_xor_sync(0xffffffffu, va, 1));
+                            vb = fmaxf(vb, __shfl_xor_sync(0xffffffffu, vb, 1));
+                            va = fmaxf(va, __shfl_xor_sync(0xffffffffu, va, 2));
+                            vb = fmaxf(vb, __shfl_xor_sync(0xffffffffu, vb, 2));
+                            const int key = (it4 + u) * kTileKeys + warp * 16 + (lane >> 2) + ((lane & 1) ? 8 : 0);
+                            if ((lane & 2) == 0 && key < n_keys_all) s_sum[key] += fast_exp2((lane & 1) ? vb : va);
+                        }
+                    }
+                    tmem_fence_before_sync();
                 }
-                float v = x0.x - c[0];
-                v = fmaxf(v, x0.y - c[1]); v = fmaxf(v, x0.z - c[2]); v = fmaxf(v, x0.w - c[3]);
-                v = fmaxf(v, x1.x - c[4]); v = fmaxf(v, x1.y - c[5]); v = fmaxf(v, x1.z - c[6]);
-                v = fmaxf(v, x1.w - c[7]);
-                sacc[t] += fast_exp2(v);
+            } else {
+                float c[8];
+#pragma unroll
+                for (int h = 0; h < 8; ++h) c[h] = (h < p.g) ? tail->fin_m[h] + log2f(tail->fin_l[h]) : INFINITY;
+                const float* g_log = p.logits + (size_t)unit_local * p.C * 8;
+                for (int t = tid; t < n_keys_all; t += kDecodeThreads) {
+                    const float4 x0 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8));
+                    const float4 x1 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8 + 4));
+                    float v = x0.x - c[0];
+                    v = fmaxf(v, x0.y - c[1]); v = fmaxf(v, x0.z - c[2]); v = fmaxf(v, x0.w - c[3]);
+                    v = fmaxf(v, x1.x - c[4]); v = fmaxf(v, x1.y - c[5]); v = fmaxf(v, x1.z - c[6]);
+                    v = fmaxf(v, x1.w - c[7]);
+                    atomicAdd(sacc + t, fast_exp2(v));
+                }
             }
         }
     }
 
     // The last CTA of a (layer, sequence) publishes the new length.
     __syncthreads();
+    if (use_tmem && warp == kConsumerWarps) {
+        tmem_fence_after_sync();
+        tmem_dealloc(*(volatile uint32_t*)&tail->tmem_base, (uint32_t)p.tmem_cols);
+    }
+    if (ACCUM == 1) {
+        float* gsum = p.sacc + (size_t)unit * p.C;
+        for (int t = tid; t < n; t += kDecodeThreads) gsum[t] = s_sum[t];
+    }
     if (tid == 0) {
         const int per_seq = p.h_kv * p.splits;
         const int prev = atomicAdd(&p.seq_done[lseq_global], 1);
@@ -385,8 +452,15 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
 
 // ---------------------------------------------------------------------------------------------
 static size_t decode_smem_bytes(int C, int accum, int splits, int stages) {
-    const size_t log_bytes = (accum && splits == 1) ? (size_t)((C + 63) & ~63) * 32 : 0;
-    return 1024 + (size_t)stages * kStageBytes + log_bytes + sizeof(DecodeSmemTail);
+    return 1024 + (size_t)stages * kStageBytes + decode_sum_bytes(C, (accum && splits == 1) ? 1 : 0) + sizeof(DecodeSmemTail);
+}
+
+// TMEM columns a window-step CTA allocates for its logits: 4 per 64-key tile, a power of two >= 32.
+int decode_tmem_cols(int C) {
+    const int need = 4 * ((C + kTileKeys - 1) / kTileKeys);
+    int cols = 32;
+    while (cols < need) cols <<= 1;
+    return cols;   // C <= 4096 -> at most 256
 }
 
 int decode_pick_splits(int units_in_launch, int C, int sm_count) {
@@ -406,11 +480,14 @@ int decode_pick_splits(int units_in_launch, int C, int sm_count) {
 int decode_pick_stages(int C, int accum, int splits, size_t* smem_bytes) {
     const size_t cap = 227 * 1024;
     int best = 2, best_score = -1;
+    // Window steps hold TMEM: resident CTAs x columns must stay within the SM's 512 columns, so that no
+    // CTA ever waits for its allocation.
+    const int cta_cap = (accum && splits == 1) ? min(3, 512 / decode_tmem_cols(C)) : 3;
     for (int st = 2; st <= kMaxStages; ++st) {
         const size_t b = decode_smem_bytes(C, accum, splits, st);
         if (b > cap) break;
         int ctas = (int)(cap / (b + 1024));  // 1 KB per-CTA reservation
-        if (ctas > 3) ctas = 3;
+        if (ctas > cta_cap) ctas = cta_cap;
         const int score = ctas * 100 + st;
         if (score > best_score) {
             best_score = score;
@@ -427,13 +504,21 @@ int decode_pick_stages(int C, int accum, int splits, size_t* smem_bytes) {
 }
 
 cudaError_t decode_kernel_setup() {
-    return cudaFuncSetAttribute(gkv_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(gkv_decode_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gkv_decode_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(gkv_decode_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }
 
-cudaError_t launch_decode(const DecodeLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v, cudaStream_t s) {
+cudaError_t launch_decode(const DecodeLaunch& p_in, const CUtensorMap& tm_k, const CUtensorMap& tm_v, cudaStream_t s) {
+    DecodeLaunch p = p_in;
+    p.tmem_cols = decode_tmem_cols(p.C);
     const size_t smem = decode_smem_bytes(p.C, p.accum, p.splits, p.stages);
     const int grid = p.n_layers * p.batch * p.h_kv * p.splits;
-    gkv_decode_kernel<<<grid, kDecodeThreads, smem, s>>>(p, tm_k, tm_v);
+    if (!p.accum) gkv_decode_kernel<0><<<grid, kDecodeThreads, smem, s>>>(p, tm_k, tm_v);
+    else if (p.splits == 1) gkv_decode_kernel<1><<<grid, kDecodeThreads, smem, s>>>(p, tm_k, tm_v);
+    else gkv_decode_kernel<2><<<grid, kDecodeThreads, smem, s>>>(p, tm_k, tm_v);
     return cudaGetLastError();
 }
 

@@ -41,6 +41,7 @@ struct DecodeLaunch {
     int32_t* status;
     int layer0, n_layers, batch, h_q, h_kv, g, C;
     int splits, stages, accum;
+    int tmem_cols;       // filled in by launch_decode
     float scale_log2;    // log2(e) / sqrt(d)
 };
 
