@@ -299,6 +299,105 @@ def run_ours(args) -> dict:
 
 
 # ------------------------------------------------------------------------------------------
+def run_sweep(args) -> dict:
+    """Eviction-step sweep (configuration 3): 32 q / 8 kv heads, one layer, b x batch x w cells, l = b + 128.
+    Per cell the stages (score, merge, select, compact) are timed as separate launches, then the step as it
+    runs in production: one fused launch reading the window sums, and the recompute path (score launch +
+    fused launch). The JSON line carries the largest cell; `sweep` holds every cell."""
+    import math
+    import torch
+    import paper_2512_00504_b200 as gkv
+    from paper_2512_00504_b200 import synth
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    gkv.build_library()
+    c3 = synth.CONFIGS[3]
+    peaks_path = ROOT / "MEASURED_PEAKS.json"
+    peaks = json.loads(peaks_path.read_text()) if peaks_path.exists() else {}
+    peak_gbs = float(peaks.get("hbm_gbs", 6650.0))
+    peak_tf = float(peaks.get("bf16_tflops", 1590.0))
+    peak_src = "measured (MEASURED_PEAKS.json)" if peaks else "fallback (6.65 TB/s, 1.59 PFLOP/s)"
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    reps = max(3, args.steps)
+    cells = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    launches = 0
+    for b in c3["b_sweep"]:
+        for batch in c3["batch_sweep"]:
+            for w in c3["w_sweep"]:
+                sh = dict(n_layers=1, batch=batch, h_q=c3["h_q"], h_kv=c3["h_kv"], d=128, b=b, buffer=c3["buffer"], w=w, s=c3["s"])
+                H, g, C = sh["h_kv"], sh["h_q"] // sh["h_kv"], b + sh["buffer"]
+                l, n_h, units = C, b - w, batch * sh["h_kv"]
+                cfg = gkv.make_config(**sh, alpha=0.8, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True)
+                cache = gkv.GKVCache(cfg, dev)
+                case = synth.eviction_case(synth.BASE_SEED + 3, batch=batch, h_q=sh["h_q"], h_kv=H, b=b, buffer=sh["buffer"],
+                                           w=w, n_planted=math.ceil(0.01 * l), device=dev)
+                cache.k[0].copy_(case.k); cache.v[0].copy_(case.v); cache.f[0].copy_(case.f_prev)
+                q_win = case.q_win.unsqueeze(0).contiguous()
+                del case
+                cache.set_state(0, l, n_h, sh["s"], False)
+                cache.evict_stage(0, gkv.GKV_STAGE_SCORE, q_win)          # the window sums of this state (w * S)
+                sums0, f0 = cache.sacc.clone(), cache.f.clone()
+                kept = torch.empty((1, batch, H, b), dtype=torch.int32, device=dev)
+
+                def restore():
+                    cache.sacc.copy_(sums0); cache.f.copy_(f0)
+                    cache.set_state(0, l, n_h, sh["s"], True)
+
+                t = {k: [] for k in ("score", "merge", "select", "compact", "fused", "recompute")}
+                moved = 0.0
+                l0 = gkv.gkv_launch_count(cache.ctx)
+                for it in range(reps + 3):
+                    e = [ev() for _ in range(9)]
+                    restore()
+                    e[0].record(); cache.evict_stage(0, gkv.GKV_STAGE_SCORE, q_win)
+                    e[1].record(); cache.evict_stage(0, gkv.GKV_STAGE_MERGE)
+                    e[2].record(); cache.evict_stage(0, gkv.GKV_STAGE_SELECT, None, kept)
+                    e[3].record(); cache.evict_stage(0, gkv.GKV_STAGE_COMPACT)
+                    e[4].record()
+                    restore()
+                    e[5].record(); cache.evict(0, None, kept); e[6].record()
+                    moved = float((kept != torch.arange(b, device=dev, dtype=torch.int32)).sum().item())
+                    restore()
+                    e[7].record(); cache.evict(0, q_win, kept); e[8].record()
+                    torch.cuda.synchronize()
+                    if it >= 3:
+                        for k, (a, z) in zip(t, ((0, 1), (1, 2), (2, 3), (3, 4), (5, 6), (7, 8))):
+                            t[k].append(e[a].elapsed_time(e[z]))
+                cache.poll()
+                launches += gkv.gkv_launch_count(cache.ctx) - l0
+                med = {k: sorted(v)[len(v) // 2] for k, v in t.items()}
+                eb = evict_bytes(sh, moved)
+                flops = 2.0 * 2.0 * units * g * w * 128 * l        # two passes over the keys (statistics, then weights)
+                kbytes = 2.0 * units * l * 256 + units * g * w * 256
+                cells.append({"b": b, "batch": batch, "w": w, "units": units, "ms": med, "moved_rows": moved,
+                              "fused_GBps": eb / (med["fused"] * 1e-3) / 1e9, "fused_frac": eb / (med["fused"] * 1e-3) / 1e9 / peak_gbs,
+                              "fused_bytes": eb, "kv_bytes_resident": 2.0 * units * C * 256,
+                              "score_TFLOPs": flops / (med["score"] * 1e-3) / 1e12, "score_K_GBps": kbytes / (med["score"] * 1e-3) / 1e9,
+                              "scored_kv_tokens_per_s": units * l / (med["recompute"] * 1e-3),
+                              "scored_kv_tokens_per_s_window_sums": units * l / (med["fused"] * 1e-3)})
+                del cache, sums0, f0, kept, q_win
+                torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = cells[-1]
+    return {"metric": "scored KV tokens/s of one eviction step (score from the window queries + merge + top-(b-w) + compaction)",
+            "value": top["scored_kv_tokens_per_s"], "unit": "tok/s", "n_gpus": 1, "steps": reps, "warmup": 3,
+            "ms_per_step": top["ms"]["recompute"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"config 3 sweep, largest cell: 1 layer, batch {top['batch']}, 32 q / 8 kv heads, d 128, b={top['b']}, "
+                                   f"buffer=128, w={top['w']}, l={top['b'] + 128}; step = one eviction step",
+                       "l2": "cells with batch >= 64 hold more K+V than L2; smaller cells are L2-resident, as they are right after a decode step"},
+            "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+            "roofline": {"kernel": "gkv_evict_fused_kernel", "bound": "hbm", "achieved": top["fused_GBps"], "peak": peak_gbs,
+                         "unit": "GB/s", "frac": top["fused_frac"], "peak_source": peak_src, "traffic": None,
+                         "algorithmic_bytes_per_launch": top["fused_bytes"], "avg_launch_ms": top["ms"]["fused"]},
+            "score_kernel": {"TFLOPs": top["score_TFLOPs"], "frac_of_bf16_peak": top["score_TFLOPs"] / peak_tf, "peak_TFLOPs": peak_tf},
+            "sweep": cells}
+
+
+# ------------------------------------------------------------------------------------------
 def cpu_baseline(sh: dict, budget_s: float = 20.0, n_units: int = 64) -> dict:
     """The oracle, as it stands, timed on the host cores on a bounded sample of the workload:
     `n_units` (layer, sequence) pairs, a few decode steps plus one eviction; extrapolated to a period."""
@@ -372,7 +471,7 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg4"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiler captures only)")
     ap.add_argument("--ring", type=int, default=0, help="distinct per-step inputs kept on the device (0 = one period)")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -380,7 +479,14 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
-    res = run_reference(args) if args.impl == "reference" else run_ours(args)
+    if args.impl == "reference":
+        if args.workload == "cfg3":
+            args.workload = "cfg2"   # the oracle arm times the default workload only
+        res = run_reference(args)
+    elif args.workload == "cfg3":
+        res = run_sweep(args)
+    else:
+        res = run_ours(args)
     if res is not None:
         print(json.dumps(res))
 

@@ -89,8 +89,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// 2-D view of a K or V buffer: [rows][128] bf16, boxes of 64 rows x 64 elements, 128-byte swizzle.
-gkv_status encode_map(CUtensorMap* map, void* base, uint64_t rows) {
+// 2-D view of a buffer of 128-element bf16 rows: [rows][128], boxes of box_rows rows x 64 elements,
+// 128-byte swizzle (K and V: 64-row boxes; the window queries: one box per head slice).
+gkv_status encode_map(CUtensorMap* map, void* base, uint64_t rows, uint32_t box_rows = kTileKeys) {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
         void* sym = nullptr;
@@ -102,7 +103,7 @@ gkv_status encode_map(CUtensorMap* map, void* base, uint64_t rows) {
     }
     const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kTileKeys};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -154,7 +155,16 @@ gkv_status launch_score_for(gkv_ctx* ctx, int l0, int nl, const void* q_window, 
     sp.layer0 = l0; sp.n_layers = nl; sp.batch = c.batch; sp.h_q = c.n_q_heads; sp.h_kv = c.n_kv_heads;
     sp.g = ctx->g; sp.C = ctx->C; sp.w = c.window;
     sp.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
-    if (launch_score(sp, ctx->tm_k, s) != cudaSuccess) return GKV_ERR_CUDA;
+    // tcgen05 kernel for windows that split into 16-, 32- or 64-row slices; the mma.sync kernel covers the rest
+    const int wk = score_tc_rows_per_cta(ctx->g, c.window);
+    if (wk > 0 && (reinterpret_cast<uintptr_t>(q_window) & 15) == 0) {
+        CUtensorMap tm_q;
+        const uint64_t q_rows = (uint64_t)nl * c.batch * c.n_q_heads * c.window;
+        if (encode_map(&tm_q, const_cast<void*>(q_window), q_rows, (uint32_t)wk) != GKV_OK) return GKV_ERR_CUDA;
+        if (launch_score_tc(sp, ctx->tm_k, tm_q, wk, s) != cudaSuccess) return GKV_ERR_CUDA;
+    } else if (launch_score(sp, ctx->tm_k, s) != cudaSuccess) {
+        return GKV_ERR_CUDA;
+    }
     ctx->launches += 1;
     return GKV_OK;
 }
@@ -242,7 +252,7 @@ gkv_status gkv_init(gkv_ctx** out, const gkv_config* cfg, const gkv_buffers* b, 
              cudaMemsetAsync(b->workspace, 0, ctx->sizes.workspace, s) == cudaSuccess &&
              (!cfg->track_positions || cudaMemsetAsync(b->pos, 0, ctx->sizes.pos, s) == cudaSuccess);
     }
-    if (ok) ok = decode_kernel_setup() == cudaSuccess && score_kernel_setup() == cudaSuccess;
+    if (ok) ok = decode_kernel_setup() == cudaSuccess && score_kernel_setup() == cudaSuccess && score_tc_kernel_setup() == cudaSuccess;
     if (ok) {
         const uint64_t rows = (uint64_t)cfg->n_layers * ctx->units_per_layer * ctx->C;
         ok = encode_map(&ctx->tm_k, b->k, rows) == GKV_OK && encode_map(&ctx->tm_v, b->v, rows) == GKV_OK;

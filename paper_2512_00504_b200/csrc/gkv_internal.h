@@ -95,6 +95,9 @@ cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s);
 cudaError_t launch_evict_select(const EvictLaunch& p, cudaStream_t s);
 cudaError_t launch_evict_compact(const EvictLaunch& p, int sm_count, cudaStream_t s);
 cudaError_t launch_score(const ScoreLaunch& p, const CUtensorMap& tm_k, cudaStream_t s);
+cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s);
+int score_tc_rows_per_cta(int g, int w);
+cudaError_t score_tc_kernel_setup();
 cudaError_t decode_kernel_setup();
 cudaError_t score_kernel_setup();
 

@@ -1,0 +1,420 @@
+// Local score recomputed from the observation window on the 5th-generation tensor cores
+// (Section 3: Eq. 1 window attention, max over the query heads of a KV head, Eq. 2 mean over the
+// window). Writes w * S into the window-sum buffer, like the decode kernel's step-by-step sums.
+//
+// The softmax of Eq. 1 needs every row's normaliser before the max over heads can be taken, so the
+// keys of a unit are streamed twice, and the two passes use the two orientations of the product so
+// that every reduction is a loop inside one thread:
+//   pass 1   D[q row][key] = Q K^T   (M = 128 query rows, N = 128 keys per tile): the thread that
+//            owns a TMEM lane owns a query row and keeps its online (max, sum) over the keys;
+//   pass 2   D[key][q row] = K Q^T   (M = 128 keys, N = g * wk query rows): the thread that owns a
+//            lane owns a key, and the max over heads and the sum over window rows run over columns.
+// One CTA handles one unit (layer, sequence, KV head) and wk <= 64 window rows of all g heads
+// (g * wk <= 256 rows; wider windows take several CTAs that add into the same sums).
+// Warp 0 streams K tiles by TMA, warp 1 issues tcgen05.mma into two 256-column TMEM accumulators,
+// warps 2-9 (two groups of four, one TMEM lane quarter per warp) read the accumulators back with
+// tcgen05.ld and do the softmax arithmetic, so copy, tensor work and exponentials overlap.
+// Window token k sees the keys t <= n - w + k (its own key included).
+#include "gkv_common.cuh"
+#include "gkv_internal.h"
+
+namespace gkv {
+
+constexpr int kTcThreads = 320;
+constexpr int kTcSoftmaxThreads = 256;
+constexpr int kTcTileKeys = 128;
+constexpr int kTcStages = 3;
+constexpr int kTcKStageBytes = kTcTileKeys * kRowBytes;      // 32 KB: d-low half then d-high half
+constexpr int kTcMaxRows = 256;
+constexpr int kTcQBytes = kTcMaxRows * kRowBytes;            // 64 KB: d-low half (32 KB) then d-high half
+constexpr int kTcAccCols = 256;                              // TMEM columns of one accumulator
+constexpr uint32_t kTcTmemCols = 512;
+
+struct __align__(8) ScoreTcTail {
+    uint64_t q_full;
+    uint64_t k_full[kTcStages];
+    uint64_t k_empty[kTcStages];
+    uint64_t d_full[2];
+    uint64_t d_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int issued;
+};
+
+// K-major operand descriptor: rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__device__ __forceinline__ uint32_t umma_idesc_bf16_m128(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier gets one arrival once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <int N>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, float (&v)[N]);
+template <>
+__device__ __forceinline__ void tmem_ld<8>(uint32_t taddr, float (&v)[8]) {
+    uint32_t r[8];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+template <>
+__device__ __forceinline__ void tmem_ld<16>(uint32_t taddr, float (&v)[16]) { tmem_ld16(taddr, v); }
+template <>
+__device__ __forceinline__ void tmem_ld<32>(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Bounded wait that also gives up as soon as another role of the CTA has raised the abort flag.
+__device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, const int* abort_flag) {
+    for (uint32_t i = 0; i < kWaitSpins; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*(volatile const int*)abort_flag) return false;
+        if (i > 64) __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void tc_abort(ScoreTcTail* tail, int32_t* status, int where) {
+    if (atomicExch(&tail->abort_flag, 1) == 0 && atomicCAS(status, 0, kStatusTimeout) == 0) {
+        status[1] = where;
+        status[2] = blockIdx.x;
+    }
+}
+__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// WK = window rows handled by one CTA (16, 32 or 64); the CTA's local query row of (head h, window
+// row k0 + kk) is h * WK + kk.
+template <int WK>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_q, int n_cta) {
+    constexpr int HW = WK / 2;   // window rows one softmax group handles in pass 2
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* q_smem = smem;
+    uint8_t* k_smem = smem + kTcQBytes;
+    float* s_c = reinterpret_cast<float*>(k_smem + kTcStages * kTcKStageBytes);   // [256] m + log2 l of every local row
+    float* s_pm = s_c + kTcMaxRows;                                               // [2][128] partial row maxima
+    float* s_pl = s_pm + 256;                                                     // [2][128] partial row sums
+    float* s_sum = s_pl + 256;                                                    // [C] window sums of this CTA's rows
+    ScoreTcTail* tail = reinterpret_cast<ScoreTcTail*>(s_sum + ((p.C + 63) & ~63));
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int unit_local = blockIdx.x / n_cta;
+    const int part = blockIdx.x - unit_local * n_cta;
+    const int k0 = part * WK;                       // first window row of this CTA
+    const int head = unit_local % p.h_kv;
+    const int ls = unit_local / p.h_kv;             // layer_local * batch + seq
+    const int lseq_global = p.layer0 * p.batch + ls;
+    const long unit = (long)lseq_global * p.h_kv + head;
+    const int n = p.len[lseq_global];
+    const int T = (n + kTcTileKeys - 1) / kTcTileKeys;
+    const int row0 = (int)(unit * p.C);
+    const int R = p.g * WK;                          // query rows of this CTA, a multiple of 16
+    const int MT = (R + 127) >> 7;                   // 128-row tiles of pass 1
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&tail->q_full), 1);
+        for (int s = 0; s < kTcStages; ++s) {
+            mbar_init(smem_u32(&tail->k_full[s]), 1);
+            mbar_init(smem_u32(&tail->k_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tail->d_full[b]), 1);
+            mbar_init(smem_u32(&tail->d_empty[b]), kTcSoftmaxThreads);
+        }
+        mbar_init(smem_u32(&tail->drain), 1);
+        tail->abort_flag = 0;
+        tail->issued = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {   // whole warp: the CTA takes all of the SM's tensor memory (one CTA per SM by shared memory)
+        tmem_alloc(smem_u32(&tail->tmem_base), kTcTmemCols);
+        tmem_relinquish_alloc_permit();
+        tmem_fence_before_sync();
+    }
+    for (int t = tid; t < p.C; t += kTcThreads) s_sum[t] = 0.f;
+    // rows R .. 128 * MT - 1 of the Q tile take part in the pass-1 products: make them zeros
+    for (int e = tid; e < (MT * 128 - R) * 8 * 2; e += kTcThreads) {
+        const int half = e / ((MT * 128 - R) * 8);
+        const int r = e - half * (MT * 128 - R) * 8;
+        *reinterpret_cast<uint4*>(q_smem + half * (kTcQBytes / 2) + (size_t)R * 128 + r * 16) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async_smem();
+    __syncthreads();
+    tmem_fence_after_sync();
+    const uint32_t tmem_base = *(volatile uint32_t*)&tail->tmem_base;
+    const int total = 2 * T;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&tm_k);
+            prefetch_tensormap(&tm_q);
+            const uint32_t qbar = smem_u32(&tail->q_full);
+            mbar_arrive_expect_tx(qbar, (uint32_t)R * kRowBytes);
+            const int qrow0 = (ls * p.h_q + head * p.g) * p.w + k0;
+            for (int h = 0; h < p.g; ++h) {
+                tma_load_2d(smem_u32(q_smem + (size_t)h * WK * 128), &tm_q, 0, qrow0 + h * p.w, qbar);
+                tma_load_2d(smem_u32(q_smem + kTcQBytes / 2 + (size_t)h * WK * 128), &tm_q, 64, qrow0 + h * p.w, qbar);
+            }
+            for (int i = 0; i < total; ++i) {
+                const int s = i % kTcStages;
+                if (i >= kTcStages && !tc_wait(smem_u32(&tail->k_empty[s]), ((i / kTcStages) - 1) & 1, &tail->abort_flag)) {
+                    tc_abort(tail, p.status, 21);
+                    break;
+                }
+                const int tile = (i < T) ? i : i - T;
+                const uint32_t bar = smem_u32(&tail->k_full[s]);
+                const uint32_t dst = smem_u32(k_smem + (size_t)s * kTcKStageBytes);
+                const int y = row0 + tile * kTcTileKeys;
+                mbar_arrive_expect_tx(bar, kTcKStageBytes);
+                tma_load_2d(dst, &tm_k, 0, y, bar);
+                tma_load_2d(dst + kBoxBytes, &tm_k, 0, y + 64, bar);
+                tma_load_2d(dst + 2 * kBoxBytes, &tm_k, 64, y, bar);
+                tma_load_2d(dst + 3 * kBoxBytes, &tm_k, 64, y + 64, bar);
+                *(volatile int*)&tail->issued = i + 1;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = tc_wait(smem_u32(&tail->q_full), 0, &tail->abort_flag);
+            if (!ok) tc_abort(tail, p.status, 22);
+            const uint32_t q_addr = smem_u32(q_smem), k_addr = smem_u32(k_smem);
+            const uint32_t idesc1 = umma_idesc_bf16_m128(kTcTileKeys), idesc2 = umma_idesc_bf16_m128(R);
+            for (int i = 0; ok && i < total; ++i) {
+                const int s = i % kTcStages, buf = i & 1;
+                if (i >= 2 && !tc_wait(smem_u32(&tail->d_empty[buf]), ((i >> 1) - 1) & 1, &tail->abort_flag)) {
+                    tc_abort(tail, p.status, 23);
+                    break;
+                }
+                if (!tc_wait(smem_u32(&tail->k_full[s]), (i / kTcStages) & 1, &tail->abort_flag)) {
+                    tc_abort(tail, p.status, 24);
+                    break;
+                }
+                tmem_fence_after_sync();
+                const uint32_t ks_addr = k_addr + (uint32_t)s * kTcKStageBytes;
+                const uint32_t d = tmem_base + (uint32_t)buf * kTcAccCols;
+                if (i < T) {
+                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)
+                            umma_bf16(d + (uint32_t)mt * 128,
+                                      umma_desc_sw128(q_addr + (ks >> 2) * (kTcQBytes / 2) + mt * 128 * 128 + (ks & 3) * 32),
+                                      umma_desc_sw128(ks_addr + (ks >> 2) * (kTcKStageBytes / 2) + (ks & 3) * 32), idesc1, ks > 0);
+                } else {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_bf16(d, umma_desc_sw128(ks_addr + (ks >> 2) * (kTcKStageBytes / 2) + (ks & 3) * 32),
+                                  umma_desc_sw128(q_addr + (ks >> 2) * (kTcQBytes / 2) + (ks & 3) * 32), idesc2, ks > 0);
+                }
+                umma_commit(smem_u32(&tail->k_empty[s]));
+                umma_commit(smem_u32(&tail->d_full[buf]));
+            }
+            // everything issued has completed before the accumulators are given back
+            umma_commit(smem_u32(&tail->drain));
+            mbar_wait_bounded(smem_u32(&tail->drain), 0);
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax warps
+        const int wg = (warp - 2) >> 2;               // group 0: warps 2-5, group 1: warps 6-9
+        const int q4 = warp & 3;                      // TMEM lane quarter this warp may touch
+        const int L = q4 * 32 + lane;                 // TMEM lane = accumulator row of this thread
+        const int stid = (warp - 2) * 32 + lane;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const float scale = p.scale_log2;
+        bool ok = true;
+
+        // ---- pass 1: online (max, sum) of the row this thread owns. Two 128-row tiles: one per group,
+        // all 128 keys of the tile; one tile: both groups share it, 64 keys each.
+        const int rl = (MT == 2) ? wg * 128 + L : L;
+        const bool valid = rl < R;
+        const int col0 = (MT == 2) ? 0 : wg * 64;
+        const int nch = (MT == 2) ? 4 : 2;
+        const uint32_t t_p1 = t_lane + (uint32_t)((MT == 2) ? wg * 128 : wg * 64);
+        const int last_vis = n - p.w + k0 + (rl % WK);    // last key the row's token sees
+        float m_raw = -INFINITY, l = 0.f;                 // maximum in unscaled logits, sum relative to it
+        for (int i = 0; i < T; ++i) {
+            const int buf = i & 1;
+            ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (i >> 1) & 1, &tail->abort_flag));
+            if (!ok) { tc_abort(tail, p.status, 25); break; }
+            tmem_fence_after_sync();
+            const int key_base = i * kTcTileKeys + col0;
+            const bool need_mask = i * kTcTileKeys + kTcTileKeys - 1 > n - p.w + k0;
+            for (int ch = 0; ch < nch; ++ch) {
+                float z[32];
+                tmem_ld<32>(t_p1 + (uint32_t)(buf * kTcAccCols + ch * 32), z);
+                if (valid) {
+                    if (need_mask) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (key_base + ch * 32 + j > last_vis) z[j] = -INFINITY;
+                    }
+                    float cm = z[0];
+#pragma unroll
+                    for (int j = 1; j < 32; ++j) cm = fmaxf(cm, z[j]);
+                    const float mn = fmaxf(m_raw, cm);
+                    if (mn != -INFINITY) {
+                        const float neg = -mn * scale;
+                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            s0 += fast_exp2(fmaf(z[j], scale, neg));
+                            s1 += fast_exp2(fmaf(z[j + 1], scale, neg));
+                            s2 += fast_exp2(fmaf(z[j + 2], scale, neg));
+                            s3 += fast_exp2(fmaf(z[j + 3], scale, neg));
+                        }
+                        l = l * fast_exp2(fmaf(m_raw, scale, neg)) + ((s0 + s1) + (s2 + s3));
+                        m_raw = mn;
+                    }
+                }
+            }
+            tmem_fence_before_sync();
+            mbar_arrive(smem_u32(&tail->d_empty[buf]));
+        }
+        // combine the partials of a row and publish c = m + log2 l (scaled, log2 domain)
+        s_pm[wg * 128 + L] = m_raw * scale;
+        s_pl[wg * 128 + L] = l;
+        softmax_bar_sync();
+        if (MT == 2) {
+            s_c[rl] = s_pm[wg * 128 + L] + log2f(s_pl[wg * 128 + L]);
+        } else if (wg == 0) {
+            const float ma = s_pm[L], mb = s_pm[128 + L];
+            const float mm = fmaxf(ma, mb);
+            const float ll = ((ma == -INFINITY) ? 0.f : s_pl[L] * fast_exp2(ma - mm)) +
+                             ((mb == -INFINITY) ? 0.f : s_pl[128 + L] * fast_exp2(mb - mm));
+            s_c[L] = mm + log2f(ll);
+        }
+        softmax_bar_sync();
+
+        // ---- pass 2: this thread owns key `tile * 128 + L`; group wg covers window rows k0 + wg*HW .. + HW - 1
+        for (int i = T; i < total; ++i) {
+            const int buf = i & 1;
+            ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (i >> 1) & 1, &tail->abort_flag));
+            if (!ok) { tc_abort(tail, p.status, 26); break; }
+            tmem_fence_after_sync();
+            float v[HW];
+#pragma unroll
+            for (int j = 0; j < HW; ++j) v[j] = -INFINITY;
+            for (int h = 0; h < p.g; ++h) {
+                float z[HW];
+                tmem_ld<HW>(t_lane + (uint32_t)(buf * kTcAccCols + h * WK + wg * HW), z);
+                const float4* c4 = reinterpret_cast<const float4*>(s_c + h * WK + wg * HW);
+#pragma unroll
+                for (int j = 0; j < HW; j += 4) {
+                    const float4 c = c4[j >> 2];
+                    v[j] = fmaxf(v[j], fmaf(z[j], scale, -c.x));
+                    v[j + 1] = fmaxf(v[j + 1], fmaf(z[j + 1], scale, -c.y));
+                    v[j + 2] = fmaxf(v[j + 2], fmaf(z[j + 2], scale, -c.z));
+                    v[j + 3] = fmaxf(v[j + 3], fmaf(z[j + 3], scale, -c.w));
+                }
+            }
+            tmem_fence_before_sync();
+            mbar_arrive(smem_u32(&tail->d_empty[buf]));
+            const int key = (i - T) * kTcTileKeys + L;
+            if (key < n) {
+                const int first_k = key - (n - p.w) - k0 - wg * HW;   // rows j < first_k decoded before this key existed
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int j = 0; j < HW; j += 2) {
+                    s0 += (j >= first_k) ? fast_exp2(v[j]) : 0.f;
+                    s1 += (j + 1 >= first_k) ? fast_exp2(v[j + 1]) : 0.f;
+                }
+                atomicAdd(&s_sum[key], s0 + s1);
+            }
+        }
+        softmax_bar_sync();
+        if (ok && !*(volatile int*)&tail->abort_flag) {
+            float* out = p.sacc + (size_t)unit * p.C;
+            if (n_cta == 1) {
+                for (int t = stid; t < p.C; t += kTcSoftmaxThreads) out[t] = (t < n) ? s_sum[t] : 0.f;
+            } else {
+                for (int t = stid; t < n; t += kTcSoftmaxThreads) atomicAdd(&out[t], s_sum[t]);   // buffer zeroed by the host
+            }
+        }
+    }
+
+    __syncthreads();
+    if (*(volatile int*)&tail->abort_flag && tid == 0) {
+        // give copies still in flight a bounded time to land before the CTA exits
+        mbar_wait_bounded(smem_u32(&tail->q_full), 0);
+        const int issued = *(volatile int*)&tail->issued;
+        for (int i = max(0, issued - kTcStages); i < issued; ++i)
+            mbar_wait_bounded(smem_u32(&tail->k_full[i % kTcStages]), (i / kTcStages) & 1);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tmem_fence_after_sync();
+        tmem_dealloc(tmem_base, kTcTmemCols);
+    }
+}
+
+static size_t score_tc_smem_bytes(int C) {
+    return 1024 + kTcQBytes + (size_t)kTcStages * kTcKStageBytes + sizeof(float) * (kTcMaxRows + 512 + ((C + 63) & ~63)) +
+           sizeof(ScoreTcTail);
+}
+
+// Window rows per CTA for this shape, or 0 when the shape is left to the mma.sync kernel.
+int score_tc_rows_per_cta(int g, int w) {
+    if (w % 16 != 0 || g < 1 || g > kMaxGroup) return 0;
+    for (int wk = 64; wk >= 16; wk >>= 1)
+        if (wk <= w && w % wk == 0 && g * wk <= kTcMaxRows) return wk;
+    return 0;
+}
+
+cudaError_t score_tc_kernel_setup() {
+    cudaError_t e = cudaFuncSetAttribute(gkv_score_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gkv_score_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(gkv_score_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+}
+
+cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s) {
+    const int n_cta = p.w / wk;
+    const int units = p.n_layers * p.batch * p.h_kv;
+    const size_t smem = score_tc_smem_bytes(p.C);
+    if (n_cta > 1) {
+        const size_t off = (size_t)p.layer0 * p.batch * p.h_kv * p.C;
+        cudaError_t e = cudaMemsetAsync(p.sacc + off, 0, sizeof(float) * (size_t)units * p.C, s);
+        if (e != cudaSuccess) return e;
+    }
+    if (wk == 16) gkv_score_tc_kernel<16><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta);
+    else if (wk == 32) gkv_score_tc_kernel<32><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta);
+    else gkv_score_tc_kernel<64><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta);
+    return cudaGetLastError();
+}
+
+}  // namespace gkv

@@ -182,6 +182,20 @@ def test_evict_large_window_and_group8():
     run_single_eviction(shape, synth.BASE_SEED + 14)
 
 
+@pytest.mark.parametrize("shape,l", [
+    (dict(batch=2, h_q=28, h_kv=4, b=300, buffer=100, w=32, s=100), None),   # 7B head geometry: 224 query rows, two 128-row tiles
+    (dict(batch=1, h_q=4, h_kv=2, b=150, buffer=50, w=48, s=50), None),      # g = 2, window split over three 16-row CTAs
+    (dict(batch=2, h_q=8, h_kv=8, b=40, buffer=24, w=16, s=24), None),       # g = 1, a single ragged 128-key tile
+    (dict(batch=1, h_q=16, h_kv=2, b=1000, buffer=153, w=64, s=153), None),  # g = 8, two CTAs per unit, last tile holds one key
+    (dict(batch=1, h_q=32, h_kv=8, b=500, buffer=140, w=64, s=140), 601),    # g = 4, 256 rows in one CTA, cache not full
+])
+def test_score_tensor_core_shapes(shape, l):
+    """Window shapes that take the tcgen05 scoring kernel (w a multiple of 16), full eviction step from the
+    window queries against the oracle."""
+    assert shape["w"] % 16 == 0
+    run_single_eviction(shape, synth.BASE_SEED + 30 + shape["w"], l=l)
+
+
 def test_evict_staged_equals_fused():
     shape = dict(batch=5, h_q=16, h_kv=4, b=300, buffer=84, w=16, s=84)
     for recompute in (True, False):
