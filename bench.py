@@ -324,9 +324,10 @@ def run_sweep(args) -> dict:
     sampler = ClockSampler(0)
     sampler.start()
     launches = 0
-    for b in c3["b_sweep"]:
-        for batch in c3["batch_sweep"]:
-            for w in c3["w_sweep"]:
+    pick = lambda arg, sweep: tuple(int(x) for x in arg.split(",")) if arg else sweep
+    for b in pick(args.sweep_b, c3["b_sweep"]):
+        for batch in pick(args.sweep_batch, c3["batch_sweep"]):
+            for w in pick(args.sweep_w, c3["w_sweep"]):
                 sh = dict(n_layers=1, batch=batch, h_q=c3["h_q"], h_kv=c3["h_kv"], d=128, b=b, buffer=c3["buffer"], w=w, s=c3["s"])
                 H, g, C = sh["h_kv"], sh["h_q"] // sh["h_kv"], b + sh["buffer"]
                 l, n_h, units = C, b - w, batch * sh["h_kv"]
@@ -476,6 +477,9 @@ def main():
     ap.add_argument("--ring", type=int, default=0, help="distinct per-step inputs kept on the device (0 = one period)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
+    ap.add_argument("--sweep-b", default="", help="cfg3: comma-separated budgets instead of the full sweep")
+    ap.add_argument("--sweep-batch", default="", help="cfg3: comma-separated batch sizes instead of the full sweep")
+    ap.add_argument("--sweep-w", default="", help="cfg3: comma-separated windows instead of the full sweep")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
