@@ -12,18 +12,22 @@
 // One CTA handles one unit (layer, sequence, KV head) and wk <= 64 window rows of all g heads
 // (g * wk <= 256 rows; wider windows take several CTAs that add into the same sums).
 // Warp 0 streams K tiles by TMA, warp 1 issues tcgen05.mma into two 256-column TMEM accumulators,
-// warps 2-9 (two groups of four, one TMEM lane quarter per warp) read the accumulators back with
-// tcgen05.ld and do the softmax arithmetic, so copy, tensor work and exponentials overlap.
+// warps 2-17 (four groups of four, one TMEM lane quarter per warp) read the accumulators back with
+// tcgen05.ld and do the softmax arithmetic, so copy, tensor work and exponentials overlap; the
+// groups split an accumulator's columns, which keeps four warps per scheduler to hide latencies.
 // Window token k sees the keys t <= n - w + k (its own key included).
+#include <stdlib.h>
+
 #include "gkv_common.cuh"
 #include "gkv_internal.h"
 
 namespace gkv {
 
-constexpr int kTcThreads = 320;
-constexpr int kTcSoftmaxThreads = 256;
+constexpr int kTcGroups = 4;                                 // softmax warp groups (4 warps each)
+constexpr int kTcSoftmaxThreads = kTcGroups * 128;
+constexpr int kTcThreads = 64 + kTcSoftmaxThreads;
 constexpr int kTcTileKeys = 128;
-constexpr int kTcStages = 3;
+constexpr int kTcMaxStages = 6;                              // K ring depth is chosen per launch from the shared memory left
 constexpr int kTcKStageBytes = kTcTileKeys * kRowBytes;      // 32 KB: d-low half then d-high half
 constexpr int kTcMaxRows = 256;
 constexpr int kTcQBytes = kTcMaxRows * kRowBytes;            // 64 KB: d-low half (32 KB) then d-high half
@@ -32,8 +36,8 @@ constexpr uint32_t kTcTmemCols = 512;
 
 struct __align__(8) ScoreTcTail {
     uint64_t q_full;
-    uint64_t k_full[kTcStages];
-    uint64_t k_empty[kTcStages];
+    uint64_t k_full[kTcMaxStages];
+    uint64_t k_empty[kTcMaxStages];
     uint64_t d_full[2];
     uint64_t d_empty[2];
     uint64_t drain;
@@ -43,8 +47,17 @@ struct __align__(8) ScoreTcTail {
 };
 
 // K-major operand descriptor: rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+// The low word holds the start address in 16-byte units (14 bits; shared memory is < 256 KB, so adding
+// a byte offset / 16 never carries out of the field); the high word is the same for every operand.
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint64_t umma_desc(uint32_t lo) {
+    constexpr uint32_t hi = 64u | (1u << 14) | (2u << 29);   // stride 1024 B, descriptor version 1, 128-byte swizzle
+    return ((uint64_t)hi << 32) | lo;
+}
+// 16-byte units from the start of an operand tile to its k-step ks (16 elements): d-low / d-high half, then
+// 32 bytes per step inside the 128-byte swizzled row.
+__device__ __forceinline__ constexpr uint32_t umma_kstep(int ks, int half_bytes) {
+    return (uint32_t)(((ks >> 2) * half_bytes + (ks & 3) * 32) >> 4);
 }
 // bf16 x bf16 -> fp32, both operands K-major, M = 128.
 __device__ __forceinline__ uint32_t umma_idesc_bf16_m128(int n) {
@@ -111,24 +124,32 @@ __device__ __forceinline__ void tc_abort(ScoreTcTail* tail, int32_t* status, int
         status[2] = blockIdx.x;
     }
 }
-__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kTcSoftmaxThreads) : "memory"); }
+template <>
+__device__ __forceinline__ void tmem_ld<4>(uint32_t taddr, float (&v)[4]) { tmem_ld4(taddr, v); }
 
 // WK = window rows handled by one CTA (16, 32 or 64); the CTA's local query row of (head h, window
 // row k0 + kk) is h * WK + kk.
 template <int WK>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_q, int n_cta) {
-    constexpr int HW = WK / 2;   // window rows one softmax group handles in pass 2
+                    const __grid_constant__ CUtensorMap tm_q, int n_cta, int stages) {
+    constexpr int HW = WK / kTcGroups;   // window rows one softmax group handles in pass 2
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int R = p.g * WK;                          // query rows of this CTA, a multiple of 16
+    const int MT = (R + 127) >> 7;                   // 128-row tiles of pass 1
+    constexpr int q_half = kTcQBytes / 2;            // bytes of one d-half of the Q tile (d-low, then d-high)
     uint8_t* q_smem = smem;
-    uint8_t* k_smem = smem + kTcQBytes;
-    float* s_c = reinterpret_cast<float*>(k_smem + kTcStages * kTcKStageBytes);   // [256] m + log2 l of every local row
-    float* s_pm = s_c + kTcMaxRows;                                               // [2][128] partial row maxima
-    float* s_pl = s_pm + 256;                                                     // [2][128] partial row sums
-    float* s_sum = s_pl + 256;                                                    // [C] window sums of this CTA's rows
-    ScoreTcTail* tail = reinterpret_cast<ScoreTcTail*>(s_sum + ((p.C + 63) & ~63));
+    uint8_t* k_smem = smem + 2 * q_half;
+    float* s_c = reinterpret_cast<float*>(k_smem + stages * kTcKStageBytes);      // [256] m + log2 l of every local row
+    float* s_pm = s_c + kTcMaxRows;                                               // [groups][128] partial row maxima
+    float* s_pl = s_pm + kTcGroups * 128;                                         // [groups][128] partial row sums
+    // [2][C] window sums of this CTA's rows: two groups add into each plane, so every sum has two addends and
+    // the result does not depend on the order in which the groups arrive
+    float* s_sum = s_pl + kTcGroups * 128;
+    const int c_pad = (p.C + 63) & ~63;
+    ScoreTcTail* tail = reinterpret_cast<ScoreTcTail*>(s_sum + 2 * c_pad);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int unit_local = blockIdx.x / n_cta;
@@ -141,18 +162,16 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
     const int n = p.len[lseq_global];
     const int T = (n + kTcTileKeys - 1) / kTcTileKeys;
     const int row0 = (int)(unit * p.C);
-    const int R = p.g * WK;                          // query rows of this CTA, a multiple of 16
-    const int MT = (R + 127) >> 7;                   // 128-row tiles of pass 1
 
     if (tid == 0) {
         mbar_init(smem_u32(&tail->q_full), 1);
-        for (int s = 0; s < kTcStages; ++s) {
+        for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(&tail->k_full[s]), 1);
             mbar_init(smem_u32(&tail->k_empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tail->d_full[b]), 1);
-            mbar_init(smem_u32(&tail->d_empty[b]), kTcSoftmaxThreads);
+            mbar_init(smem_u32(&tail->d_empty[b]), kTcSoftmaxThreads / 32);   // one arrival per softmax warp
         }
         mbar_init(smem_u32(&tail->drain), 1);
         tail->abort_flag = 0;
@@ -164,12 +183,12 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
         tmem_relinquish_alloc_permit();
         tmem_fence_before_sync();
     }
-    for (int t = tid; t < p.C; t += kTcThreads) s_sum[t] = 0.f;
+    for (int t = tid; t < 2 * c_pad; t += kTcThreads) s_sum[t] = 0.f;
     // rows R .. 128 * MT - 1 of the Q tile take part in the pass-1 products: make them zeros
     for (int e = tid; e < (MT * 128 - R) * 8 * 2; e += kTcThreads) {
         const int half = e / ((MT * 128 - R) * 8);
         const int r = e - half * (MT * 128 - R) * 8;
-        *reinterpret_cast<uint4*>(q_smem + half * (kTcQBytes / 2) + (size_t)R * 128 + r * 16) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(q_smem + half * q_half + (size_t)R * 128 + r * 16) = make_uint4(0, 0, 0, 0);
     }
     fence_proxy_async_smem();
     __syncthreads();
@@ -187,15 +206,14 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
             const int qrow0 = (ls * p.h_q + head * p.g) * p.w + k0;
             for (int h = 0; h < p.g; ++h) {
                 tma_load_2d(smem_u32(q_smem + (size_t)h * WK * 128), &tm_q, 0, qrow0 + h * p.w, qbar);
-                tma_load_2d(smem_u32(q_smem + kTcQBytes / 2 + (size_t)h * WK * 128), &tm_q, 64, qrow0 + h * p.w, qbar);
+                tma_load_2d(smem_u32(q_smem + q_half + (size_t)h * WK * 128), &tm_q, 64, qrow0 + h * p.w, qbar);
             }
-            for (int i = 0; i < total; ++i) {
-                const int s = i % kTcStages;
-                if (i >= kTcStages && !tc_wait(smem_u32(&tail->k_empty[s]), ((i / kTcStages) - 1) & 1, &tail->abort_flag)) {
+            for (int i = 0, s = 0, round = 0; i < total; ++i) {
+                if (round > 0 && !tc_wait(smem_u32(&tail->k_empty[s]), (round - 1) & 1, &tail->abort_flag)) {
                     tc_abort(tail, p.status, 21);
                     break;
                 }
-                const int tile = (i < T) ? i : i - T;
+                const int tile = (i < T) ? i : total - 1 - i;   // pass 2 walks back: the tiles read last are still in L2
                 const uint32_t bar = smem_u32(&tail->k_full[s]);
                 const uint32_t dst = smem_u32(k_smem + (size_t)s * kTcKStageBytes);
                 const int y = row0 + tile * kTcTileKeys;
@@ -205,6 +223,7 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                 tma_load_2d(dst + 2 * kBoxBytes, &tm_k, 64, y, bar);
                 tma_load_2d(dst + 3 * kBoxBytes, &tm_k, 64, y + 64, bar);
                 *(volatile int*)&tail->issued = i + 1;
+                if (++s == stages) { s = 0; ++round; }
             }
         }
     } else if (warp == 1) {
@@ -212,36 +231,41 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
         if (lane == 0) {
             bool ok = tc_wait(smem_u32(&tail->q_full), 0, &tail->abort_flag);
             if (!ok) tc_abort(tail, p.status, 22);
-            const uint32_t q_addr = smem_u32(q_smem), k_addr = smem_u32(k_smem);
+            const uint32_t q_lo = umma_desc_lo(smem_u32(q_smem)), k_lo = umma_desc_lo(smem_u32(k_smem));
             const uint32_t idesc1 = umma_idesc_bf16_m128(kTcTileKeys), idesc2 = umma_idesc_bf16_m128(R);
-            for (int i = 0; ok && i < total; ++i) {
-                const int s = i % kTcStages, buf = i & 1;
+            for (int i = 0, s = 0, round = 0; ok && i < total; ++i) {
+                const int buf = i & 1;
                 if (i >= 2 && !tc_wait(smem_u32(&tail->d_empty[buf]), ((i >> 1) - 1) & 1, &tail->abort_flag)) {
                     tc_abort(tail, p.status, 23);
                     break;
                 }
-                if (!tc_wait(smem_u32(&tail->k_full[s]), (i / kTcStages) & 1, &tail->abort_flag)) {
+                if (!tc_wait(smem_u32(&tail->k_full[s]), round & 1, &tail->abort_flag)) {
                     tc_abort(tail, p.status, 24);
                     break;
                 }
                 tmem_fence_after_sync();
-                const uint32_t ks_addr = k_addr + (uint32_t)s * kTcKStageBytes;
+                const uint32_t ks_lo = k_lo + (uint32_t)s * (kTcKStageBytes >> 4);
                 const uint32_t d = tmem_base + (uint32_t)buf * kTcAccCols;
                 if (i < T) {
-                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_bf16(d, umma_desc(q_lo + umma_kstep(ks, q_half)), umma_desc(ks_lo + umma_kstep(ks, kTcKStageBytes / 2)),
+                                  idesc1, ks > 0);
+                    if (MT == 2) {
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks)
-                            umma_bf16(d + (uint32_t)mt * 128,
-                                      umma_desc_sw128(q_addr + (ks >> 2) * (kTcQBytes / 2) + mt * 128 * 128 + (ks & 3) * 32),
-                                      umma_desc_sw128(ks_addr + (ks >> 2) * (kTcKStageBytes / 2) + (ks & 3) * 32), idesc1, ks > 0);
+                            umma_bf16(d + 128, umma_desc(q_lo + ((128 * 128) >> 4) + umma_kstep(ks, q_half)),
+                                      umma_desc(ks_lo + umma_kstep(ks, kTcKStageBytes / 2)), idesc1, ks > 0);
+                    }
                 } else {
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
-                        umma_bf16(d, umma_desc_sw128(ks_addr + (ks >> 2) * (kTcKStageBytes / 2) + (ks & 3) * 32),
-                                  umma_desc_sw128(q_addr + (ks >> 2) * (kTcQBytes / 2) + (ks & 3) * 32), idesc2, ks > 0);
+                        umma_bf16(d, umma_desc(ks_lo + umma_kstep(ks, kTcKStageBytes / 2)), umma_desc(q_lo + umma_kstep(ks, q_half)),
+                                  idesc2, ks > 0);
                 }
                 umma_commit(smem_u32(&tail->k_empty[s]));
                 umma_commit(smem_u32(&tail->d_full[buf]));
+                if (++s == stages) { s = 0; ++round; }
             }
             // everything issued has completed before the accumulators are given back
             umma_commit(smem_u32(&tail->drain));
@@ -249,7 +273,7 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
         }
     } else {
         // ------------------------------------------------------------------ softmax warps
-        const int wg = (warp - 2) >> 2;               // group 0: warps 2-5, group 1: warps 6-9
+        const int wg = (warp - 2) >> 2;               // group of four consecutive warps
         const int q4 = warp & 3;                      // TMEM lane quarter this warp may touch
         const int L = q4 * 32 + lane;                 // TMEM lane = accumulator row of this thread
         const int stid = (warp - 2) * 32 + lane;
@@ -257,13 +281,13 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
         const float scale = p.scale_log2;
         bool ok = true;
 
-        // ---- pass 1: online (max, sum) of the row this thread owns. Two 128-row tiles: one per group,
-        // all 128 keys of the tile; one tile: both groups share it, 64 keys each.
-        const int rl = (MT == 2) ? wg * 128 + L : L;
+        // ---- pass 1: online (max, sum) of the row this thread owns over its share of the tile's keys.
+        // Two 128-row tiles: two groups per tile, 64 keys each; one tile: all four groups, 32 keys each.
+        const int rl = (MT == 2) ? (wg >> 1) * 128 + L : L;
         const bool valid = rl < R;
-        const int col0 = (MT == 2) ? 0 : wg * 64;
-        const int nch = (MT == 2) ? 4 : 2;
-        const uint32_t t_p1 = t_lane + (uint32_t)((MT == 2) ? wg * 128 : wg * 64);
+        const int col0 = (MT == 2) ? (wg & 1) * 64 : wg * 32;
+        const int nch = (MT == 2) ? 2 : 1;
+        const uint32_t t_p1 = t_lane + (uint32_t)((MT == 2) ? (wg >> 1) * 128 + col0 : col0);
         const int last_vis = n - p.w + k0 + (rl % WK);    // last key the row's token sees
         float m_raw = -INFINITY, l = 0.f;                 // maximum in unscaled logits, sum relative to it
         for (int i = 0; i < T; ++i) {
@@ -282,10 +306,15 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                         for (int j = 0; j < 32; ++j)
                             if (key_base + ch * 32 + j > last_vis) z[j] = -INFINITY;
                     }
-                    float cm = z[0];
+                    float c0 = fmaxf(z[0], z[1]), c1 = fmaxf(z[2], z[3]), c2 = fmaxf(z[4], z[5]), c3 = fmaxf(z[6], z[7]);
 #pragma unroll
-                    for (int j = 1; j < 32; ++j) cm = fmaxf(cm, z[j]);
-                    const float mn = fmaxf(m_raw, cm);
+                    for (int j = 8; j < 32; j += 8) {
+                        c0 = fmaxf(c0, fmaxf(z[j], z[j + 1]));
+                        c1 = fmaxf(c1, fmaxf(z[j + 2], z[j + 3]));
+                        c2 = fmaxf(c2, fmaxf(z[j + 4], z[j + 5]));
+                        c3 = fmaxf(c3, fmaxf(z[j + 6], z[j + 7]));
+                    }
+                    const float mn = fmaxf(m_raw, fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)));
                     if (mn != -INFINITY) {
                         const float neg = -mn * scale;
                         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
@@ -302,20 +331,22 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                 }
             }
             tmem_fence_before_sync();
-            mbar_arrive(smem_u32(&tail->d_empty[buf]));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tail->d_empty[buf]));
         }
         // combine the partials of a row and publish c = m + log2 l (scaled, log2 domain)
         s_pm[wg * 128 + L] = m_raw * scale;
         s_pl[wg * 128 + L] = l;
         softmax_bar_sync();
-        if (MT == 2) {
-            s_c[rl] = s_pm[wg * 128 + L] + log2f(s_pl[wg * 128 + L]);
-        } else if (wg == 0) {
-            const float ma = s_pm[L], mb = s_pm[128 + L];
-            const float mm = fmaxf(ma, mb);
-            const float ll = ((ma == -INFINITY) ? 0.f : s_pl[L] * fast_exp2(ma - mm)) +
-                             ((mb == -INFINITY) ? 0.f : s_pl[128 + L] * fast_exp2(mb - mm));
-            s_c[L] = mm + log2f(ll);
+        if ((MT == 2) ? (wg & 1) == 0 : wg == 0) {
+            const int first = (MT == 2) ? wg : 0, count = (MT == 2) ? 2 : kTcGroups;   // groups that shared this row
+            float mm = -INFINITY, ll = 0.f;
+            for (int q = first; q < first + count; ++q) mm = fmaxf(mm, s_pm[q * 128 + L]);
+            for (int q = first; q < first + count; ++q) {
+                const float mq = s_pm[q * 128 + L];
+                ll += (mq == -INFINITY) ? 0.f : s_pl[q * 128 + L] * fast_exp2(mq - mm);
+            }
+            s_c[rl] = mm + log2f(ll);
         }
         softmax_bar_sync();
 
@@ -342,8 +373,9 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                 }
             }
             tmem_fence_before_sync();
-            mbar_arrive(smem_u32(&tail->d_empty[buf]));
-            const int key = (i - T) * kTcTileKeys + L;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tail->d_empty[buf]));
+            const int key = (total - 1 - i) * kTcTileKeys + L;
             if (key < n) {
                 const int first_k = key - (n - p.w) - k0 - wg * HW;   // rows j < first_k decoded before this key existed
                 float s0 = 0.f, s1 = 0.f;
@@ -352,16 +384,16 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                     s0 += (j >= first_k) ? fast_exp2(v[j]) : 0.f;
                     s1 += (j + 1 >= first_k) ? fast_exp2(v[j + 1]) : 0.f;
                 }
-                atomicAdd(&s_sum[key], s0 + s1);
+                atomicAdd(&s_sum[(wg >> 1) * c_pad + key], s0 + s1);
             }
         }
         softmax_bar_sync();
         if (ok && !*(volatile int*)&tail->abort_flag) {
             float* out = p.sacc + (size_t)unit * p.C;
             if (n_cta == 1) {
-                for (int t = stid; t < p.C; t += kTcSoftmaxThreads) out[t] = (t < n) ? s_sum[t] : 0.f;
+                for (int t = stid; t < p.C; t += kTcSoftmaxThreads) out[t] = (t < n) ? s_sum[t] + s_sum[c_pad + t] : 0.f;
             } else {
-                for (int t = stid; t < n; t += kTcSoftmaxThreads) atomicAdd(&out[t], s_sum[t]);   // buffer zeroed by the host
+                for (int t = stid; t < n; t += kTcSoftmaxThreads) atomicAdd(&out[t], s_sum[t] + s_sum[c_pad + t]);   // buffer zeroed by the host
             }
         }
     }
@@ -371,8 +403,8 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
         // give copies still in flight a bounded time to land before the CTA exits
         mbar_wait_bounded(smem_u32(&tail->q_full), 0);
         const int issued = *(volatile int*)&tail->issued;
-        for (int i = max(0, issued - kTcStages); i < issued; ++i)
-            mbar_wait_bounded(smem_u32(&tail->k_full[i % kTcStages]), (i / kTcStages) & 1);
+        for (int i = max(0, issued - stages); i < issued; ++i)
+            mbar_wait_bounded(smem_u32(&tail->k_full[i % stages]), (i / stages) & 1);
     }
     __syncthreads();
     if (warp == 1) {
@@ -381,9 +413,10 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
     }
 }
 
-static size_t score_tc_smem_bytes(int C) {
-    return 1024 + kTcQBytes + (size_t)kTcStages * kTcKStageBytes + sizeof(float) * (kTcMaxRows + 512 + ((C + 63) & ~63)) +
-           sizeof(ScoreTcTail);
+static size_t score_tc_smem_bytes(int C, int rows, int stages) {
+    (void)rows;
+    return 1024 + (size_t)kTcQBytes + (size_t)stages * kTcKStageBytes +
+           sizeof(float) * (kTcMaxRows + 2 * kTcGroups * 128 + 2 * ((C + 63) & ~63)) + sizeof(ScoreTcTail);
 }
 
 // Window rows per CTA for this shape, or 0 when the shape is left to the mma.sync kernel.
@@ -405,15 +438,22 @@ cudaError_t score_tc_kernel_setup() {
 cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s) {
     const int n_cta = p.w / wk;
     const int units = p.n_layers * p.batch * p.h_kv;
-    const size_t smem = score_tc_smem_bytes(p.C);
+    // the deepest K ring that fits: bytes in flight per SM are what hides the copy latency (one CTA per SM)
+    int stages = 2;
+    while (stages < kTcMaxStages && score_tc_smem_bytes(p.C, p.g * wk, stages + 1) <= 227 * 1024) ++stages;
+    if (const char* e = getenv("GKV_SCORE_STAGES")) {   // tuning knob for experiments
+        const int st = atoi(e);
+        if (st >= 2 && st <= stages) stages = st;
+    }
+    const size_t smem = score_tc_smem_bytes(p.C, p.g * wk, stages);
     if (n_cta > 1) {
         const size_t off = (size_t)p.layer0 * p.batch * p.h_kv * p.C;
         cudaError_t e = cudaMemsetAsync(p.sacc + off, 0, sizeof(float) * (size_t)units * p.C, s);
         if (e != cudaSuccess) return e;
     }
-    if (wk == 16) gkv_score_tc_kernel<16><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta);
-    else if (wk == 32) gkv_score_tc_kernel<32><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta);
-    else gkv_score_tc_kernel<64><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta);
+    if (wk == 16) gkv_score_tc_kernel<16><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages);
+    else if (wk == 32) gkv_score_tc_kernel<32><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages);
+    else gkv_score_tc_kernel<64><<<units * n_cta, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages);
     return cudaGetLastError();
 }
 
