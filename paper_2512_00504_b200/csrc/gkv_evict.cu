@@ -173,6 +173,61 @@ __device__ void compact_phase(__nv_bfloat16* kbase, __nv_bfloat16* vbase, const 
     }
 }
 
+// The same move for whole rows, without register staging: the rows of a group of kCopyRows consecutive
+// DESTINATION rows are gathered into a shared-memory stage by 16-byte cp.async (the stage holds them
+// in destination order), and once they have landed one bulk copy per tensor writes the stage to the
+// group's contiguous destination. kCopyStages - 2 groups of loads are in flight while older groups
+// are stored. In place is safe for the same reason as above: a group's destination ends below the
+// sources of every later group, and its own rows are all in shared memory before it is stored.
+constexpr int kCopyRows = 32;
+constexpr int kCopyStages = 5;
+constexpr int kCopyStageBytes = kCopyRows * kRowBytes * 2;   // K rows then V rows
+constexpr int kCopyRingBytes = kCopyStages * kCopyStageBytes;
+
+__device__ void compact_phase_async(__nv_bfloat16* kbase, __nv_bfloat16* vbase, const int* kept, int b, int r_first,
+                                    uint8_t* ring, int tid) {
+    constexpr int D = kCopyStages - 2;                        // groups of loads in flight
+    const int n_groups = (b - r_first + kCopyRows - 1) / kCopyRows;
+    const uint32_t ring_addr = smem_u32(ring);
+    const uint4* k4 = reinterpret_cast<const uint4*>(kbase);
+    const uint4* v4 = reinterpret_cast<const uint4*>(vbase);
+    for (int j = 0; j < n_groups + D; ++j) {
+        // the stage group j loads into was last read by the store issued two iterations ago
+        if (tid == 0) bulk_wait_read<1>();
+        __syncthreads();
+        if (j < n_groups) {
+            const uint32_t stage = ring_addr + (uint32_t)(j % kCopyStages) * kCopyStageBytes;
+            const int r0 = r_first + j * kCopyRows;
+            // 32 rows x 16 chunks x 2 tensors = 1024 copies over 256 threads
+#pragma unroll
+            for (int u = 0; u < 2 * kCopyRows * 16 / kEvictThreads; ++u) {
+                const int e = u * kEvictThreads + tid;
+                const int is_v = e >> 9, row = (e >> 4) & (kCopyRows - 1), chunk = e & 15;
+                const int r = r0 + row;
+                if (r < b) {
+                    const uint4* src = (is_v ? v4 : k4) + (size_t)kept[r] * 16 + chunk;
+                    cp_async_16(stage + (uint32_t)(is_v * kCopyRows * kRowBytes + row * kRowBytes + chunk * 16), src);
+                }
+            }
+        }
+        cp_async_commit();
+        cp_async_wait_group<D>();          // this thread's copies of group j - D have landed
+        fence_proxy_async_smem();          // ... and are visible to the bulk copy engine
+        __syncthreads();
+        const int jd = j - D;
+        if (jd >= 0 && tid == 0) {
+            const uint32_t stage = ring_addr + (uint32_t)(jd % kCopyStages) * kCopyStageBytes;
+            const int r0 = r_first + jd * kCopyRows;
+            const uint32_t bytes = (uint32_t)min(kCopyRows, b - r0) * kRowBytes;
+            bulk_store(kbase + (size_t)r0 * kHeadDim, stage, bytes);
+            bulk_store(vbase + (size_t)r0 * kHeadDim, stage + kCopyRows * kRowBytes, bytes);
+            bulk_commit();
+        }
+    }
+    if (tid == 0) bulk_wait<0>();          // all rows written before the state is published
+    __syncthreads();
+}
+
 struct UnitIndex {
     int unit_local, lseq_global;
     long unit;
@@ -227,14 +282,17 @@ __device__ __forceinline__ void carve(uint8_t* smem, const EvictLaunch& p, float
     *s_kept = reinterpret_cast<int*>(*s_f + p.C);
     *s_pos = *s_kept + p.b;
 }
-static size_t evict_smem_bytes(const EvictLaunch& p) {
+static size_t evict_state_bytes(const EvictLaunch& p) {
     return sizeof(EvictShared) + sizeof(float) * p.C + sizeof(int) * p.b + (p.pos ? sizeof(int) * p.C : 0);
 }
+static size_t evict_smem_bytes(const EvictLaunch& p) { return evict_state_bytes(p); }
+// the fused kernel adds the copy ring, 128-byte aligned behind the score state
+static size_t evict_ring_offset(const EvictLaunch& p) { return (evict_state_bytes(p) + 127) & ~size_t(127); }
 
 // ---------------------------------------------------------------------------------------------
 // Whole step in one launch: merge -> select -> score-state update -> K/V compaction.
-__global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const EvictLaunch p) {
-    extern __shared__ __align__(16) uint8_t evict_smem[];
+__global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const EvictLaunch p, int ring_offset) {
+    extern __shared__ __align__(128) uint8_t evict_smem[];
     float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
     carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
     const int tid = threadIdx.x;
@@ -250,15 +308,15 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const Ev
     merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
     const int r_first = select_phase(s_f, s_kept, n_c, p.b - p.w, p.w, sh, tid);
     write_score_state(p, u, s_f, s_kept, s_pos, n, tid);
-    compact_phase(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
-                  p.b, r_first, 0, 16, tid);
+    compact_phase_async(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
+                        p.b, r_first, evict_smem + ring_offset, tid);
     publish_state(p, u, p.h_kv, sh, tid);
 }
 
 // ---------------------------------------------------------------------------------------------
 // The same step as separate launches (timed one by one); they hand over through the workspace.
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const EvictLaunch p) {
-    extern __shared__ __align__(16) uint8_t evict_smem[];
+    extern __shared__ __align__(128) uint8_t evict_smem[];
     float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
     carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
     const int tid = threadIdx.x;
@@ -273,7 +331,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const Ev
 }
 
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const EvictLaunch p) {
-    extern __shared__ __align__(16) uint8_t evict_smem[];
+    extern __shared__ __align__(128) uint8_t evict_smem[];
     float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
     carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
     const int tid = threadIdx.x;
@@ -296,7 +354,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const E
 
 // grid = units x slices: each CTA moves one column slice of every row of its unit.
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_compact_kernel(const EvictLaunch p, int slices) {
-    extern __shared__ __align__(16) uint8_t evict_smem[];
+    extern __shared__ __align__(128) uint8_t evict_smem[];
     float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
     carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
     const int tid = threadIdx.x;
@@ -328,10 +386,11 @@ static cudaError_t ensure_smem(const void* fn, size_t bytes) {
 }
 
 cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s) {
-    const size_t smem = evict_smem_bytes(p);
+    const size_t ring = evict_ring_offset(p);
+    const size_t smem = ring + kCopyRingBytes;
     cudaError_t e = ensure_smem((const void*)gkv_evict_fused_kernel, smem);
     if (e != cudaSuccess) return e;
-    gkv_evict_fused_kernel<<<p.n_layers * p.batch * p.h_kv, kEvictThreads, smem, s>>>(p);
+    gkv_evict_fused_kernel<<<p.n_layers * p.batch * p.h_kv, kEvictThreads, smem, s>>>(p, (int)ring);
     return cudaGetLastError();
 }
 cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s) {
