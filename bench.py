@@ -7,7 +7,9 @@ followed by one eviction of every layer (normalise, merge with history, top-(b-w
 The default workload is the 7B-reasoning-model shape the paper's compression-time table is
 quoted on (28 layers, batch 32, 28 q / 4 kv heads, d = 128, b = 1024, w = 32, s = 128).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg4] [--impl reference]
+
+--workload cfg3 runs the eviction-step sweep (stages timed separately and fused) instead of the decode loop.
 
 N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has no exchange step.
 One JSON line is printed by rank 0.
@@ -29,10 +31,11 @@ METRIC = "decode tok/s over the compressed cache incl. eviction (attention + evi
 UNIT = "tok/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
-# summarised in profiles/decode_kernel_cfg2.md: measured on a 4-layer stack (512 units) as 1.041 x the
-# algorithmic bytes of the captured launch, scaled to the full 3584-unit launch at the period's
-# average length (traffic grows in proportion to units). None where no capture exists.
-NCU_TRAFFIC_BYTES = {"cfg2": 1.041 * 2.022e9, "cfg1": None, "cfg4": None}
+# summarised in profiles/decode_kernel_cfg2.md: measured on a 4-layer stack (512 units) as 1.040 (plain
+# steps) and 1.029 (window steps) x the algorithmic bytes of the captured launches, i.e. 1.037 over a
+# period, scaled to the full 3584-unit launch at the period's average length (traffic grows in
+# proportion to units). None where no capture exists.
+NCU_TRAFFIC_BYTES = {"cfg2": 1.037 * 2.022e9, "cfg1": None, "cfg4": None}
 
 
 def workload_shape(name: str) -> dict:
