@@ -333,3 +333,51 @@ def test_full_size_config2_sampled():
     kk = kept.cpu().numpy()
     assert (np.diff(kk, axis=-1) > 0).all() and (kk[..., b - w:] == np.arange(C - w, C)).all()
     assert int(cache.len[0].min()) == int(cache.len[0].max()) == b
+
+
+def test_full_size_config4_sampled():
+    """Configuration 4 at full size (64 layers x batch 128, 64 q / 8 kv, b = 2048, w = 64; 77 GB of K+V
+    resident): one decode window and one in-place eviction in the benchmark's launch configuration,
+    sampled units against the oracle and structural properties for every unit."""
+    free, _ = torch.cuda.mem_get_info(0)
+    if free < 100 * 2**30:
+        pytest.skip("needs about 90 GB of free device memory")
+    shape = {k: v for k, v in synth.CONFIGS[4].items() if k != "steps"}
+    cfg = gkv.make_config(**shape, fuse_window_scores=True)
+    cache = gkv.GKVCache(cfg, DEV)
+    L, B, Hq, H, C, w, b, s = 64, 128, 64, 8, 2304, 64, 2048, 256
+    gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 4)
+    for layer in range(L):
+        cache.k[layer].copy_(torch.randn(cache.k[layer].shape, generator=gen, device=DEV).to(torch.bfloat16))
+        cache.v[layer].copy_(torch.randn(cache.v[layer].shape, generator=gen, device=DEV).to(torch.bfloat16))
+        cache.f[layer].copy_(torch.rand(cache.f[layer].shape, generator=gen, device=DEV))
+    cache.set_state(-1, C - w, b - w, s - w)
+    sample = [(0, 0), (31, 77), (63, 127)]
+    out = torch.empty((L, B, Hq, 128), dtype=torch.bfloat16, device=DEV)
+    q_keep = {ls: [] for ls in sample}
+    for t in range(w):
+        q = torch.randn((L, B, Hq, 128), generator=gen, device=DEV).to(torch.bfloat16)
+        kn = torch.randn((L, B, H, 128), generator=gen, device=DEV).to(torch.bfloat16)
+        vn = torch.randn((L, B, H, 128), generator=gen, device=DEV).to(torch.bfloat16)
+        cache.decode_attn(-1, q, kn, vn, out)
+        for ls in sample:
+            q_keep[ls].append(q[ls[0], ls[1]].clone())
+    for layer, seq in sample:
+        K, V = synth.bits(cache.k[layer, seq]), synth.bits(cache.v[layer, seq])
+        ref = oracle.decode_attention(synth.bits(q_keep[(layer, seq)][-1]), K, V, C)
+        assert np.abs(out[layer, seq].float().cpu().numpy() - ref).max() < DECODE_ATOL
+        qw = synth.bits(torch.stack(q_keep[(layer, seq)], dim=1).contiguous())
+        S = oracle.window_mean(oracle.group_max(oracle.window_attention(qw, K, C), H))
+        np.testing.assert_allclose(cache.sacc[layer, seq].cpu().numpy() / w, S, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+    snaps = {ls: snapshot(cache, ls[0], [ls[1]]) for ls in sample}
+    kept = torch.empty((L, B, H, b), dtype=torch.int32, device=DEV)
+    cache.evict(-1, None, kept)
+    cache.poll()
+    for layer, seq in sample:
+        check_evict_against_oracle(cache, layer, [seq], snaps[(layer, seq)], kept[layer, seq:seq + 1].cpu().numpy(),
+                                   l=C, n_h=b - w)
+    assert bool((kept[..., 1:] > kept[..., :-1]).all())
+    assert bool((kept[..., b - w:] == torch.arange(C - w, C, device=DEV, dtype=torch.int32)).all())
+    assert int(cache.len[0].min()) == int(cache.len[0].max()) == b
+    del cache, out, kept
+    torch.cuda.empty_cache()
