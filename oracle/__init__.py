@@ -45,6 +45,7 @@ def lib() -> ctypes.CDLL:
         _lib = ctypes.CDLL(str(_LIB))
         _lib.gkvo_num_threads.restype = ctypes.c_int
         _lib.gkvo_evict_step.restype = ctypes.c_int
+        _lib.gkvo_evict_step_redundancy.restype = ctypes.c_int
     return _lib
 
 
@@ -143,6 +144,51 @@ def evict_step(Q_win, S_in, K, V, pos, F_prev, *, l, n_h, b, w, alpha, mode):
         _p(out["V"], np.uint16), _p(out["pos"], np.int32), _p(out["F_state"], np.float64))
     out["len"] = int(new_len)
     out["evicted"] = True
+    return out
+
+
+def redundancy(K, l, *, tau, recent, eps, band_width=0.0):
+    """Redundancy score of the appendix. K [h_kv][C][d] uint16 -> dict of cbar, R, Rn [h_kv][l] float64 and
+    band [h_kv][l] int32 (entries per column within band_width of tau)."""
+    h_kv, C, d = K.shape
+    out = {k: np.empty((h_kv, l), np.float64) for k in ("cbar", "R", "Rn")}
+    out["band"] = np.zeros((h_kv, l), np.int32)
+    lib().gkvo_redundancy(_p(K, np.uint16), h_kv, C, d, l, ctypes.c_double(tau), int(recent), ctypes.c_double(eps),
+                          _p(out["cbar"], np.float64), _p(out["R"], np.float64), _p(out["Rn"], np.float64),
+                          _p(out["band"], np.int32), ctypes.c_double(band_width))
+    return out
+
+
+def combine(F, Rn, lam):
+    """Fsel = lam * F - (1 - lam) * Rn over the candidates. F [h_kv][n_c], Rn [h_kv][l] float64."""
+    h_kv, n_c = F.shape
+    l = Rn.shape[1]
+    Fsel = np.empty((h_kv, n_c), np.float64)
+    lib().gkvo_combine(_p(F, np.float64), _p(Rn, np.float64), h_kv, n_c, l, ctypes.c_double(lam), _p(Fsel, np.float64))
+    return Fsel
+
+
+def evict_step_redundancy(Q_win, S_in, K, V, pos, F_prev, *, l, n_h, b, w, alpha, mode, lam, tau, recent, eps,
+                          band_width=0.0):
+    """One eviction step whose selection runs on lam * F - (1 - lam) * Rn; F itself is recorded."""
+    h_kv, C, d = K.shape
+    assert (Q_win is None) != (S_in is None) and l > b
+    h_q = Q_win.shape[0] if Q_win is not None else h_kv
+    n_c = l - w
+    out = {
+        "F": np.empty((h_kv, n_c), np.float64), "cbar": np.empty((h_kv, l), np.float64),
+        "Rn": np.empty((h_kv, l), np.float64), "Fsel": np.empty((h_kv, n_c), np.float64),
+        "band": np.zeros((h_kv, l), np.int32), "kept": np.empty((h_kv, b), np.int32),
+        "K": np.zeros_like(K), "V": np.zeros_like(V), "pos": None if pos is None else np.zeros_like(pos),
+        "F_state": np.zeros((h_kv, C), np.float64),
+    }
+    out["len"] = int(lib().gkvo_evict_step_redundancy(
+        _p(Q_win, np.uint16), _p(S_in, np.float32), _p(K, np.uint16), _p(V, np.uint16), _p(pos, np.int32),
+        _p(F_prev, np.float32), h_q, h_kv, d, C, l, n_h, b, w, ctypes.c_double(alpha), mode, ctypes.c_double(lam),
+        ctypes.c_double(tau), int(recent), ctypes.c_double(eps), ctypes.c_double(band_width),
+        _p(out["F"], np.float64), _p(out["cbar"], np.float64), _p(out["Rn"], np.float64), _p(out["Fsel"], np.float64),
+        _p(out["band"], np.int32), _p(out["kept"], np.int32), _p(out["K"], np.uint16), _p(out["V"], np.uint16),
+        _p(out["pos"], np.int32), _p(out["F_state"], np.float64)))
     return out
 
 

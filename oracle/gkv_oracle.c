@@ -12,7 +12,11 @@
  *   Section 5 ("Training-Free KV Cache Compression with Global Attention"): max-normalisation
  *       of S, the three global-score forms Eq. 3 (max), Eq. 4 (average), Eq. 5 (summation), the
  *       rule for rows without history, the first-step rule, and the recording of F for the
- *       next step.
+ *       next step;
+ *   Appendix on combining the global score with other methods: the redundancy score (normalised
+ *       keys, thresholded cosine similarity, column sums, softmax, max-normalisation) and
+ *       F' = lambda F - (1 - lambda) R' (gkvo_redundancy, gkvo_combine; its threshold, recent-token
+ *       count and epsilon are not in the paper and are parameters).
  * Inputs are the exact bits the GPU consumes: bf16 as uint16 (widened exactly to double) and
  * fp32 score state (widened exactly to double). All arithmetic is double. No blocking, fusion or
  * reordering beyond what the text states.
@@ -310,4 +314,105 @@ void gkvo_decode_batch(int n_seq, const uint16_t* q, const uint16_t* K, const ui
         gkvo_decode_attention(q + (size_t)s * h_q * d, K + s * kv_stride, V + s * kv_stride, h_q, h_kv, d,
                               C, n, out + (size_t)s * h_q * d, NULL,
                               Sacc ? Sacc + (size_t)s * h_kv * C : NULL);
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Appendix "combining the global score with other methods": the redundancy score (of R-KV, as the
+ * paper restates it) and its combination with the global score.
+ *
+ *   Kbar[j,t,:] = K[j,t,:] / (||K[j,t,:]||_2 + eps)                 (normalised key states)
+ *   Cm[j]       = Kbar[j] Kbar[j]^T                                  (cosine similarity, l x l)
+ *   C'[j,k,t]   = 0 where Cm[j,k,t] < tau, and in the columns t of the `recent` most recent tokens
+ *                 (t >= l - recent); Cm elsewhere                    (thresholded similarity)
+ *   cbar[j,t]   = sum_k C'[j,k,t]                                    (redundancy level of token t)
+ *   R[j,t]      = softmax_t(cbar[j,:])                               (redundancy score)
+ *   Rn[j,t]     = R[j,t] / max_t R[j,t]                              (normalised, as the global score is)
+ *   Fsel[j,t]   = lambda F[j,t] - (1 - lambda) Rn[j,t]               (the score the selection runs on)
+ *
+ * The paper gives no value for tau, for the number of recent tokens or for eps (it defers to the
+ * R-KV paper): they are parameters here. Reading taken for "those corresponding to the most recent
+ * tokens": the COLUMNS of the recent tokens are zeroed, so a recent token is never rated redundant,
+ * while its row still counts as a witness of the redundancy of older tokens. The diagonal is not
+ * special-cased (the text does not): every kept column carries its own ~1.
+ * band (optional, [h_kv][l] int32) counts, per column, the entries whose similarity lies within
+ * band_width of tau: a comparison in lower precision may flip exactly those.
+ * ------------------------------------------------------------------------------------------ */
+void gkvo_redundancy(const uint16_t* K, int h_kv, int C, int d, int l, double tau, int recent, double eps,
+                     double* cbar, double* R, double* Rn, int32_t* band, double band_width) {
+    double* Kbar = (double*)malloc(sizeof(double) * (size_t)l * d);
+    for (int j = 0; j < h_kv; ++j) {
+        for (int t = 0; t < l; ++t) {
+            const uint16_t* row = K + ((size_t)j * C + t) * d;
+            double ss = 0.0;
+            for (int c = 0; c < d; ++c) { const double x = bf16_to_double(row[c]); ss += x * x; }
+            const double inv = 1.0 / (sqrt(ss) + eps);
+            for (int c = 0; c < d; ++c) Kbar[(size_t)t * d + c] = bf16_to_double(row[c]) * inv;
+        }
+        double* cb = cbar + (size_t)j * l;
+        for (int t = 0; t < l; ++t) {
+            double sum = 0.0;
+            int near = 0;
+            for (int k = 0; k < l; ++k) {
+                double dot = 0.0;
+                for (int c = 0; c < d; ++c) dot += Kbar[(size_t)k * d + c] * Kbar[(size_t)t * d + c];
+                if (fabs(dot - tau) < band_width) ++near;
+                const int masked = (dot < tau) || (t >= l - recent);
+                sum += masked ? 0.0 : dot;
+            }
+            cb[t] = sum;
+            if (band) band[(size_t)j * l + t] = near;
+        }
+        double m = cb[0];
+        for (int t = 1; t < l; ++t) if (cb[t] > m) m = cb[t];
+        double Z = 0.0;
+        for (int t = 0; t < l; ++t) Z += exp(cb[t] - m);
+        double rmax = 0.0;
+        for (int t = 0; t < l; ++t) {
+            R[(size_t)j * l + t] = exp(cb[t] - m) / Z;
+            if (R[(size_t)j * l + t] > rmax) rmax = R[(size_t)j * l + t];
+        }
+        for (int t = 0; t < l; ++t) Rn[(size_t)j * l + t] = R[(size_t)j * l + t] / rmax;
+    }
+    free(Kbar);
+}
+
+/* Fsel = lambda F - (1 - lambda) Rn over the n_c candidates. F [h_kv][n_c], Rn [h_kv][l]. */
+void gkvo_combine(const double* F, const double* Rn, int h_kv, int n_c, int l, double lambda, double* Fsel) {
+    for (int j = 0; j < h_kv; ++j)
+        for (int t = 0; t < n_c; ++t)
+            Fsel[(size_t)j * n_c + t] = lambda * F[(size_t)j * n_c + t] - (1.0 - lambda) * Rn[(size_t)j * l + t];
+}
+
+/* The eviction step with the redundancy term: as gkvo_evict_step up to the global score F; the
+ * top-(b-w) selection runs on Fsel; the score recorded for the next step is F itself (Section 5
+ * records F_t; the redundancy term only steers the selection). Extra outputs (may be NULL):
+ * cbar_out, Rn_out [h_kv][l], Fsel_out [h_kv][n_c], band_out [h_kv][l]. */
+int gkvo_evict_step_redundancy(const uint16_t* Q_win, const float* S_in, const uint16_t* K, const uint16_t* V,
+                               const int32_t* pos, const float* F_prev, int h_q, int h_kv, int d, int C, int l,
+                               int n_h, int b, int w, double alpha, int mode, double lambda, double tau,
+                               int recent, double eps, double band_width, double* F_out, double* cbar_out,
+                               double* Rn_out, double* Fsel_out, int32_t* band_out, int32_t* kept_out,
+                               uint16_t* K_out, uint16_t* V_out, int32_t* pos_out, double* F_state) {
+    if (l <= b) return l;
+    const int n_c = l - w;
+    double* F = (double*)malloc(sizeof(double) * (size_t)h_kv * n_c);
+    gkvo_evict_step(Q_win, S_in, K, V, pos, F_prev, h_q, h_kv, d, C, l, n_h, b, w, alpha, mode, NULL, NULL, F,
+                    NULL, NULL, NULL, NULL, NULL);
+    double* cbar = (double*)malloc(sizeof(double) * (size_t)h_kv * l);
+    double* R = (double*)malloc(sizeof(double) * (size_t)h_kv * l);
+    double* Rn = (double*)malloc(sizeof(double) * (size_t)h_kv * l);
+    double* Fsel = (double*)malloc(sizeof(double) * (size_t)h_kv * n_c);
+    int32_t* kept = (int32_t*)malloc(sizeof(int32_t) * (size_t)h_kv * b);
+    gkvo_redundancy(K, h_kv, C, d, l, tau, recent, eps, cbar, R, Rn, band_out, band_width);
+    gkvo_combine(F, Rn, h_kv, n_c, l, lambda, Fsel);
+    gkvo_select(Fsel, h_kv, n_c, l, b, w, kept);
+    if (K_out && V_out && F_state)
+        gkvo_compact(K, V, pos, F, kept, h_kv, C, d, n_c, b, w, K_out, V_out, pos_out, F_state);
+    if (F_out) memcpy(F_out, F, sizeof(double) * (size_t)h_kv * n_c);
+    if (cbar_out) memcpy(cbar_out, cbar, sizeof(double) * (size_t)h_kv * l);
+    if (Rn_out) memcpy(Rn_out, Rn, sizeof(double) * (size_t)h_kv * l);
+    if (Fsel_out) memcpy(Fsel_out, Fsel, sizeof(double) * (size_t)h_kv * n_c);
+    if (kept_out) memcpy(kept_out, kept, sizeof(int32_t) * (size_t)h_kv * b);
+    free(F); free(cbar); free(R); free(Rn); free(Fsel); free(kept);
+    return b;
 }
