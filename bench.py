@@ -139,6 +139,14 @@ def evict_bytes(sh: dict, moved_rows: float) -> float:
     return float(units * per_unit + moved_rows * 4 * sh["d"] * 2)
 
 
+def redundancy_kwargs(args) -> dict:
+    """Configuration of the redundancy term (appendix on combining the global score with other methods);
+    off unless --redundancy LAMBDA is given. Threshold and protected recent tokens are the benchmark's choice."""
+    if args.redundancy is None:
+        return {}
+    return dict(redundancy_lambda=args.redundancy, redundancy_threshold=args.redundancy_threshold)
+
+
 def run_ours(args) -> dict:
     import torch
     import paper_2512_00504_b200 as gkv
@@ -161,7 +169,7 @@ def run_ours(args) -> dict:
         sh["n_layers"] = args.layers   # reduced stack for profiler captures; not a benchmark number
     L, B, Hq, H, d, b, w, s = (sh[k] for k in ("n_layers", "batch", "h_q", "h_kv", "d", "b", "w", "s"))
     C = b + sh["buffer"]
-    cfg = gkv.make_config(**sh, alpha=0.8, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True)
+    cfg = gkv.make_config(**sh, alpha=0.8, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True, **redundancy_kwargs(args))
     cache = gkv.GKVCache(cfg, dev, staging=True)
 
     # steady-state cache: b rows of N(0,1) keys/values, history on the first b-w rows
@@ -279,6 +287,10 @@ def run_ours(args) -> dict:
              "scored_kv_tokens_per_s": units * (b + s) / (evict_ms * 1e-3), "moved_rows": moved,
              "algorithmic_bytes": eb, "achieved_GBps": eb / (evict_ms * 1e-3) / 1e9,
              "frac": eb / (evict_ms * 1e-3) / 1e9 / peak_gbs, "overhead_frac_of_step": evict_ms / (max_ms / args.steps)}
+    if args.redundancy is not None:   # the eviction then has two more launches (key norms, similarity sums on tcgen05)
+        evict["redundancy"] = {"lambda": args.redundancy, "threshold": args.redundancy_threshold,
+                               "note": "ms includes gkv_keynorm_kernel and gkv_redundancy_tc_kernel; GB/s and frac do not describe them",
+                               "gram_flop": 2.0 * units * (b + s) * (b + s) * d}
 
     result = {
         "metric": METRIC, "value": summ["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -334,8 +346,9 @@ def run_sweep(args) -> dict:
                 sh = dict(n_layers=1, batch=batch, h_q=c3["h_q"], h_kv=c3["h_kv"], d=128, b=b, buffer=c3["buffer"], w=w, s=c3["s"])
                 H, g, C = sh["h_kv"], sh["h_q"] // sh["h_kv"], b + sh["buffer"]
                 l, n_h, units = C, b - w, batch * sh["h_kv"]
-                cfg = gkv.make_config(**sh, alpha=0.8, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True)
+                cfg = gkv.make_config(**sh, alpha=0.8, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True, **redundancy_kwargs(args))
                 cache = gkv.GKVCache(cfg, dev)
+                red = args.redundancy is not None
                 case = synth.eviction_case(synth.BASE_SEED + 3, batch=batch, h_q=sh["h_q"], h_kv=H, b=b, buffer=sh["buffer"],
                                            w=w, n_planted=math.ceil(0.01 * l), device=dev)
                 cache.k[0].copy_(case.k); cache.v[0].copy_(case.v); cache.f[0].copy_(case.f_prev)
@@ -350,13 +363,17 @@ def run_sweep(args) -> dict:
                     cache.sacc.copy_(sums0); cache.f.copy_(f0)
                     cache.set_state(0, l, n_h, sh["s"], True)
 
-                t = {k: [] for k in ("score", "merge", "select", "compact", "fused", "recompute")}
+                t = {k: [] for k in ("score", "merge", "select", "compact", "fused", "recompute", "redundancy")}
                 moved = 0.0
                 l0 = gkv.gkv_launch_count(cache.ctx)
                 for it in range(reps + 3):
-                    e = [ev() for _ in range(9)]
+                    e = [ev() for _ in range(11)]
                     restore()
                     e[0].record(); cache.evict_stage(0, gkv.GKV_STAGE_SCORE, q_win)
+                    e[9].record()
+                    if red:
+                        cache.evict_stage(0, gkv.GKV_STAGE_REDUNDANCY)
+                    e[10].record()
                     e[1].record(); cache.evict_stage(0, gkv.GKV_STAGE_MERGE)
                     e[2].record(); cache.evict_stage(0, gkv.GKV_STAGE_SELECT, None, kept)
                     e[3].record(); cache.evict_stage(0, gkv.GKV_STAGE_COMPACT)
@@ -368,7 +385,7 @@ def run_sweep(args) -> dict:
                     e[7].record(); cache.evict(0, q_win, kept); e[8].record()
                     torch.cuda.synchronize()
                     if it >= 3:
-                        for k, (a, z) in zip(t, ((0, 1), (1, 2), (2, 3), (3, 4), (5, 6), (7, 8))):
+                        for k, (a, z) in zip(t, ((0, 9), (1, 2), (2, 3), (3, 4), (5, 6), (7, 8), (9, 10))):
                             t[k].append(e[a].elapsed_time(e[z]))
                 cache.poll()
                 launches += gkv.gkv_launch_count(cache.ctx) - l0
@@ -380,6 +397,7 @@ def run_sweep(args) -> dict:
                               "fused_GBps": eb / (med["fused"] * 1e-3) / 1e9, "fused_frac": eb / (med["fused"] * 1e-3) / 1e9 / peak_gbs,
                               "fused_bytes": eb, "kv_bytes_resident": 2.0 * units * C * 256,
                               "score_TFLOPs": flops / (med["score"] * 1e-3) / 1e12, "score_K_GBps": kbytes / (med["score"] * 1e-3) / 1e9,
+                              "redundancy_TFLOPs": (2.0 * units * l * l * 128 / (med["redundancy"] * 1e-3) / 1e12) if red else None,
                               "scored_kv_tokens_per_s": units * l / (med["recompute"] * 1e-3),
                               "scored_kv_tokens_per_s_window_sums": units * l / (med["fused"] * 1e-3)})
                 del cache, sums0, f0, kept, q_win
@@ -483,6 +501,9 @@ def main():
     ap.add_argument("--sweep-b", default="", help="cfg3: comma-separated budgets instead of the full sweep")
     ap.add_argument("--sweep-batch", default="", help="cfg3: comma-separated batch sizes instead of the full sweep")
     ap.add_argument("--sweep-w", default="", help="cfg3: comma-separated windows instead of the full sweep")
+    ap.add_argument("--redundancy", type=float, default=None, metavar="LAMBDA",
+                    help="select on LAMBDA * F - (1 - LAMBDA) * R' (redundancy term on; adds two launches per eviction)")
+    ap.add_argument("--redundancy-threshold", type=float, default=0.5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

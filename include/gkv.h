@@ -79,6 +79,17 @@ typedef struct {
     int32_t fuse_window_scores; /* 1: gkv_decode_attn adds each window token's group-max attention
                                    row to sacc, and gkv_evict needs no q_window                 */
     int32_t track_positions;    /* 1: pos carries original token positions through compaction   */
+    /* Redundancy term of the appendix on combining the global score with other methods (off when
+     * use_redundancy == 0; the remaining fields are then ignored): the selection runs on
+     * lambda * F - (1 - lambda) * R', R' the max-normalised softmax of each key's summed cosine
+     * similarity to the cached keys; F itself is what is recorded for the next step. The paper
+     * reports lambda = 0.7 / 0.9 as best for its two models and gives no value for the similarity
+     * threshold, the number of protected recent tokens or epsilon: they are the caller's. */
+    int32_t use_redundancy;
+    float redundancy_lambda;    /* in [0,1]                                                       */
+    float redundancy_threshold; /* tau > 0: cosine similarities below it count as 0              */
+    int32_t redundancy_recent;  /* this many most recent tokens are never rated redundant, >= 0  */
+    float redundancy_eps;       /* epsilon of the key normalisation K / (|K| + eps), >= 0        */
 } gkv_config;
 
 typedef struct { uint64_t k, v, f, sacc, pos, len, workspace, staging; } gkv_sizes; /* bytes      */
@@ -125,6 +136,9 @@ gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const voi
  *   q_window != NULL : the local score is recomputed from the window queries and K (Eq. 1-2),
  *                      each window token seeing the keys up to and including its own.
  *   kept_idx_out     : optional; receives the pre-compaction row index of every kept row.
+ * With use_redundancy the step first computes every key's redundancy level (two more launches: key
+ * norms, then the thresholded cosine-similarity sums on the tensor cores) and selects on the
+ * combined score of the appendix.
  * If len <= b nothing is evicted: the call only resets since_evict and sacc.
  * layer = -1 compresses all layers in one launch (leading [n_layers] dimension on the arguments).
  * Errors: STATE (no valid window scores and no q_window; len < w), INVALID_ARG, CUDA. */
@@ -135,7 +149,8 @@ gkv_status gkv_evict(gkv_ctx* ctx, int32_t layer, const void* q_window, int32_t*
  * through the workspace and must be called in order SCORE (only with q_window) -> MERGE ->
  * SELECT -> COMPACT on one layer (or -1); after COMPACT the state equals that after gkv_evict.
  * Results are identical to gkv_evict. Errors: as gkv_evict; STATE for an out-of-order stage. */
-typedef enum { GKV_STAGE_SCORE = 0, GKV_STAGE_MERGE = 1, GKV_STAGE_SELECT = 2, GKV_STAGE_COMPACT = 3 } gkv_stage;
+typedef enum { GKV_STAGE_SCORE = 0, GKV_STAGE_MERGE = 1, GKV_STAGE_SELECT = 2, GKV_STAGE_COMPACT = 3,
+               GKV_STAGE_REDUNDANCY = 4 /* only with use_redundancy: after SCORE (if any), before MERGE */ } gkv_stage;
 gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const void* q_window,
                            int32_t* kept_idx_out, void* stream);
 
@@ -174,6 +189,13 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
 gkv_status gkv_decode_attn_static(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                   void* v_cache, void* out, int32_t batch, int32_t n_q_heads,
                                   int32_t n_kv_heads, int32_t capacity, int32_t len, void* stream);
+
+/* With use_redundancy: copies the redundancy levels cbar (summed thresholded cosine similarity of every
+ * cached key, 0 for the protected recent tokens) that the last gkv_evict / REDUNDANCY stage computed for
+ * `layer` into out_device [batch][n_kv_heads][C] fp32 (device pointer), asynchronously on `stream`.
+ * The values refer to the rows as they were BEFORE that step's compaction.
+ * Errors: INVALID_ARG (NULL, bad layer, layer = -1), STATE (redundancy term off), CUDA. */
+gkv_status gkv_get_redundancy(gkv_ctx* ctx, int32_t layer, float* out_device, void* stream);
 
 /* Host counters of one layer (no synchronisation): cache length, rows with history, tokens
  * decoded since the last compression. Any output pointer may be NULL. */

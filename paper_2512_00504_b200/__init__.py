@@ -18,12 +18,13 @@ from pathlib import Path
 _PKG = Path(__file__).resolve().parent
 _ROOT = _PKG.parent
 LIB_PATH = _PKG / "libgkv.so"
-_SOURCES = ["gkv_api.cu", "gkv_decode.cu", "gkv_evict.cu", "gkv_score.cu", "gkv_score_tc.cu", "gkv_static_scratch.cu"]
+_SOURCES = ["gkv_api.cu", "gkv_decode.cu", "gkv_evict.cu", "gkv_score.cu", "gkv_score_tc.cu", "gkv_redundancy.cu",
+            "gkv_static_scratch.cu"]
 
 GKV_OK, GKV_ERR_INVALID_ARG, GKV_ERR_STATE, GKV_ERR_CAPACITY, GKV_ERR_CUDA, GKV_ERR_TIMEOUT, GKV_ERR_UNSUPPORTED, \
     GKV_ERR_SCRATCH_LIMIT = range(8)
 GKV_MODE_MAX, GKV_MODE_MEAN, GKV_MODE_SUM, GKV_MODE_LOCAL = range(4)
-GKV_STAGE_SCORE, GKV_STAGE_MERGE, GKV_STAGE_SELECT, GKV_STAGE_COMPACT = range(4)
+GKV_STAGE_SCORE, GKV_STAGE_MERGE, GKV_STAGE_SELECT, GKV_STAGE_COMPACT, GKV_STAGE_REDUNDANCY = range(5)
 
 
 class GKVError(RuntimeError):
@@ -36,7 +37,9 @@ class gkv_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "budget", "buffer", "window", "interval")] + \
                [("alpha", ctypes.c_float), ("mode", ctypes.c_int32), ("fuse_window_scores", ctypes.c_int32),
-                ("track_positions", ctypes.c_int32)]
+                ("track_positions", ctypes.c_int32), ("use_redundancy", ctypes.c_int32),
+                ("redundancy_lambda", ctypes.c_float), ("redundancy_threshold", ctypes.c_float),
+                ("redundancy_recent", ctypes.c_int32), ("redundancy_eps", ctypes.c_float)]
 
 
 class gkv_sizes(ctypes.Structure):
@@ -89,6 +92,7 @@ def lib() -> ctypes.CDLL:
         L.gkv_decode_attn_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.gkv_evict_host.argtypes = [vp, i32, vp, vp, vp]
         L.gkv_get_state.argtypes = [vp, i32, P(i32), P(i32), P(i32)]
+        L.gkv_get_redundancy.argtypes = [vp, i32, vp, vp]
         L.gkv_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.gkv_decode_attn_static.restype = ctypes.c_int
         L.gkv_launch_count.argtypes = [vp]
@@ -100,7 +104,7 @@ def lib() -> ctypes.CDLL:
         L.gkv_destroy.argtypes = [vp]
         L.gkv_destroy.restype = None
         for name in ("gkv_query_sizes", "gkv_init", "gkv_set_state", "gkv_decode_attn", "gkv_evict", "gkv_evict_stage",
-                     "gkv_decode_attn_host", "gkv_evict_host", "gkv_get_state", "gkv_poll_device_status",
+                     "gkv_decode_attn_host", "gkv_evict_host", "gkv_get_state", "gkv_get_redundancy", "gkv_poll_device_status",
                      "gkv_memory_model"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
@@ -128,9 +132,14 @@ def _stream():
 
 
 def make_config(*, n_layers, batch, h_q, h_kv, d=128, b, buffer, w, s, alpha=0.8, mode=GKV_MODE_MAX,
-                fuse_window_scores=True, track_positions=False, **_ignored) -> gkv_config:
+                fuse_window_scores=True, track_positions=False, redundancy_lambda=None, redundancy_threshold=0.5,
+                redundancy_recent=None, redundancy_eps=1e-6, **_ignored) -> gkv_config:
+    """redundancy_lambda=None leaves the redundancy term off; redundancy_recent defaults to the window."""
+    use = redundancy_lambda is not None
     return gkv_config(n_layers, batch, h_q, h_kv, d, b, buffer, w, s, alpha, mode,
-                      int(fuse_window_scores), int(track_positions))
+                      int(fuse_window_scores), int(track_positions), int(use), float(redundancy_lambda if use else 1.0),
+                      float(redundancy_threshold), int(w if redundancy_recent is None else redundancy_recent),
+                      float(redundancy_eps))
 
 
 # ------------------------------------------------------------------ C-ABI calls, same names
@@ -195,6 +204,10 @@ def gkv_get_state(ctx, layer):
     a, b, c = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
     _check(lib().gkv_get_state(ctx, layer, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)), "gkv_get_state")
     return a.value, b.value, c.value
+
+
+def gkv_get_redundancy(ctx, layer, out):
+    _check(lib().gkv_get_redundancy(ctx, layer, _ptr(out), _stream()), "gkv_get_redundancy")
 
 
 def gkv_launch_count(ctx) -> int:
@@ -262,6 +275,13 @@ class GKVCache:
 
     def state(self, layer=0):
         return gkv_get_state(self.ctx, layer)
+
+    def redundancy(self, layer=0):
+        """cbar [batch][h_kv][C] of the last eviction of `layer` (redundancy term on)."""
+        import torch
+        out = torch.empty((self.cfg.batch, self.cfg.n_kv_heads, self.C), dtype=torch.float32, device=self.device)
+        gkv_get_redundancy(self.ctx, layer, out)
+        return out
 
     def poll(self):
         gkv_poll_device_status(self.ctx)

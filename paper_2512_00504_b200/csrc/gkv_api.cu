@@ -27,6 +27,11 @@ gkv_status check_config(const gkv_config* c) {
     if (!(c->alpha >= 0.f && c->alpha <= 1.f)) return GKV_ERR_INVALID_ARG;
     if (c->mode < GKV_MODE_MAX || c->mode > GKV_MODE_LOCAL) return GKV_ERR_INVALID_ARG;
     if (c->n_q_heads % c->n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
+    if (c->use_redundancy) {
+        if (!(c->redundancy_lambda >= 0.f && c->redundancy_lambda <= 1.f)) return GKV_ERR_INVALID_ARG;
+        if (!(c->redundancy_threshold > 0.f) || !(c->redundancy_eps >= 0.f) || c->redundancy_recent < 0)
+            return GKV_ERR_INVALID_ARG;
+    }
     if (c->head_dim != kHeadDim) return GKV_ERR_UNSUPPORTED;
     if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return GKV_ERR_UNSUPPORTED;
     if (c->budget + c->buffer > kMaxCapacity) return GKV_ERR_UNSUPPORTED;
@@ -62,6 +67,10 @@ void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     w->logits = off;   off = align_up(off + logits);
     w->kept = off;     off = align_up(off + upl * c->budget * sizeof(int32_t));
     w->fscratch = off; off = align_up(off + upl * C * sizeof(float));
+    const uint64_t red = c->use_redundancy ? 1 : 0;   // the redundancy term's scratch exists only when it is on
+    w->fsel = off;     off = align_up(off + red * upl * C * sizeof(float));
+    w->inv_norm = off; off = align_up(off + red * L * upl * C * sizeof(float));
+    w->cbar = off;     off = align_up(off + red * L * upl * C * sizeof(float));
     w->total = off;
 }
 
@@ -142,7 +151,30 @@ EvictLaunch make_evict(gkv_ctx* ctx, int l0, int nl, int32_t* kept_out) {
     p.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
     p.layer0 = l0; p.n_layers = nl; p.L_total = c.n_layers; p.batch = c.batch; p.h_kv = c.n_kv_heads;
     p.C = ctx->C; p.b = c.budget; p.w = c.window; p.alpha = c.alpha; p.mode = c.mode;
+    p.cbar = c.use_redundancy ? ws_ptr<float>(ctx, ctx->ws.cbar) : nullptr;
+    p.fsel_ws = ws_ptr<float>(ctx, ctx->ws.fsel);
+    p.lambda = c.redundancy_lambda;
     return p;
+}
+
+// Redundancy level of every cached key of the layers [l0, l0 + nl): key norms, then the thresholded
+// cosine-similarity sums (two launches).
+gkv_status launch_redundancy_for(gkv_ctx* ctx, int l0, int nl, cudaStream_t s) {
+    RedundancyLaunch rp;
+    const gkv_config& c = ctx->cfg;
+    rp.k_cache = static_cast<const __nv_bfloat16*>(ctx->buf.k);
+    rp.len = static_cast<const int32_t*>(ctx->buf.len);
+    rp.inv_norm = ws_ptr<float>(ctx, ctx->ws.inv_norm);
+    rp.cbar = ws_ptr<float>(ctx, ctx->ws.cbar);
+    rp.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
+    rp.layer0 = l0; rp.n_layers = nl; rp.batch = c.batch; rp.h_kv = c.n_kv_heads; rp.C = ctx->C;
+    rp.recent = c.redundancy_recent; rp.tau = c.redundancy_threshold; rp.eps = c.redundancy_eps;
+    if (launch_keynorm(rp, s) != cudaSuccess || launch_redundancy(rp, ctx->tm_k, s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GKV_ERR_CUDA;
+    }
+    ctx->launches += 2;
+    return GKV_OK;
 }
 
 gkv_status launch_score_for(gkv_ctx* ctx, int l0, int nl, const void* q_window, cudaStream_t s) {
@@ -195,6 +227,7 @@ void after_evict(gkv_ctx* ctx, int l0, int nl, bool noop) {
         ctx->since_evict[i] = 0;
         ctx->sacc_valid[i] = 0;
         ctx->stage_next[i] = 0;
+        ctx->cbar_valid[i] = 0;
     }
 }
 
@@ -252,7 +285,8 @@ gkv_status gkv_init(gkv_ctx** out, const gkv_config* cfg, const gkv_buffers* b, 
              cudaMemsetAsync(b->workspace, 0, ctx->sizes.workspace, s) == cudaSuccess &&
              (!cfg->track_positions || cudaMemsetAsync(b->pos, 0, ctx->sizes.pos, s) == cudaSuccess);
     }
-    if (ok) ok = decode_kernel_setup() == cudaSuccess && score_kernel_setup() == cudaSuccess && score_tc_kernel_setup() == cudaSuccess;
+    if (ok) ok = decode_kernel_setup() == cudaSuccess && score_kernel_setup() == cudaSuccess && score_tc_kernel_setup() == cudaSuccess &&
+                 redundancy_kernel_setup() == cudaSuccess;
     if (ok) {
         const uint64_t rows = (uint64_t)cfg->n_layers * ctx->units_per_layer * ctx->C;
         ok = encode_map(&ctx->tm_k, b->k, rows) == GKV_OK && encode_map(&ctx->tm_v, b->v, rows) == GKV_OK;
@@ -267,6 +301,7 @@ gkv_status gkv_init(gkv_ctx** out, const gkv_config* cfg, const gkv_buffers* b, 
     ctx->since_evict.assign(cfg->n_layers, 0);
     ctx->sacc_valid.assign(cfg->n_layers, 0);
     ctx->stage_next.assign(cfg->n_layers, 0);
+    ctx->cbar_valid.assign(cfg->n_layers, 0);
     *out = ctx;
     return GKV_OK;
 }
@@ -294,6 +329,7 @@ gkv_status gkv_set_state(gkv_ctx* ctx, int32_t layer, int32_t len, int32_t n_his
         ctx->since_evict[i] = since_evict;
         ctx->sacc_valid[i] = window_scores_valid ? 1 : 0;
         ctx->stage_next[i] = 0;
+        ctx->cbar_valid[i] = 0;
     }
     return GKV_OK;
 }
@@ -337,6 +373,7 @@ gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const voi
         ctx->len[i] += 1;
         ctx->since_evict[i] += 1;
         ctx->stage_next[i] = 0;
+        ctx->cbar_valid[i] = 0;
         // window sums written by hand are stale once further tokens are decoded without accumulation
         if (!p.accum) ctx->sacc_valid[i] = 0;
     }
@@ -359,6 +396,10 @@ gkv_status gkv_evict(gkv_ctx* ctx, int32_t layer, const void* q_window, int32_t*
         st = launch_score_for(ctx, l0, nl, q_window, s);
         if (st != GKV_OK) return st;
     }
+    if (ctx->cfg.use_redundancy) {
+        st = launch_redundancy_for(ctx, l0, nl, s);
+        if (st != GKV_OK) return st;
+    }
     const EvictLaunch p = make_evict(ctx, l0, nl, kept_idx_out);
     if (launch_evict_fused(p, s) != cudaSuccess) {
         (void)cudaGetLastError();
@@ -373,7 +414,8 @@ gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const voi
                            void* stream) {
     int l0, nl;
     bool noop;
-    if (stage < GKV_STAGE_SCORE || stage > GKV_STAGE_COMPACT) return GKV_ERR_INVALID_ARG;
+    if (stage < GKV_STAGE_SCORE || stage > GKV_STAGE_REDUNDANCY) return GKV_ERR_INVALID_ARG;
+    if (stage == GKV_STAGE_REDUNDANCY && !ctx->cfg.use_redundancy) return GKV_ERR_INVALID_ARG;
     gkv_status st = evict_precheck(ctx, layer, false, &l0, &nl, &noop);
     if (st != GKV_OK) return st;
     if (nl != 1) return GKV_ERR_UNSUPPORTED;  // the staged scratch holds one layer
@@ -395,12 +437,20 @@ gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const voi
         next = GKV_STAGE_MERGE;
         return GKV_OK;
     }
+    if (stage == GKV_STAGE_REDUNDANCY) {
+        if (next != 0 && next != GKV_STAGE_MERGE) return GKV_ERR_STATE;
+        st = launch_redundancy_for(ctx, l0, nl, s);
+        if (st != GKV_OK) return st;
+        ctx->cbar_valid[l0] = 1;
+        return GKV_OK;
+    }
     const EvictLaunch p = make_evict(ctx, l0, nl, stage == GKV_STAGE_SELECT ? kept_idx_out : nullptr);
     cudaError_t e;
     if (stage == GKV_STAGE_MERGE) {
         if (next != 0 && next != GKV_STAGE_MERGE) return GKV_ERR_STATE;
         const bool fused_ready = ctx->cfg.fuse_window_scores && ctx->since_evict[l0] == ctx->cfg.interval;
         if (!fused_ready && !ctx->sacc_valid[l0]) return GKV_ERR_STATE;
+        if (ctx->cfg.use_redundancy && !ctx->cbar_valid[l0]) return GKV_ERR_STATE;   // REDUNDANCY stage first
         e = launch_evict_merge(p, s);
         if (e == cudaSuccess) next = GKV_STAGE_SELECT;
     } else if (stage == GKV_STAGE_SELECT) {
@@ -464,6 +514,18 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
     if (kept_idx_out_host && will_evict &&
         cudaMemcpyAsync(kept_idx_out_host, dkept, kb, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return GKV_ERR_CUDA;
+    return GKV_OK;
+}
+
+gkv_status gkv_get_redundancy(gkv_ctx* ctx, int32_t layer, float* out_device, void* stream) {
+    if (!ctx || !out_device || layer < 0 || layer >= ctx->cfg.n_layers) return GKV_ERR_INVALID_ARG;
+    if (!ctx->cfg.use_redundancy) return GKV_ERR_STATE;
+    const size_t per_layer = (size_t)ctx->units_per_layer * ctx->C;
+    if (cudaMemcpyAsync(out_device, ws_ptr<float>(ctx, ctx->ws.cbar) + layer * per_layer, per_layer * sizeof(float),
+                        cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GKV_ERR_CUDA;
+    }
     return GKV_OK;
 }
 

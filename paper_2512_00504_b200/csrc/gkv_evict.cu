@@ -78,6 +78,24 @@ __device__ void merge_phase(const float* __restrict__ sums, const float* __restr
     __syncthreads();
 }
 
+// Appendix on combining the global score with other methods: R = softmax(cbar), R' = R / max R =
+// exp(cbar - max cbar) (maximum over all n cached tokens), selection score = lambda F - (1 - lambda) R'.
+__device__ void combine_phase(const float* __restrict__ cbar, const float* s_f, float* s_sel, int n, int n_c,
+                              float lambda, EvictShared* sh, int tid) {
+    float mx = -INFINITY;
+    for (int t = tid; t < n; t += kEvictThreads) mx = fmaxf(mx, cbar[t]);
+    mx = block_max(mx, sh->warp_max, tid);
+    for (int t = tid; t < n_c; t += kEvictThreads)
+        s_sel[t] = lambda * s_f[t] - (1.f - lambda) * fast_exp2((cbar[t] - mx) * 1.4426950408889634f);
+    __syncthreads();
+}
+
+// fp32 bit pattern -> unsigned integer with the same order (negative values included: the combined
+// score of the redundancy term is lambda * F - (1 - lambda) * R').
+__device__ __forceinline__ uint32_t ordered_bits(uint32_t x) {
+    return x ^ (static_cast<uint32_t>(static_cast<int32_t>(x) >> 31) | 0x80000000u);
+}
+
 // Top-n_keep of s_f[0..n_c) with ties toward the lower index; kept rows ascending into s_kept,
 // followed by the w window rows n_c .. n_c+w-1. Returns (CTA-uniform) the first row that moves.
 __device__ int select_phase(const float* s_f, int* s_kept, int n_c, int n_keep, int w, EvictShared* sh, int tid) {
@@ -90,7 +108,7 @@ __device__ int select_phase(const float* s_f, int* s_kept, int n_c, int n_keep, 
         __syncthreads();
         const uint32_t mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
         for (int t = tid; t < n_c; t += kEvictThreads) {
-            const uint32_t x = bits[t];
+            const uint32_t x = ordered_bits(bits[t]);
             if ((x & mask) == prefix) atomicAdd(&sh->hist[(x >> shift) & 255], 1);
         }
         __syncthreads();
@@ -106,14 +124,14 @@ __device__ int select_phase(const float* s_f, int* s_kept, int n_c, int n_keep, 
         prefix |= static_cast<uint32_t>(sh->digit) << shift;
         k = sh->k_rem;
     }
-    // prefix = bit pattern T of the n_keep-th largest score; take everything above it and the
+    // prefix = ordered bit pattern T of the n_keep-th largest score; take everything above it and the
     // first k rows equal to it
     const uint32_t T = prefix;
     const int per = (n_c + kEvictThreads - 1) / kEvictThreads;
     const int t0 = tid * per, t1 = min(t0 + per, n_c);
     int gt = 0, eq = 0;
     for (int t = t0; t < t1; ++t) {
-        const uint32_t x = bits[t];
+        const uint32_t x = ordered_bits(bits[t]);
         gt += (x > T);
         eq += (x == T);
     }
@@ -122,7 +140,7 @@ __device__ int select_phase(const float* s_f, int* s_kept, int n_c, int n_keep, 
     int gt_before = (packed & 0xffff) - gt, eq_before = (packed >> 16) - eq;
     int first_drop = n_c;
     for (int t = t0; t < t1; ++t) {
-        const uint32_t x = bits[t];
+        const uint32_t x = ordered_bits(bits[t]);
         if (x > T) {
             s_kept[gt_before + min(eq_before, k)] = t;
             ++gt_before;
@@ -275,15 +293,18 @@ __device__ void publish_state(const EvictLaunch& p, const UnitIndex& u, int ctas
     }
 }
 
+// s_sel (the scores the selection runs on) is s_f itself unless the redundancy term is on.
 __device__ __forceinline__ void carve(uint8_t* smem, const EvictLaunch& p, float** s_f, int** s_kept, int** s_pos,
-                                      EvictShared** sh) {
+                                      EvictShared** sh, float** s_sel) {
     *sh = reinterpret_cast<EvictShared*>(smem);
     *s_f = reinterpret_cast<float*>(smem + sizeof(EvictShared));
     *s_kept = reinterpret_cast<int*>(*s_f + p.C);
     *s_pos = *s_kept + p.b;
+    *s_sel = p.cbar ? reinterpret_cast<float*>(*s_pos + (p.pos ? p.C : 0)) : *s_f;
 }
 static size_t evict_state_bytes(const EvictLaunch& p) {
-    return sizeof(EvictShared) + sizeof(float) * p.C + sizeof(int) * p.b + (p.pos ? sizeof(int) * p.C : 0);
+    return sizeof(EvictShared) + sizeof(float) * p.C + sizeof(int) * p.b + (p.pos ? sizeof(int) * p.C : 0) +
+           (p.cbar ? sizeof(float) * p.C : 0);
 }
 static size_t evict_smem_bytes(const EvictLaunch& p) { return evict_state_bytes(p); }
 // the fused kernel adds the copy ring, 128-byte aligned behind the score state
@@ -293,8 +314,8 @@ static size_t evict_ring_offset(const EvictLaunch& p) { return (evict_state_byte
 // Whole step in one launch: merge -> select -> score-state update -> K/V compaction.
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const EvictLaunch p, int ring_offset) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel);
     const int tid = threadIdx.x;
     const UnitIndex u = unit_of(p, blockIdx.x);
     const int n = p.len[u.lseq_global];
@@ -306,7 +327,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const Ev
     }
     const int n_c = n - p.w;
     merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
-    const int r_first = select_phase(s_f, s_kept, n_c, p.b - p.w, p.w, sh, tid);
+    if (p.cbar) combine_phase(p.cbar + (size_t)u.unit * p.C, s_f, s_sel, n, n_c, p.lambda, sh, tid);
+    const int r_first = select_phase(s_sel, s_kept, n_c, p.b - p.w, p.w, sh, tid);
     write_score_state(p, u, s_f, s_kept, s_pos, n, tid);
     compact_phase_async(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
                         p.b, r_first, evict_smem + ring_offset, tid);
@@ -317,8 +339,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const Ev
 // The same step as separate launches (timed one by one); they hand over through the workspace.
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const EvictLaunch p) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel);
     const int tid = threadIdx.x;
     const UnitIndex u = unit_of(p, blockIdx.x);
     const int n = p.len[u.lseq_global];
@@ -328,12 +350,17 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const Ev
     merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
     float* out = p.f_ws + (size_t)u.unit_local * p.C;
     for (int t = tid; t < n_c; t += kEvictThreads) out[t] = s_f[t];
+    if (p.cbar) {
+        combine_phase(p.cbar + (size_t)u.unit * p.C, s_f, s_sel, n, n_c, p.lambda, sh, tid);
+        float* out2 = p.fsel_ws + (size_t)u.unit_local * p.C;
+        for (int t = tid; t < n_c; t += kEvictThreads) out2[t] = s_sel[t];
+    }
 }
 
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const EvictLaunch p) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel);
     const int tid = threadIdx.x;
     const UnitIndex u = unit_of(p, blockIdx.x);
     const int n = p.len[u.lseq_global];
@@ -345,8 +372,12 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const E
     const int n_c = n - p.w;
     const float* in = p.f_ws + (size_t)u.unit_local * p.C;
     for (int t = tid; t < n_c; t += kEvictThreads) s_f[t] = in[t];
+    if (p.cbar) {
+        const float* in2 = p.fsel_ws + (size_t)u.unit_local * p.C;
+        for (int t = tid; t < n_c; t += kEvictThreads) s_sel[t] = in2[t];
+    }
     __syncthreads();
-    select_phase(s_f, s_kept, n_c, p.b - p.w, p.w, sh, tid);
+    select_phase(s_sel, s_kept, n_c, p.b - p.w, p.w, sh, tid);
     write_score_state(p, u, s_f, s_kept, s_pos, n, tid);
     int32_t* kw = p.kept_ws + (size_t)u.unit_local * p.b;
     for (int r = tid; r < p.b; r += kEvictThreads) kw[r] = s_kept[r];
@@ -355,8 +386,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const E
 // grid = units x slices: each CTA moves one column slice of every row of its unit.
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_compact_kernel(const EvictLaunch p, int slices) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh);
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel);
     const int tid = threadIdx.x;
     const int unit_local = blockIdx.x / slices, slice = blockIdx.x - unit_local * slices;
     const UnitIndex u = unit_of(p, unit_local);

@@ -22,6 +22,9 @@ struct WorkspaceLayout {
     uint64_t logits;      // split-K window steps: per unit C x 8 fp32 scaled logits
     uint64_t kept;        // int32[units_per_layer * b]   kept lists of the staged eviction path
     uint64_t fscratch;    // fp32[units_per_layer * C]    merged scores of the staged eviction path
+    uint64_t fsel;        // fp32[units_per_layer * C]    selection scores of the staged path (redundancy term on)
+    uint64_t inv_norm;    // fp32[L * units_per_layer * C] 1 / (|K row| + eps)            (redundancy term on)
+    uint64_t cbar;        // fp32[L * units_per_layer * C] redundancy level of every row  (redundancy term on)
     uint64_t total;
 };
 
@@ -60,6 +63,20 @@ struct EvictLaunch {
     int layer0, n_layers, L_total, batch, h_kv, C, b, w;
     float alpha;
     int mode;
+    // redundancy term: selection on lambda * F - (1 - lambda) * exp(cbar - max cbar); cbar == NULL turns it off
+    const float* cbar;   // [all units][C]
+    float* fsel_ws;      // staged path scratch
+    float lambda;
+};
+
+struct RedundancyLaunch {
+    const __nv_bfloat16* k_cache;
+    const int32_t* len;
+    float* inv_norm;     // [all units][C]
+    float* cbar;         // [all units][C]
+    int32_t* status;
+    int layer0, n_layers, batch, h_kv, C, recent;
+    float tau, eps;
 };
 
 struct ScoreLaunch {
@@ -80,7 +97,7 @@ struct gkv_ctx {
     int C, g, units_per_layer;
     int device, sm_count;
     CUtensorMap tm_k, tm_v;
-    std::vector<int32_t> len, n_hist, since_evict, sacc_valid, stage_next;
+    std::vector<int32_t> len, n_hist, since_evict, sacc_valid, stage_next, cbar_valid;
     int64_t launches;
     gkv_sizes sizes;
 };
@@ -98,6 +115,9 @@ cudaError_t launch_score(const ScoreLaunch& p, const CUtensorMap& tm_k, cudaStre
 cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s);
 int score_tc_rows_per_cta(int g, int w);
 cudaError_t score_tc_kernel_setup();
+cudaError_t launch_keynorm(const RedundancyLaunch& p, cudaStream_t s);
+cudaError_t launch_redundancy(const RedundancyLaunch& p, const CUtensorMap& tm_k, cudaStream_t s);
+cudaError_t redundancy_kernel_setup();
 cudaError_t decode_kernel_setup();
 cudaError_t score_kernel_setup();
 

@@ -1,0 +1,296 @@
+// Redundancy level of every cached key (the paper's appendix on combining the global score with other
+// methods): Kbar = K / (|K| + eps), Cm = Kbar Kbar^T, entries below the threshold tau zeroed, the
+// columns of the most recent tokens zeroed, cbar[t] = sum over k of the masked column t.
+//
+// Cm is symmetric and so is the threshold mask, so the column sum of column t equals the sum over
+// row t: the thread that owns an accumulator row owns a key and adds up its own row, no
+// cross-thread reduction. The Gram matrix is taken of the RAW bf16 keys on tcgen05 (products exact,
+// fp32 accumulation) and scaled by the two inverse norms in the epilogue, so normalisation costs no
+// precision before the threshold comparison.
+//
+// Two launches: gkv_keynorm_kernel writes 1 / (|K_t| + eps) per cached row; gkv_redundancy_tc_kernel
+// (one CTA per unit and block of 256 keys) keeps its 256 keys resident in shared memory as the A
+// operand (two 128-row tiles), streams all keys of the unit as 128-key B tiles by TMA, accumulates
+// D[own key][other key] in two 256-column TMEM buffers, and 16 epilogue warps (same roles and
+// barriers as the scoring kernel) scale, threshold and add. The softmax and the max-normalisation
+// of the appendix reduce to exp(cbar - max cbar), which the eviction kernel applies.
+#include <stdlib.h>
+
+#include "gkv_common.cuh"
+#include "gkv_internal.h"
+#include "gkv_tcgen05.cuh"
+
+namespace gkv {
+
+constexpr int kRdGroups = 4;
+constexpr int kRdEpiThreads = kRdGroups * 128;
+constexpr int kRdThreads = 64 + kRdEpiThreads;
+constexpr int kRdTileKeys = 128;
+constexpr int kRdBlockRows = 256;
+constexpr int kRdMaxStages = 4;
+constexpr int kRdStageBytes = kRdTileKeys * kRowBytes;       // 32 KB: d-low half then d-high half
+constexpr int kRdABytes = kRdBlockRows * kRowBytes;          // 64 KB
+constexpr int kRdAccCols = 256;
+constexpr uint32_t kRdTmemCols = 512;
+
+// ---------------------------------------------------------------------------------------------
+// inv[unit][t] = 1 / (|K[unit][t]| + eps) for t < len, 0 beyond. 16 lanes per row, 16 rows per pass.
+__global__ void __launch_bounds__(256) gkv_keynorm_kernel(const RedundancyLaunch p) {
+    const int blocks_per_unit = (p.C + 127) / 128;
+    const int unit_local = blockIdx.x / blocks_per_unit;
+    const int rb = blockIdx.x - unit_local * blocks_per_unit;
+    const int ls = unit_local / p.h_kv;
+    const int lseq_global = p.layer0 * p.batch + ls;
+    const long unit = (long)lseq_global * p.h_kv + (unit_local - ls * p.h_kv);
+    const int n = p.len[lseq_global];
+    const int sub = threadIdx.x >> 4, c = threadIdx.x & 15;
+    const uint4* k4 = reinterpret_cast<const uint4*>(p.k_cache + (size_t)unit * p.C * kHeadDim);
+    float* inv = p.inv_norm + (size_t)unit * p.C;
+    for (int it = 0; it < 8; ++it) {                   // warp-uniform trip count: the shuffles below need every lane
+        const int r = rb * 128 + it * 16 + sub;
+        float ss = 0.f;
+        if (r < n) {
+            const uint4 x = k4[(size_t)r * 16 + c];
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xffff0000u);
+                ss = fmaf(lo, lo, ss);
+                ss = fmaf(hi, hi, ss);
+            }
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (c == 0 && r < p.C) inv[r] = (r < n) ? __frcp_rn(__fsqrt_rn(ss) + p.eps) : 0.f;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+struct __align__(8) RedundancyTail {
+    uint64_t a_full;
+    uint64_t k_full[kRdMaxStages];
+    uint64_t k_empty[kRdMaxStages];
+    uint64_t d_full[2];
+    uint64_t d_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int issued;
+};
+
+__device__ __forceinline__ void rd_abort(RedundancyTail* tail, int32_t* status, int where) {
+    if (atomicExch(&tail->abort_flag, 1) == 0 && atomicCAS(status, 0, kStatusTimeout) == 0) {
+        status[1] = where;
+        status[2] = blockIdx.x;
+    }
+}
+__device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kRdEpiThreads) : "memory"); }
+
+__global__ void __launch_bounds__(kRdThreads, 1)
+gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUtensorMap tm_k, int blocks_per_unit,
+                         int stages) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    constexpr int a_half = kRdABytes / 2;
+    uint8_t* a_smem = smem;
+    uint8_t* k_smem = smem + kRdABytes;
+    const int c_pad = (p.C + 127) & ~127;
+    float* s_inv = reinterpret_cast<float*>(k_smem + stages * kRdStageBytes);   // [c_pad] inverse norms of the unit, 0 beyond n
+    float* s_part = s_inv + c_pad;                                              // [groups][128] partial row sums
+    RedundancyTail* tail = reinterpret_cast<RedundancyTail*>(s_part + kRdGroups * 128);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int unit_local = blockIdx.x / blocks_per_unit;
+    const int a0 = (blockIdx.x - unit_local * blocks_per_unit) * kRdBlockRows;   // first key of this CTA's block
+    const int ls = unit_local / p.h_kv;
+    const int lseq_global = p.layer0 * p.batch + ls;
+    const long unit = (long)lseq_global * p.h_kv + (unit_local - ls * p.h_kv);
+    const int n = p.len[lseq_global];
+    if (a0 >= n) return;                              // the whole CTA: no key of the cache in this block
+    const int T = (n + kRdTileKeys - 1) / kRdTileKeys;
+    const int row0 = (int)(unit * p.C);
+    const int MT = (min(kRdBlockRows, n - a0) + 127) >> 7;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&tail->a_full), 1);
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(smem_u32(&tail->k_full[s]), 1);
+            mbar_init(smem_u32(&tail->k_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tail->d_full[b]), 1);
+            mbar_init(smem_u32(&tail->d_empty[b]), kRdEpiThreads / 32);
+        }
+        mbar_init(smem_u32(&tail->drain), 1);
+        tail->abort_flag = 0;
+        tail->issued = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {   // whole warp: all of the SM's tensor memory (one CTA per SM by shared memory)
+        tmem_alloc(smem_u32(&tail->tmem_base), kRdTmemCols);
+        tmem_relinquish_alloc_permit();
+        tmem_fence_before_sync();
+    }
+    {
+        const float* ginv = p.inv_norm + (size_t)unit * p.C;
+        for (int t = tid; t < c_pad; t += kRdThreads) s_inv[t] = (t < n) ? ginv[t] : 0.f;
+    }
+    __syncthreads();
+    tmem_fence_after_sync();
+    const uint32_t tmem_base = *(volatile uint32_t*)&tail->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&tm_k);
+            const uint32_t abar = smem_u32(&tail->a_full);
+            mbar_arrive_expect_tx(abar, (uint32_t)MT * 128 * kRowBytes);
+            for (int rb = 0; rb < 2 * MT; ++rb) {      // 64-row boxes; rows past the tensor's end arrive as zeros
+                tma_load_2d(smem_u32(a_smem + (size_t)rb * kBoxBytes), &tm_k, 0, row0 + a0 + rb * 64, abar);
+                tma_load_2d(smem_u32(a_smem + a_half + (size_t)rb * kBoxBytes), &tm_k, 64, row0 + a0 + rb * 64, abar);
+            }
+            for (int i = 0, s = 0, round = 0; i < T; ++i) {
+                if (round > 0 && !tc_wait(smem_u32(&tail->k_empty[s]), (round - 1) & 1, &tail->abort_flag)) {
+                    rd_abort(tail, p.status, 31);
+                    break;
+                }
+                const uint32_t bar = smem_u32(&tail->k_full[s]);
+                const uint32_t dst = smem_u32(k_smem + (size_t)s * kRdStageBytes);
+                const int y = row0 + i * kRdTileKeys;
+                mbar_arrive_expect_tx(bar, kRdStageBytes);
+                tma_load_2d(dst, &tm_k, 0, y, bar);
+                tma_load_2d(dst + kBoxBytes, &tm_k, 0, y + 64, bar);
+                tma_load_2d(dst + 2 * kBoxBytes, &tm_k, 64, y, bar);
+                tma_load_2d(dst + 3 * kBoxBytes, &tm_k, 64, y + 64, bar);
+                *(volatile int*)&tail->issued = i + 1;
+                if (++s == stages) { s = 0; ++round; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = tc_wait(smem_u32(&tail->a_full), 0, &tail->abort_flag);
+            if (!ok) rd_abort(tail, p.status, 32);
+            const uint32_t a_lo = umma_desc_lo(smem_u32(a_smem)), k_lo = umma_desc_lo(smem_u32(k_smem));
+            const uint32_t idesc = umma_idesc_bf16_m128(kRdTileKeys);
+            for (int i = 0, s = 0, round = 0; ok && i < T; ++i) {
+                const int buf = i & 1;
+                if (i >= 2 && !tc_wait(smem_u32(&tail->d_empty[buf]), ((i >> 1) - 1) & 1, &tail->abort_flag)) {
+                    rd_abort(tail, p.status, 33);
+                    break;
+                }
+                if (!tc_wait(smem_u32(&tail->k_full[s]), round & 1, &tail->abort_flag)) {
+                    rd_abort(tail, p.status, 34);
+                    break;
+                }
+                tmem_fence_after_sync();
+                const uint32_t ks_lo = k_lo + (uint32_t)s * (kRdStageBytes >> 4);
+                const uint32_t d = tmem_base + (uint32_t)buf * kRdAccCols;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    umma_bf16(d, umma_desc(a_lo + umma_kstep(ks, a_half)), umma_desc(ks_lo + umma_kstep(ks, kRdStageBytes / 2)),
+                              idesc, ks > 0);
+                if (MT == 2) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_bf16(d + 128, umma_desc(a_lo + ((128 * 128) >> 4) + umma_kstep(ks, a_half)),
+                                  umma_desc(ks_lo + umma_kstep(ks, kRdStageBytes / 2)), idesc, ks > 0);
+                }
+                umma_commit(smem_u32(&tail->k_empty[s]));
+                umma_commit(smem_u32(&tail->d_full[buf]));
+                if (++s == stages) { s = 0; ++round; }
+            }
+            umma_commit(smem_u32(&tail->drain));     // everything issued has completed before TMEM is given back
+            mbar_wait_bounded(smem_u32(&tail->drain), 0);
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int wg = (warp - 2) >> 2;
+        const int q4 = warp & 3;
+        const int L = q4 * 32 + lane;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        // two row tiles: two groups per tile, 64 columns each; one tile: four groups, 32 columns each
+        const int rl = (MT == 2) ? (wg >> 1) * 128 + L : L;
+        const int col0 = (MT == 2) ? (wg & 1) * 64 : wg * 32;
+        const int nch = (MT == 2) ? 2 : 1;
+        const uint32_t t_p = t_lane + (uint32_t)((MT == 2) ? (wg >> 1) * 128 + col0 : col0);
+        const int row = a0 + rl;                       // the key this thread sums for
+        const float inv_r = (row < n) ? s_inv[row] : 0.f;
+        const float thr = (row < n) ? __fdiv_rn(p.tau, inv_r) : INFINITY;   // Cm >= tau  <=>  G * inv_col >= tau / inv_row
+        float sum = 0.f;
+        bool ok = true;
+        for (int i = 0; i < T; ++i) {
+            const int buf = i & 1;
+            ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (i >> 1) & 1, &tail->abort_flag));
+            if (!ok) { rd_abort(tail, p.status, 35); break; }
+            tmem_fence_after_sync();
+            for (int ch = 0; ch < nch; ++ch) {
+                float gacc[32];
+                tmem_ld<32>(t_p + (uint32_t)(buf * kRdAccCols + ch * 32), gacc);
+                const float4* iv = reinterpret_cast<const float4*>(s_inv + i * kRdTileKeys + col0 + ch * 32);
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float4 c = iv[j >> 2];       // 0 for keys past the end of the cache: those terms vanish
+                    const float t0 = gacc[j] * c.x, t1 = gacc[j + 1] * c.y, t2 = gacc[j + 2] * c.z, t3 = gacc[j + 3] * c.w;
+                    s0 += (t0 >= thr) ? t0 : 0.f;
+                    s1 += (t1 >= thr) ? t1 : 0.f;
+                    s2 += (t2 >= thr) ? t2 : 0.f;
+                    s3 += (t3 >= thr) ? t3 : 0.f;
+                }
+                sum += (s0 + s1) + (s2 + s3);
+            }
+            tmem_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tail->d_empty[buf]));
+        }
+        s_part[wg * 128 + L] = sum;
+        epilogue_bar_sync();
+        if (ok && !*(volatile int*)&tail->abort_flag && ((MT == 2) ? (wg & 1) == 0 : wg == 0) && row < n) {
+            float tot;
+            if (MT == 2) tot = s_part[wg * 128 + L] + s_part[(wg + 1) * 128 + L];
+            else tot = (s_part[L] + s_part[128 + L]) + (s_part[256 + L] + s_part[384 + L]);
+            p.cbar[(size_t)unit * p.C + row] = (row < n - p.recent) ? tot * inv_r : 0.f;   // recent tokens: column zeroed
+        }
+    }
+
+    __syncthreads();
+    if (*(volatile int*)&tail->abort_flag && tid == 0) {
+        mbar_wait_bounded(smem_u32(&tail->a_full), 0);
+        const int issued = *(volatile int*)&tail->issued;
+        for (int i = max(0, issued - stages); i < issued; ++i)
+            mbar_wait_bounded(smem_u32(&tail->k_full[i % stages]), (i / stages) & 1);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tmem_fence_after_sync();
+        tmem_dealloc(tmem_base, kRdTmemCols);
+    }
+}
+
+static size_t redundancy_smem_bytes(int C, int stages) {
+    return 1024 + (size_t)kRdABytes + (size_t)stages * kRdStageBytes +
+           sizeof(float) * (((C + 127) & ~127) + kRdGroups * 128) + sizeof(RedundancyTail);
+}
+
+cudaError_t redundancy_kernel_setup() {
+    return cudaFuncSetAttribute(gkv_redundancy_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+}
+
+cudaError_t launch_keynorm(const RedundancyLaunch& p, cudaStream_t s) {
+    const int units = p.n_layers * p.batch * p.h_kv;
+    gkv_keynorm_kernel<<<units * ((p.C + 127) / 128), 256, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_redundancy(const RedundancyLaunch& p, const CUtensorMap& tm_k, cudaStream_t s) {
+    const int units = p.n_layers * p.batch * p.h_kv;
+    const int blocks_per_unit = (p.C + kRdBlockRows - 1) / kRdBlockRows;
+    int stages = 2;
+    while (stages < kRdMaxStages && redundancy_smem_bytes(p.C, stages + 1) <= 227 * 1024) ++stages;
+    gkv_redundancy_tc_kernel<<<units * blocks_per_unit, kRdThreads, redundancy_smem_bytes(p.C, stages), s>>>(
+        p, tm_k, blocks_per_unit, stages);
+    return cudaGetLastError();
+}
+
+}  // namespace gkv
