@@ -190,6 +190,16 @@ gkv_status gkv_decode_attn_static(const void* q, const void* k_new, const void* 
                                   void* v_cache, void* out, int32_t batch, int32_t n_q_heads,
                                   int32_t n_kv_heads, int32_t capacity, int32_t len, void* stream);
 
+/* Eviction log (what the paper's sparse-training recipes need to rebuild the attention mask of a compressed
+ * rollout: which tokens left the cache at which compression step). After this call every gkv_evict /
+ * SELECT stage also writes, for each (layer, sequence, KV head) it processes, the tokens it evicted into
+ * log_device [n_layers][batch][n_kv_heads][buffer] int32 (device pointer, caller-owned, kept alive while
+ * set): original token positions when track_positions is on, else pre-compaction row indices; ascending;
+ * unused entries (a step evicts len - b <= buffer tokens) are -1; a step that evicts nothing writes all -1.
+ * Only the layers of the call are written. NULL switches the log off.
+ * Errors: INVALID_ARG (NULL context, misaligned pointer). */
+gkv_status gkv_set_eviction_log(gkv_ctx* ctx, int32_t* log_device);
+
 /* With use_redundancy: copies the redundancy levels cbar (summed thresholded cosine similarity of every
  * cached key, 0 for the protected recent tokens) that the last gkv_evict / REDUNDANCY stage computed for
  * `layer` into out_device [batch][n_kv_heads][C] fp32 (device pointer), asynchronously on `stream`.

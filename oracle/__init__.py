@@ -192,6 +192,16 @@ def evict_step_redundancy(Q_win, S_in, K, V, pos, F_prev, *, l, n_h, b, w, alpha
     return out
 
 
+def evicted(kept, pos, l):
+    """Tokens evicted by a step: complement of kept [h_kv][b] in 0..l-1, ascending, as original positions
+    (pos [h_kv][C] int32) or row indices (pos None). Returns [h_kv][l - b] int32."""
+    h_kv, b = kept.shape
+    C = pos.shape[1] if pos is not None else l
+    out = np.empty((h_kv, l - b), np.int32)
+    lib().gkvo_evicted(_p(np.ascontiguousarray(kept), np.int32), _p(pos, np.int32), h_kv, C, l, b, _p(out, np.int32))
+    return out
+
+
 def evict_batch(Q_win, S_in, K, V, F_prev, *, h_q, l, n_h, b, w, alpha, mode, want_kv=False):
     """Eviction step for n_seq independent sequences (parallel across sequences).
 

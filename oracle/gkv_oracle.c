@@ -416,3 +416,19 @@ int gkvo_evict_step_redundancy(const uint16_t* Q_win, const float* S_in, const u
     free(F); free(cbar); free(R); free(Rn); free(Fsel); free(kept);
     return b;
 }
+
+/* Eviction log of one step: the tokens that are NOT in kept, in ascending cache position, reported by their
+ * original position pos[j][t] (or by t itself when pos is NULL). kept [h_kv][b] as gkvo_select returns it,
+ * out [h_kv][l - b]. This is the information the paper's sparse-training recipes record per compression
+ * step to rebuild the attention mask of a compressed rollout. */
+void gkvo_evicted(const int32_t* kept, const int32_t* pos, int h_kv, int C, int l, int b, int32_t* out) {
+    unsigned char* in_kept = (unsigned char*)malloc((size_t)l);
+    for (int j = 0; j < h_kv; ++j) {
+        memset(in_kept, 0, (size_t)l);
+        for (int r = 0; r < b; ++r) in_kept[kept[(size_t)j * b + r]] = 1;
+        int e = 0;
+        for (int t = 0; t < l; ++t)
+            if (!in_kept[t]) out[(size_t)j * (l - b) + e++] = pos ? pos[(size_t)j * C + t] : t;
+    }
+    free(in_kept);
+}

@@ -93,6 +93,7 @@ def lib() -> ctypes.CDLL:
         L.gkv_evict_host.argtypes = [vp, i32, vp, vp, vp]
         L.gkv_get_state.argtypes = [vp, i32, P(i32), P(i32), P(i32)]
         L.gkv_get_redundancy.argtypes = [vp, i32, vp, vp]
+        L.gkv_set_eviction_log.argtypes = [vp, vp]
         L.gkv_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.gkv_decode_attn_static.restype = ctypes.c_int
         L.gkv_launch_count.argtypes = [vp]
@@ -104,7 +105,7 @@ def lib() -> ctypes.CDLL:
         L.gkv_destroy.argtypes = [vp]
         L.gkv_destroy.restype = None
         for name in ("gkv_query_sizes", "gkv_init", "gkv_set_state", "gkv_decode_attn", "gkv_evict", "gkv_evict_stage",
-                     "gkv_decode_attn_host", "gkv_evict_host", "gkv_get_state", "gkv_get_redundancy", "gkv_poll_device_status",
+                     "gkv_decode_attn_host", "gkv_evict_host", "gkv_get_state", "gkv_get_redundancy", "gkv_set_eviction_log", "gkv_poll_device_status",
                      "gkv_memory_model"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
@@ -206,6 +207,10 @@ def gkv_get_state(ctx, layer):
     return a.value, b.value, c.value
 
 
+def gkv_set_eviction_log(ctx, log):
+    _check(lib().gkv_set_eviction_log(ctx, _ptr(log)), "gkv_set_eviction_log")
+
+
 def gkv_get_redundancy(ctx, layer, out):
     _check(lib().gkv_get_redundancy(ctx, layer, _ptr(out), _stream()), "gkv_get_redundancy")
 
@@ -275,6 +280,15 @@ class GKVCache:
 
     def state(self, layer=0):
         return gkv_get_state(self.ctx, layer)
+
+    def enable_eviction_log(self):
+        """Allocates [n_layers][batch][h_kv][buffer] int32 and has every eviction write its evicted tokens there."""
+        import torch
+        cfg = self.cfg
+        self.evict_log = torch.full((cfg.n_layers, cfg.batch, cfg.n_kv_heads, cfg.buffer), -1, dtype=torch.int32,
+                                    device=self.device)
+        gkv_set_eviction_log(self.ctx, self.evict_log)
+        return self.evict_log
 
     def redundancy(self, layer=0):
         """cbar [batch][h_kv][C] of the last eviction of `layer` (redundancy term on)."""

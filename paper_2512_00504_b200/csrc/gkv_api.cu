@@ -151,6 +151,7 @@ EvictLaunch make_evict(gkv_ctx* ctx, int l0, int nl, int32_t* kept_out) {
     p.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
     p.layer0 = l0; p.n_layers = nl; p.L_total = c.n_layers; p.batch = c.batch; p.h_kv = c.n_kv_heads;
     p.C = ctx->C; p.b = c.budget; p.w = c.window; p.alpha = c.alpha; p.mode = c.mode;
+    p.evict_log = ctx->evict_log;
     p.cbar = c.use_redundancy ? ws_ptr<float>(ctx, ctx->ws.cbar) : nullptr;
     p.fsel_ws = ws_ptr<float>(ctx, ctx->ws.fsel);
     p.lambda = c.redundancy_lambda;
@@ -231,10 +232,16 @@ void after_evict(gkv_ctx* ctx, int l0, int nl, bool noop) {
     }
 }
 
+// A compression call that evicts nothing: the window sums restart and the eviction log (if any) reads "nothing".
 gkv_status reset_sacc(gkv_ctx* ctx, int l0, int nl, cudaStream_t s) {
     const size_t per_layer = (size_t)ctx->units_per_layer * ctx->C * sizeof(float);
     if (cudaMemsetAsync(static_cast<uint8_t*>(ctx->buf.sacc) + l0 * per_layer, 0, nl * per_layer, s) != cudaSuccess)
         return GKV_ERR_CUDA;
+    if (ctx->evict_log) {
+        const size_t log_layer = (size_t)ctx->units_per_layer * ctx->cfg.buffer * sizeof(int32_t);
+        if (cudaMemsetAsync(reinterpret_cast<uint8_t*>(ctx->evict_log) + l0 * log_layer, 0xFF, nl * log_layer, s) != cudaSuccess)
+            return GKV_ERR_CUDA;
+    }
     return GKV_OK;
 }
 
@@ -272,6 +279,7 @@ gkv_status gkv_init(gkv_ctx** out, const gkv_config* cfg, const gkv_buffers* b, 
     ctx->g = cfg->n_q_heads / cfg->n_kv_heads;
     ctx->units_per_layer = cfg->batch * cfg->n_kv_heads;
     ctx->launches = 0;
+    ctx->evict_log = nullptr;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     bool ok = cudaGetDevice(&ctx->device) == cudaSuccess &&
               cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) == cudaSuccess;
@@ -514,6 +522,13 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
     if (kept_idx_out_host && will_evict &&
         cudaMemcpyAsync(kept_idx_out_host, dkept, kb, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return GKV_ERR_CUDA;
+    return GKV_OK;
+}
+
+gkv_status gkv_set_eviction_log(gkv_ctx* ctx, int32_t* log_device) {
+    if (!ctx) return GKV_ERR_INVALID_ARG;
+    if (log_device && (reinterpret_cast<uintptr_t>(log_device) & 3) != 0) return GKV_ERR_INVALID_ARG;
+    ctx->evict_log = log_device;
     return GKV_OK;
 }
 

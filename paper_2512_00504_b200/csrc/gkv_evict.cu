@@ -98,7 +98,9 @@ __device__ __forceinline__ uint32_t ordered_bits(uint32_t x) {
 
 // Top-n_keep of s_f[0..n_c) with ties toward the lower index; kept rows ascending into s_kept,
 // followed by the w window rows n_c .. n_c+w-1. Returns (CTA-uniform) the first row that moves.
-__device__ int select_phase(const float* s_f, int* s_kept, int n_c, int n_keep, int w, EvictShared* sh, int tid) {
+// s_evict (may be NULL) receives the n_c - n_keep evicted rows in ascending order.
+__device__ int select_phase(const float* s_f, int* s_kept, int* s_evict, int n_c, int n_keep, int w, EvictShared* sh,
+                            int tid) {
     const uint32_t* bits = reinterpret_cast<const uint32_t*>(s_f);
     uint32_t prefix = 0;
     int k = n_keep;
@@ -141,15 +143,21 @@ __device__ int select_phase(const float* s_f, int* s_kept, int n_c, int n_keep, 
     int first_drop = n_c;
     for (int t = t0; t < t1; ++t) {
         const uint32_t x = ordered_bits(bits[t]);
+        const int kept_before = gt_before + min(eq_before, k);   // kept rows below t
+        bool dropped = false;
         if (x > T) {
-            s_kept[gt_before + min(eq_before, k)] = t;
+            s_kept[kept_before] = t;
             ++gt_before;
         } else if (x == T) {
-            if (eq_before < k) s_kept[gt_before + eq_before] = t;
-            else first_drop = min(first_drop, t);
+            if (eq_before < k) s_kept[kept_before] = t;
+            else dropped = true;
             ++eq_before;
         } else {
+            dropped = true;
+        }
+        if (dropped) {
             first_drop = min(first_drop, t);
+            if (s_evict) s_evict[t - kept_before] = t;
         }
     }
     if (first_drop < n_c) atomicMin(&sh->first_evicted, first_drop);
@@ -262,7 +270,7 @@ __device__ __forceinline__ UnitIndex unit_of(const EvictLaunch& p, int unit_loca
 
 // Record the per-row state after selection: compact F and pos, clear the window sums, export kept.
 __device__ void write_score_state(const EvictLaunch& p, const UnitIndex& u, const float* s_f, const int* s_kept,
-                                  int* s_pos, int n, int tid) {
+                                  int* s_pos, const int* s_evict, int n, int tid) {
     const int n_keep = p.b - p.w;
     float* f = p.f + (size_t)u.unit * p.C;
     for (int r = tid; r < p.C; r += kEvictThreads) f[r] = (r < n_keep) ? s_f[s_kept[r]] : 0.f;
@@ -271,6 +279,12 @@ __device__ void write_score_state(const EvictLaunch& p, const UnitIndex& u, cons
         for (int t = tid; t < n; t += kEvictThreads) s_pos[t] = pos[t];
         __syncthreads();
         for (int r = tid; r < p.b; r += kEvictThreads) pos[r] = s_pos[s_kept[r]];
+    }
+    if (p.evict_log) {   // what left the cache: original positions when they are tracked, else pre-compaction rows
+        int32_t* log = p.evict_log + (size_t)u.unit * (p.C - p.b);
+        const int n_ev = n - p.b;
+        for (int e = tid; e < p.C - p.b; e += kEvictThreads)
+            log[e] = (e < n_ev) ? (p.pos ? s_pos[s_evict[e]] : s_evict[e]) : -1;
     }
     float* sacc = p.sacc + (size_t)u.unit * p.C;
     for (int t = tid; t < p.C; t += kEvictThreads) sacc[t] = 0.f;
@@ -295,16 +309,17 @@ __device__ void publish_state(const EvictLaunch& p, const UnitIndex& u, int ctas
 
 // s_sel (the scores the selection runs on) is s_f itself unless the redundancy term is on.
 __device__ __forceinline__ void carve(uint8_t* smem, const EvictLaunch& p, float** s_f, int** s_kept, int** s_pos,
-                                      EvictShared** sh, float** s_sel) {
+                                      EvictShared** sh, float** s_sel, int** s_evict) {
     *sh = reinterpret_cast<EvictShared*>(smem);
     *s_f = reinterpret_cast<float*>(smem + sizeof(EvictShared));
     *s_kept = reinterpret_cast<int*>(*s_f + p.C);
     *s_pos = *s_kept + p.b;
     *s_sel = p.cbar ? reinterpret_cast<float*>(*s_pos + (p.pos ? p.C : 0)) : *s_f;
+    *s_evict = p.evict_log ? *s_pos + (p.pos ? p.C : 0) + (p.cbar ? p.C : 0) : nullptr;
 }
 static size_t evict_state_bytes(const EvictLaunch& p) {
     return sizeof(EvictShared) + sizeof(float) * p.C + sizeof(int) * p.b + (p.pos ? sizeof(int) * p.C : 0) +
-           (p.cbar ? sizeof(float) * p.C : 0);
+           (p.cbar ? sizeof(float) * p.C : 0) + (p.evict_log ? sizeof(int) * (p.C - p.b) : 0);
 }
 static size_t evict_smem_bytes(const EvictLaunch& p) { return evict_state_bytes(p); }
 // the fused kernel adds the copy ring, 128-byte aligned behind the score state
@@ -314,8 +329,8 @@ static size_t evict_ring_offset(const EvictLaunch& p) { return (evict_state_byte
 // Whole step in one launch: merge -> select -> score-state update -> K/V compaction.
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const EvictLaunch p, int ring_offset) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel);
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel; int* s_evict;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel, &s_evict);
     const int tid = threadIdx.x;
     const UnitIndex u = unit_of(p, blockIdx.x);
     const int n = p.len[u.lseq_global];
@@ -323,13 +338,15 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const Ev
     if (n <= p.b) {  // nothing to evict: only the window sums restart
         float* sacc = p.sacc + (size_t)u.unit * p.C;
         for (int t = tid; t < p.C; t += kEvictThreads) sacc[t] = 0.f;
+        if (p.evict_log)
+            for (int e = tid; e < p.C - p.b; e += kEvictThreads) p.evict_log[(size_t)u.unit * (p.C - p.b) + e] = -1;
         return;
     }
     const int n_c = n - p.w;
     merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
     if (p.cbar) combine_phase(p.cbar + (size_t)u.unit * p.C, s_f, s_sel, n, n_c, p.lambda, sh, tid);
-    const int r_first = select_phase(s_sel, s_kept, n_c, p.b - p.w, p.w, sh, tid);
-    write_score_state(p, u, s_f, s_kept, s_pos, n, tid);
+    const int r_first = select_phase(s_sel, s_kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
+    write_score_state(p, u, s_f, s_kept, s_pos, s_evict, n, tid);
     compact_phase_async(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
                         p.b, r_first, evict_smem + ring_offset, tid);
     publish_state(p, u, p.h_kv, sh, tid);
@@ -339,8 +356,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const Ev
 // The same step as separate launches (timed one by one); they hand over through the workspace.
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const EvictLaunch p) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel);
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel; int* s_evict;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel, &s_evict);
     const int tid = threadIdx.x;
     const UnitIndex u = unit_of(p, blockIdx.x);
     const int n = p.len[u.lseq_global];
@@ -359,8 +376,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const Ev
 
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const EvictLaunch p) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel);
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel; int* s_evict;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel, &s_evict);
     const int tid = threadIdx.x;
     const UnitIndex u = unit_of(p, blockIdx.x);
     const int n = p.len[u.lseq_global];
@@ -377,8 +394,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const E
         for (int t = tid; t < n_c; t += kEvictThreads) s_sel[t] = in2[t];
     }
     __syncthreads();
-    select_phase(s_sel, s_kept, n_c, p.b - p.w, p.w, sh, tid);
-    write_score_state(p, u, s_f, s_kept, s_pos, n, tid);
+    select_phase(s_sel, s_kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
+    write_score_state(p, u, s_f, s_kept, s_pos, s_evict, n, tid);
     int32_t* kw = p.kept_ws + (size_t)u.unit_local * p.b;
     for (int r = tid; r < p.b; r += kEvictThreads) kw[r] = s_kept[r];
 }
@@ -386,8 +403,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const E
 // grid = units x slices: each CTA moves one column slice of every row of its unit.
 __global__ void __launch_bounds__(kEvictThreads) gkv_evict_compact_kernel(const EvictLaunch p, int slices) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel);
+    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel; int* s_evict;
+    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel, &s_evict);
     const int tid = threadIdx.x;
     const int unit_local = blockIdx.x / slices, slice = blockIdx.x - unit_local * slices;
     const UnitIndex u = unit_of(p, unit_local);

@@ -64,6 +64,7 @@ struct EvictLaunch {
     float alpha;
     int mode;
     // redundancy term: selection on lambda * F - (1 - lambda) * exp(cbar - max cbar); cbar == NULL turns it off
+    int32_t* evict_log;  // may be NULL: [all units][C - b] evicted positions of this step, -1 padded
     const float* cbar;   // [all units][C]
     float* fsel_ws;      // staged path scratch
     float lambda;
@@ -99,6 +100,7 @@ struct gkv_ctx {
     CUtensorMap tm_k, tm_v;
     std::vector<int32_t> len, n_hist, since_evict, sacc_valid, stage_next, cbar_valid;
     int64_t launches;
+    int32_t* evict_log;  // caller's device buffer for the eviction log, or NULL
     gkv_sizes sizes;
 };
 

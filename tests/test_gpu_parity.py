@@ -381,3 +381,38 @@ def test_full_size_config4_sampled():
     assert int(cache.len[0].min()) == int(cache.len[0].max()) == b
     del cache, out, kept
     torch.cuda.empty_cache()
+
+
+def test_eviction_log_lists_what_left_the_cache():
+    """The optional eviction log against the oracle's complement of its own kept list, through a short decode
+    loop with shifted original positions, fused and staged, with and without tracked positions."""
+    shape = dict(n_layers=2, batch=2, h_q=8, h_kv=2, b=96, buffer=32, w=8, s=32)
+    for track in (True, False):
+        cfg = gkv.make_config(**shape, fuse_window_scores=False, track_positions=track)
+        cache = gkv.GKVCache(cfg, DEV)
+        log = cache.enable_eviction_log()
+        case = synth.eviction_case(synth.BASE_SEED + 60, batch=2, h_q=8, h_kv=2, b=96, buffer=32, w=8, l=121, device=DEV)
+        for layer in range(2):
+            cache.k[layer].copy_(case.k); cache.v[layer].copy_(case.v); cache.f[layer].copy_(case.f_prev)
+            if track:
+                cache.pos[layer].copy_(case.pos * 3 + 1000 * layer)
+        cache.set_state(-1, 121, 88, 32, False)
+        snaps = [snapshot(cache, layer, [0, 1]) for layer in range(2)]
+        kept = torch.empty((2, 2, 2, 96), dtype=torch.int32, device=DEV)
+        q_win = torch.stack([case.q_win, case.q_win]).contiguous()
+        cache.evict(0, q_win[0], kept[0])                                   # fused, layer 0 only
+        assert (log[1] == -1).all()                                         # layer 1 not touched yet
+        cache.evict_stage(1, gkv.GKV_STAGE_SCORE, q_win[1])
+        cache.evict_stage(1, gkv.GKV_STAGE_MERGE)
+        cache.evict_stage(1, gkv.GKV_STAGE_SELECT, None, kept[1])
+        cache.evict_stage(1, gkv.GKV_STAGE_COMPACT)
+        cache.poll()
+        got = log.cpu().numpy()
+        for layer in range(2):
+            for n in range(2):
+                want = oracle.evicted(kept[layer, n].cpu().numpy(), snaps[layer]["pos"][n] if track else None, 121)
+                assert (got[layer, n, :, :25] == want).all() and (got[layer, n, :, 25:] == -1).all()
+        # a scheduled compression that evicts nothing reports nothing
+        cache.set_state(-1, 90, 0, 32, True)
+        cache.evict(-1)
+        assert (log == -1).all()

@@ -153,3 +153,17 @@ def test_step_drops_the_older_duplicate_and_records_f_not_fsel():
     for j in range(2):
         order = sorted(range(l - w), key=lambda t: (-out["Fsel"][j, t], t))[: b - w]
         assert sorted(order) == out["kept"][j, : b - w].tolist()
+
+
+def test_eviction_log_is_the_complement_of_kept():
+    """Hand case: l = 7, kept rows {0, 2, 3, 6} -> evicted rows 1, 4, 5, reported through pos; plus the
+    complement property on a random step."""
+    kept = np.array([[0, 2, 3, 6]], np.int32)
+    pos = np.array([[10, 11, 12, 13, 14, 15, 16, 99]], np.int32)
+    assert oracle.evicted(kept, pos, 7).tolist() == [[11, 14, 15]]
+    assert oracle.evicted(kept, None, 7).tolist() == [[1, 4, 5]]
+    K, V, S, F_prev, pos = _case(6)
+    out = oracle.evict_step(None, S, K, V, pos, F_prev, l=40, n_h=20, b=24, w=4, alpha=0.8, mode=oracle.MODE_MAX)
+    ev = oracle.evicted(out["kept"], pos, 40)
+    for j in range(2):
+        assert sorted(ev[j].tolist() + out["kept"][j].tolist()) == list(range(40)) and (np.diff(ev[j]) > 0).all()
