@@ -46,6 +46,7 @@ def lib() -> ctypes.CDLL:
         _lib.gkvo_num_threads.restype = ctypes.c_int
         _lib.gkvo_evict_step.restype = ctypes.c_int
         _lib.gkvo_evict_step_redundancy.restype = ctypes.c_int
+        _lib.gkvo_evict_step_full.restype = ctypes.c_int
     return _lib
 
 
@@ -189,6 +190,33 @@ def evict_step_redundancy(Q_win, S_in, K, V, pos, F_prev, *, l, n_h, b, w, alpha
         _p(out["F"], np.float64), _p(out["cbar"], np.float64), _p(out["Rn"], np.float64), _p(out["Fsel"], np.float64),
         _p(out["band"], np.int32), _p(out["kept"], np.int32), _p(out["K"], np.uint16), _p(out["V"], np.uint16),
         _p(out["pos"], np.int32), _p(out["F_state"], np.float64)))
+    return out
+
+
+def maxpool(X, kernel):
+    """Sequence-wise max-pooling of a score [h_kv][n] (odd kernel, window clipped at the ends)."""
+    h_kv, n = X.shape
+    out = np.empty((h_kv, n), np.float64)
+    lib().gkvo_maxpool(_p(np.ascontiguousarray(X, dtype=np.float64), np.float64), h_kv, n, int(kernel), _p(out, np.float64))
+    return out
+
+
+def evict_step_full(Q_win, S_in, K, V, pos, F_prev, *, l, n_h, b, w, alpha, mode, pool_kernel=1, lam=None, tau=0.5,
+                    recent=0, eps=1e-6):
+    """One eviction step with the optional pooling (pool_kernel > 1) and redundancy (lam not None) terms."""
+    h_kv, C, d = K.shape
+    assert (Q_win is None) != (S_in is None) and l > b
+    h_q = Q_win.shape[0] if Q_win is not None else h_kv
+    n_c = l - w
+    out = {"F": np.empty((h_kv, n_c), np.float64), "Fsel": np.empty((h_kv, n_c), np.float64),
+           "kept": np.empty((h_kv, b), np.int32), "K": np.zeros_like(K), "V": np.zeros_like(V),
+           "pos": None if pos is None else np.zeros_like(pos), "F_state": np.zeros((h_kv, C), np.float64)}
+    out["len"] = int(lib().gkvo_evict_step_full(
+        _p(Q_win, np.uint16), _p(S_in, np.float32), _p(K, np.uint16), _p(V, np.uint16), _p(pos, np.int32),
+        _p(F_prev, np.float32), h_q, h_kv, d, C, l, n_h, b, w, ctypes.c_double(alpha), mode, int(pool_kernel),
+        int(lam is not None), ctypes.c_double(1.0 if lam is None else lam), ctypes.c_double(tau), int(recent),
+        ctypes.c_double(eps), _p(out["F"], np.float64), _p(out["Fsel"], np.float64), _p(out["kept"], np.int32),
+        _p(out["K"], np.uint16), _p(out["V"], np.uint16), _p(out["pos"], np.int32), _p(out["F_state"], np.float64)))
     return out
 
 

@@ -432,3 +432,56 @@ void gkvo_evicted(const int32_t* kept, const int32_t* pos, int h_kv, int C, int 
     }
     free(in_kept);
 }
+
+/* Appendix on combining the global score with other methods, SnapKV: a sequence-wise max-pooling of the
+ * score before the selection ("it suffices to replace the local score utilized by SnapKV with the global
+ * score"). out[j][t] = max of X[j][t'] over |t' - t| <= kernel / 2 within 0..n-1 (kernel odd; the window is
+ * clipped at the ends, which equals padding with -inf). The paper does not give the kernel size: parameter. */
+void gkvo_maxpool(const double* X, int h_kv, int n, int kernel, double* out) {
+    const int half = kernel / 2;
+    for (int j = 0; j < h_kv; ++j)
+        for (int t = 0; t < n; ++t) {
+            double m = -INFINITY;
+            for (int u = t - half; u <= t + half; ++u)
+                if (u >= 0 && u < n && X[(size_t)j * n + u] > m) m = X[(size_t)j * n + u];
+            out[(size_t)j * n + t] = m;
+        }
+}
+
+/* The eviction step with every optional term: F as in gkvo_evict_step; P = maxpool(F) when kernel > 1
+ * (else F); Fsel = lambda P - (1 - lambda) Rn when use_redundancy (else P); top-(b-w) on Fsel; F itself is
+ * what is recorded. Outputs may be NULL. */
+int gkvo_evict_step_full(const uint16_t* Q_win, const float* S_in, const uint16_t* K, const uint16_t* V,
+                         const int32_t* pos, const float* F_prev, int h_q, int h_kv, int d, int C, int l, int n_h,
+                         int b, int w, double alpha, int mode, int pool_kernel, int use_redundancy, double lambda,
+                         double tau, int recent, double eps, double* F_out, double* Fsel_out, int32_t* kept_out,
+                         uint16_t* K_out, uint16_t* V_out, int32_t* pos_out, double* F_state) {
+    if (l <= b) return l;
+    const int n_c = l - w;
+    double* F = (double*)malloc(sizeof(double) * (size_t)h_kv * n_c);
+    double* P = (double*)malloc(sizeof(double) * (size_t)h_kv * n_c);
+    double* Fsel = (double*)malloc(sizeof(double) * (size_t)h_kv * n_c);
+    int32_t* kept = (int32_t*)malloc(sizeof(int32_t) * (size_t)h_kv * b);
+    gkvo_evict_step(Q_win, S_in, K, V, pos, F_prev, h_q, h_kv, d, C, l, n_h, b, w, alpha, mode, NULL, NULL, F,
+                    NULL, NULL, NULL, NULL, NULL);
+    if (pool_kernel > 1) gkvo_maxpool(F, h_kv, n_c, pool_kernel, P);
+    else memcpy(P, F, sizeof(double) * (size_t)h_kv * n_c);
+    if (use_redundancy) {
+        double* cbar = (double*)malloc(sizeof(double) * (size_t)h_kv * l);
+        double* R = (double*)malloc(sizeof(double) * (size_t)h_kv * l);
+        double* Rn = (double*)malloc(sizeof(double) * (size_t)h_kv * l);
+        gkvo_redundancy(K, h_kv, C, d, l, tau, recent, eps, cbar, R, Rn, NULL, 0.0);
+        gkvo_combine(P, Rn, h_kv, n_c, l, lambda, Fsel);
+        free(cbar); free(R); free(Rn);
+    } else {
+        memcpy(Fsel, P, sizeof(double) * (size_t)h_kv * n_c);
+    }
+    gkvo_select(Fsel, h_kv, n_c, l, b, w, kept);
+    if (K_out && V_out && F_state)
+        gkvo_compact(K, V, pos, F, kept, h_kv, C, d, n_c, b, w, K_out, V_out, pos_out, F_state);
+    if (F_out) memcpy(F_out, F, sizeof(double) * (size_t)h_kv * n_c);
+    if (Fsel_out) memcpy(Fsel_out, Fsel, sizeof(double) * (size_t)h_kv * n_c);
+    if (kept_out) memcpy(kept_out, kept, sizeof(int32_t) * (size_t)h_kv * b);
+    free(F); free(P); free(Fsel); free(kept);
+    return b;
+}

@@ -167,3 +167,39 @@ def test_eviction_log_is_the_complement_of_kept():
     ev = oracle.evicted(out["kept"], pos, 40)
     for j in range(2):
         assert sorted(ev[j].tolist() + out["kept"][j].tolist()) == list(range(40)) and (np.diff(ev[j]) > 0).all()
+
+
+@pytest.mark.parametrize("kernel", [1, 3, 5, 7, 13])
+def test_maxpool_matches_library_filters(kernel):
+    """scipy's 1-D maximum filter with -inf padding and torch's max_pool1d (stride 1, padding k // 2: the
+    SnapKV operation) give the same result; hand case for kernel 3."""
+    import scipy.ndimage
+    import torch
+    rng = np.random.default_rng(kernel)
+    X = rng.random((3, 37))
+    got = oracle.maxpool(X, kernel)
+    want = scipy.ndimage.maximum_filter1d(X, size=kernel, axis=-1, mode="constant", cval=-np.inf)
+    np.testing.assert_array_equal(got, want)
+    tp = torch.nn.functional.max_pool1d(torch.from_numpy(X)[None], kernel, stride=1, padding=kernel // 2)[0].numpy()
+    np.testing.assert_array_equal(got, tp)
+    if kernel == 3:
+        assert oracle.maxpool(np.array([[1.0, 5.0, 2.0, 0.0, 3.0]]), 3).tolist() == [[5.0, 5.0, 5.0, 3.0, 3.0]]
+
+
+def test_full_step_reduces_and_pools_before_combining():
+    K, V, S, F_prev, pos = _case(7)
+    kw = dict(l=40, n_h=20, b=24, w=4, alpha=0.8, mode=oracle.MODE_MAX)
+    plain = oracle.evict_step(None, S, K, V, pos, F_prev, **kw)
+    full = oracle.evict_step_full(None, S, K, V, pos, F_prev, **kw)                       # both terms off
+    assert (plain["kept"] == full["kept"]).all() and (plain["K"] == full["K"]).all()
+    red = oracle.evict_step_redundancy(None, S, K, V, pos, F_prev, **kw, lam=0.7, tau=0.4, recent=4, eps=EPS)
+    full = oracle.evict_step_full(None, S, K, V, pos, F_prev, **kw, lam=0.7, tau=0.4, recent=4, eps=EPS)
+    assert (red["kept"] == full["kept"]).all()
+    np.testing.assert_array_equal(red["Fsel"], full["Fsel"])
+    pooled = oracle.evict_step_full(None, S, K, V, pos, F_prev, **kw, pool_kernel=5)
+    np.testing.assert_array_equal(pooled["Fsel"], oracle.maxpool(plain["F"], 5))
+    np.testing.assert_array_equal(pooled["F"], plain["F"])                                  # the recorded score is not pooled
+    for j in range(2):
+        np.testing.assert_array_equal(pooled["F_state"][j, :20], plain["F"][j, pooled["kept"][j, :20]])
+    both = oracle.evict_step_full(None, S, K, V, pos, F_prev, **kw, pool_kernel=5, lam=0.7, tau=0.4, recent=4, eps=EPS)
+    np.testing.assert_allclose(both["Fsel"], oracle.combine(oracle.maxpool(plain["F"], 5), red["Rn"], 0.7), rtol=1e-15)
