@@ -90,6 +90,11 @@ typedef struct {
     float redundancy_threshold; /* tau > 0: cosine similarities below it count as 0              */
     int32_t redundancy_recent;  /* this many most recent tokens are never rated redundant, >= 0  */
     float redundancy_eps;       /* epsilon of the key normalisation K / (|K| + eps), >= 0        */
+    /* SnapKV combination of the same appendix: sequence-wise max-pooling (this kernel size, odd; 0 or 1 =
+     * off; window clipped at the ends of the candidate range) of the global score before the selection
+     * (and before the redundancy term, if both are on). The unpooled F is what is recorded. The paper
+     * gives no kernel size and reports that pooling does not help at decode time. */
+    int32_t pool_kernel;
 } gkv_config;
 
 typedef struct { uint64_t k, v, f, sacc, pos, len, workspace, staging; } gkv_sizes; /* bytes      */

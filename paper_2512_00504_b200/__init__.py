@@ -39,7 +39,8 @@ class gkv_config(ctypes.Structure):
                [("alpha", ctypes.c_float), ("mode", ctypes.c_int32), ("fuse_window_scores", ctypes.c_int32),
                 ("track_positions", ctypes.c_int32), ("use_redundancy", ctypes.c_int32),
                 ("redundancy_lambda", ctypes.c_float), ("redundancy_threshold", ctypes.c_float),
-                ("redundancy_recent", ctypes.c_int32), ("redundancy_eps", ctypes.c_float)]
+                ("redundancy_recent", ctypes.c_int32), ("redundancy_eps", ctypes.c_float),
+                ("pool_kernel", ctypes.c_int32)]
 
 
 class gkv_sizes(ctypes.Structure):
@@ -134,13 +135,13 @@ def _stream():
 
 def make_config(*, n_layers, batch, h_q, h_kv, d=128, b, buffer, w, s, alpha=0.8, mode=GKV_MODE_MAX,
                 fuse_window_scores=True, track_positions=False, redundancy_lambda=None, redundancy_threshold=0.5,
-                redundancy_recent=None, redundancy_eps=1e-6, **_ignored) -> gkv_config:
+                redundancy_recent=None, redundancy_eps=1e-6, pool_kernel=0, **_ignored) -> gkv_config:
     """redundancy_lambda=None leaves the redundancy term off; redundancy_recent defaults to the window."""
     use = redundancy_lambda is not None
     return gkv_config(n_layers, batch, h_q, h_kv, d, b, buffer, w, s, alpha, mode,
                       int(fuse_window_scores), int(track_positions), int(use), float(redundancy_lambda if use else 1.0),
                       float(redundancy_threshold), int(w if redundancy_recent is None else redundancy_recent),
-                      float(redundancy_eps))
+                      float(redundancy_eps), int(pool_kernel))
 
 
 # ------------------------------------------------------------------ C-ABI calls, same names

@@ -27,6 +27,7 @@ gkv_status check_config(const gkv_config* c) {
     if (!(c->alpha >= 0.f && c->alpha <= 1.f)) return GKV_ERR_INVALID_ARG;
     if (c->mode < GKV_MODE_MAX || c->mode > GKV_MODE_LOCAL) return GKV_ERR_INVALID_ARG;
     if (c->n_q_heads % c->n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
+    if (c->pool_kernel < 0 || (c->pool_kernel > 1 && (c->pool_kernel & 1) == 0)) return GKV_ERR_INVALID_ARG;
     if (c->use_redundancy) {
         if (!(c->redundancy_lambda >= 0.f && c->redundancy_lambda <= 1.f)) return GKV_ERR_INVALID_ARG;
         if (!(c->redundancy_threshold > 0.f) || !(c->redundancy_eps >= 0.f) || c->redundancy_recent < 0)
@@ -68,7 +69,8 @@ void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     w->kept = off;     off = align_up(off + upl * c->budget * sizeof(int32_t));
     w->fscratch = off; off = align_up(off + upl * C * sizeof(float));
     const uint64_t red = c->use_redundancy ? 1 : 0;   // the redundancy term's scratch exists only when it is on
-    w->fsel = off;     off = align_up(off + red * upl * C * sizeof(float));
+    const uint64_t sel = (c->use_redundancy || c->pool_kernel > 1) ? 1 : 0;
+    w->fsel = off;     off = align_up(off + sel * upl * C * sizeof(float));
     w->inv_norm = off; off = align_up(off + red * L * upl * C * sizeof(float));
     w->cbar = off;     off = align_up(off + red * L * upl * C * sizeof(float));
     w->total = off;
@@ -155,6 +157,7 @@ EvictLaunch make_evict(gkv_ctx* ctx, int l0, int nl, int32_t* kept_out) {
     p.cbar = c.use_redundancy ? ws_ptr<float>(ctx, ctx->ws.cbar) : nullptr;
     p.fsel_ws = ws_ptr<float>(ctx, ctx->ws.fsel);
     p.lambda = c.redundancy_lambda;
+    p.pool_kernel = c.pool_kernel;
     return p;
 }
 

@@ -78,16 +78,38 @@ __device__ void merge_phase(const float* __restrict__ sums, const float* __restr
     __syncthreads();
 }
 
-// Appendix on combining the global score with other methods: R = softmax(cbar), R' = R / max R =
-// exp(cbar - max cbar) (maximum over all n cached tokens), selection score = lambda F - (1 - lambda) R'.
-__device__ void combine_phase(const float* __restrict__ cbar, const float* s_f, float* s_sel, int n, int n_c,
+// Appendix on combining the global score with other methods, SnapKV: sequence-wise max-pooling of the score
+// the selection runs on (odd kernel, window clipped at the ends of the candidate range).
+__device__ void pool_phase(const float* s_f, float* s_sel, int n_c, int kernel, int tid) {
+    const int half = kernel >> 1;
+    for (int t = tid; t < n_c; t += kEvictThreads) {
+        float m = s_f[t];
+        for (int u = max(t - half, 0); u <= min(t + half, n_c - 1); ++u) m = fmaxf(m, s_f[u]);
+        s_sel[t] = m;
+    }
+    __syncthreads();
+}
+
+// Same appendix, redundancy term: R = softmax(cbar), R' = R / max R = exp(cbar - max cbar) (maximum over all
+// n cached tokens), selection score = lambda P - (1 - lambda) R' with P = s_in (F, or pooled F; s_in may be s_sel).
+__device__ void combine_phase(const float* __restrict__ cbar, const float* s_in, float* s_sel, int n, int n_c,
                               float lambda, EvictShared* sh, int tid) {
     float mx = -INFINITY;
     for (int t = tid; t < n; t += kEvictThreads) mx = fmaxf(mx, cbar[t]);
     mx = block_max(mx, sh->warp_max, tid);
     for (int t = tid; t < n_c; t += kEvictThreads)
-        s_sel[t] = lambda * s_f[t] - (1.f - lambda) * fast_exp2((cbar[t] - mx) * 1.4426950408889634f);
+        s_sel[t] = lambda * s_in[t] - (1.f - lambda) * fast_exp2((cbar[t] - mx) * 1.4426950408889634f);
     __syncthreads();
+}
+
+// F in s_f -> the scores the selection runs on in s_sel (s_sel == s_f when no optional term is on):
+// P = maxpool(F) if pooling is on, then lambda P - (1 - lambda) R' if the redundancy term is on.
+__device__ __forceinline__ bool has_selection_terms(const EvictLaunch& p) { return p.cbar != nullptr || p.pool_kernel > 1; }
+__device__ void selection_scores(const EvictLaunch& p, long unit, const float* s_f, float* s_sel, int n, int n_c,
+                                 EvictShared* sh, int tid) {
+    const bool pool = p.pool_kernel > 1;
+    if (pool) pool_phase(s_f, s_sel, n_c, p.pool_kernel, tid);
+    if (p.cbar) combine_phase(p.cbar + (size_t)unit * p.C, pool ? s_sel : s_f, s_sel, n, n_c, p.lambda, sh, tid);
 }
 
 // fp32 bit pattern -> unsigned integer with the same order (negative values included: the combined
@@ -314,12 +336,13 @@ __device__ __forceinline__ void carve(uint8_t* smem, const EvictLaunch& p, float
     *s_f = reinterpret_cast<float*>(smem + sizeof(EvictShared));
     *s_kept = reinterpret_cast<int*>(*s_f + p.C);
     *s_pos = *s_kept + p.b;
-    *s_sel = p.cbar ? reinterpret_cast<float*>(*s_pos + (p.pos ? p.C : 0)) : *s_f;
-    *s_evict = p.evict_log ? *s_pos + (p.pos ? p.C : 0) + (p.cbar ? p.C : 0) : nullptr;
+    const bool terms = p.cbar != nullptr || p.pool_kernel > 1;
+    *s_sel = terms ? reinterpret_cast<float*>(*s_pos + (p.pos ? p.C : 0)) : *s_f;
+    *s_evict = p.evict_log ? *s_pos + (p.pos ? p.C : 0) + (terms ? p.C : 0) : nullptr;
 }
 static size_t evict_state_bytes(const EvictLaunch& p) {
     return sizeof(EvictShared) + sizeof(float) * p.C + sizeof(int) * p.b + (p.pos ? sizeof(int) * p.C : 0) +
-           (p.cbar ? sizeof(float) * p.C : 0) + (p.evict_log ? sizeof(int) * (p.C - p.b) : 0);
+           ((p.cbar || p.pool_kernel > 1) ? sizeof(float) * p.C : 0) + (p.evict_log ? sizeof(int) * (p.C - p.b) : 0);
 }
 static size_t evict_smem_bytes(const EvictLaunch& p) { return evict_state_bytes(p); }
 // the fused kernel adds the copy ring, 128-byte aligned behind the score state
@@ -344,7 +367,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const Ev
     }
     const int n_c = n - p.w;
     merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
-    if (p.cbar) combine_phase(p.cbar + (size_t)u.unit * p.C, s_f, s_sel, n, n_c, p.lambda, sh, tid);
+    selection_scores(p, u.unit, s_f, s_sel, n, n_c, sh, tid);
     const int r_first = select_phase(s_sel, s_kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
     write_score_state(p, u, s_f, s_kept, s_pos, s_evict, n, tid);
     compact_phase_async(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
@@ -367,8 +390,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const Ev
     merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
     float* out = p.f_ws + (size_t)u.unit_local * p.C;
     for (int t = tid; t < n_c; t += kEvictThreads) out[t] = s_f[t];
-    if (p.cbar) {
-        combine_phase(p.cbar + (size_t)u.unit * p.C, s_f, s_sel, n, n_c, p.lambda, sh, tid);
+    if (has_selection_terms(p)) {
+        selection_scores(p, u.unit, s_f, s_sel, n, n_c, sh, tid);
         float* out2 = p.fsel_ws + (size_t)u.unit_local * p.C;
         for (int t = tid; t < n_c; t += kEvictThreads) out2[t] = s_sel[t];
     }
@@ -389,7 +412,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const E
     const int n_c = n - p.w;
     const float* in = p.f_ws + (size_t)u.unit_local * p.C;
     for (int t = tid; t < n_c; t += kEvictThreads) s_f[t] = in[t];
-    if (p.cbar) {
+    if (has_selection_terms(p)) {
         const float* in2 = p.fsel_ws + (size_t)u.unit_local * p.C;
         for (int t = tid; t < n_c; t += kEvictThreads) s_sel[t] = in2[t];
     }

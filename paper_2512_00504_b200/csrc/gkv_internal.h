@@ -68,6 +68,7 @@ struct EvictLaunch {
     const float* cbar;   // [all units][C]
     float* fsel_ws;      // staged path scratch
     float lambda;
+    int pool_kernel;     // > 1: sequence-wise max-pooling of the score before the selection
 };
 
 struct RedundancyLaunch {

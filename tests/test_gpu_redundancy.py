@@ -123,3 +123,51 @@ def test_redundancy_staged_equals_fused_and_lambda_one_is_plain():
     assert (kept_p.cpu().numpy() == kept3).all()
     with pytest.raises(gkv.GKVError):
         plain.redundancy(0)                                   # term off: no levels to read
+
+
+@pytest.mark.parametrize("pool,lam", [(7, None), (3, 0.7), (13, None)])
+def test_pooled_selection_matches_oracle(pool, lam):
+    """Sequence-wise max-pooling of the global score before the selection (SnapKV combination), alone and
+    followed by the redundancy term; fused and staged launches give the same result."""
+    shape = dict(batch=2, h_q=16, h_kv=4, b=200, buffer=56, w=16, s=56)
+    kw = {k: shape[k] for k in ("batch", "h_q", "h_kv", "b", "buffer", "w")}
+    B, H, b, w = 2, 4, 200, 16
+    results = []
+    for staged in (False, True):
+        cfg = gkv.make_config(n_layers=1, **shape, alpha=0.8, fuse_window_scores=False, track_positions=True,
+                              pool_kernel=pool, redundancy_lambda=lam, redundancy_threshold=0.5, redundancy_recent=16)
+        cache = gkv.GKVCache(cfg, DEV)
+        case = synth.eviction_case(synth.BASE_SEED + 70 + pool, **kw, device=DEV)
+        cache.k[0].copy_(case.k); cache.v[0].copy_(case.v); cache.f[0].copy_(case.f_prev); cache.pos[0].copy_(case.pos)
+        cache.set_state(0, case.l, case.n_h, 56, False)
+        snap = snapshot(cache, 0, [0, 1])
+        kept = torch.empty((B, H, b), dtype=torch.int32, device=DEV)
+        if staged:
+            cache.evict_stage(0, gkv.GKV_STAGE_SCORE, case.q_win)
+            if lam is not None:
+                cache.evict_stage(0, gkv.GKV_STAGE_REDUNDANCY)
+            cache.evict_stage(0, gkv.GKV_STAGE_MERGE)
+            cache.evict_stage(0, gkv.GKV_STAGE_SELECT, None, kept)
+            cache.evict_stage(0, gkv.GKV_STAGE_COMPACT)
+        else:
+            cache.evict(0, case.q_win, kept)
+        cache.poll()
+        kept = kept.cpu().numpy()
+        results.append((kept, cache.k[0, :, :, :b].clone(), cache.f[0].clone()))
+        for n in range(B):
+            ref = oracle.evict_step_full(synth.bits(case.q_win[n]), None, snap["K"][n], snap["V"][n], snap["pos"][n],
+                                         snap["F"][n], l=case.l, n_h=case.n_h, b=b, w=w, alpha=0.8, mode=oracle.MODE_MAX,
+                                         pool_kernel=pool, lam=lam, tau=0.5, recent=16, eps=1e-6)
+            for j in range(H):
+                fsel = ref["Fsel"][j]
+                order = np.lexsort((np.arange(case.l - w), -fsel))
+                thr = fsel[order[b - w - 1]]
+                band = SCORE_RTOL * (abs(thr) + (0.0 if lam is None else 1.0 - lam)) + SCORE_ATOL
+                k = kept[n, j]
+                for t in set(order[: b - w].tolist()) ^ set(k[: b - w].tolist()):
+                    assert abs(fsel[t] - thr) <= band, f"seq {n} head {j}: row {t} differs outside the band"
+                assert (synth.bits(cache.k[0])[n, j, :b] == snap["K"][n, j, k]).all()
+                np.testing.assert_allclose(cache.f[0, n, j, : b - w].cpu().numpy(), ref["F"][j, k[: b - w]],
+                                           rtol=SCORE_RTOL, atol=SCORE_ATOL)   # recorded score: unpooled F
+    assert (results[0][0] == results[1][0]).all() and torch.equal(results[0][1], results[1][1])
+    assert torch.equal(results[0][2], results[1][2])
