@@ -95,6 +95,9 @@ typedef struct {
      * (and before the redundancy term, if both are on). The unpooled F is what is recorded. The paper
      * gives no kernel size and reports that pooling does not help at decode time. */
     int32_t pool_kernel;
+    /* Longest prompt gkv_compress_prompt will be given (rows per head of its K / V buffers); 0 = that call is
+     * not used. At most 8192. Sizes part of the workspace. */
+    int32_t max_prompt;
 } gkv_config;
 
 typedef struct { uint64_t k, v, f, sacc, pos, len, workspace, staging; } gkv_sizes; /* bytes      */
@@ -194,6 +197,28 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
 gkv_status gkv_decode_attn_static(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                   void* v_cache, void* out, int32_t batch, int32_t n_q_heads,
                                   int32_t n_kv_heads, int32_t capacity, int32_t len, void* stream);
+
+/* First compression of a freshly prefilled prompt that may be longer than the cache (Section 3 starts from a
+ * prefilled cache; Section 5: the first compression uses the normalised local score alone, no history).
+ * k_prompt, v_prompt: device, [batch][n_kv_heads][max_prompt][128] bf16 (16-byte aligned), sequence i holding
+ * prompt_len_host[i] rows (HOST array of batch int32, 1..max_prompt; lengths may differ per sequence).
+ * q_window: device, [batch][n_q_heads][w][128], the queries of each prompt's last w tokens, oldest first
+ * (may be NULL when no prompt is longer than b). Per sequence and KV head: a prompt of at most b tokens is
+ * copied whole into cache rows 0..len-1 (n_hist = 0); a longer one keeps the top-(b-w) of its first
+ * len - w tokens by the max-normalised window score (Eq. 1-2, after the optional pooling; the redundancy
+ * term is not applied to prompts) plus the last w tokens, in ascending position, in rows 0..b-1, with F of
+ * the kept rows recorded and pos = position in the prompt (with track_positions). sacc of the layer is
+ * cleared, since_evict = 0. kept_idx_out (optional, device [batch][n_kv_heads][b]) receives the kept
+ * prompt positions, -1 padded. One layer per call (prefill proceeds layer by layer).
+ * Afterwards the sequences of the layer may have different cache lengths: the device keeps one length per
+ * sequence, every later call handles each sequence at its own length (a scheduled compression evicts
+ * nothing from a sequence that holds at most b tokens), and the host counters of gkv_get_state follow the
+ * longest sequence.
+ * Errors: STATE (max_prompt == 0), INVALID_ARG (NULL / misaligned pointer, layer = -1, a length outside
+ * 1..max_prompt, q_window == NULL with a prompt longer than b), CUDA. */
+gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt, const void* v_prompt,
+                               const void* q_window, const int32_t* prompt_len_host, int32_t* kept_idx_out,
+                               void* stream);
 
 /* Eviction log (what the paper's sparse-training recipes need to rebuild the attention mask of a compressed
  * rollout: which tokens left the cache at which compression step). After this call every gkv_evict /

@@ -40,7 +40,7 @@ class gkv_config(ctypes.Structure):
                 ("track_positions", ctypes.c_int32), ("use_redundancy", ctypes.c_int32),
                 ("redundancy_lambda", ctypes.c_float), ("redundancy_threshold", ctypes.c_float),
                 ("redundancy_recent", ctypes.c_int32), ("redundancy_eps", ctypes.c_float),
-                ("pool_kernel", ctypes.c_int32)]
+                ("pool_kernel", ctypes.c_int32), ("max_prompt", ctypes.c_int32)]
 
 
 class gkv_sizes(ctypes.Structure):
@@ -95,6 +95,7 @@ def lib() -> ctypes.CDLL:
         L.gkv_get_state.argtypes = [vp, i32, P(i32), P(i32), P(i32)]
         L.gkv_get_redundancy.argtypes = [vp, i32, vp, vp]
         L.gkv_set_eviction_log.argtypes = [vp, vp]
+        L.gkv_compress_prompt.argtypes = [vp, i32, vp, vp, vp, P(i32), vp, vp]
         L.gkv_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.gkv_decode_attn_static.restype = ctypes.c_int
         L.gkv_launch_count.argtypes = [vp]
@@ -106,7 +107,7 @@ def lib() -> ctypes.CDLL:
         L.gkv_destroy.argtypes = [vp]
         L.gkv_destroy.restype = None
         for name in ("gkv_query_sizes", "gkv_init", "gkv_set_state", "gkv_decode_attn", "gkv_evict", "gkv_evict_stage",
-                     "gkv_decode_attn_host", "gkv_evict_host", "gkv_get_state", "gkv_get_redundancy", "gkv_set_eviction_log", "gkv_poll_device_status",
+                     "gkv_decode_attn_host", "gkv_evict_host", "gkv_get_state", "gkv_get_redundancy", "gkv_set_eviction_log", "gkv_compress_prompt", "gkv_poll_device_status",
                      "gkv_memory_model"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
@@ -135,13 +136,13 @@ def _stream():
 
 def make_config(*, n_layers, batch, h_q, h_kv, d=128, b, buffer, w, s, alpha=0.8, mode=GKV_MODE_MAX,
                 fuse_window_scores=True, track_positions=False, redundancy_lambda=None, redundancy_threshold=0.5,
-                redundancy_recent=None, redundancy_eps=1e-6, pool_kernel=0, **_ignored) -> gkv_config:
+                redundancy_recent=None, redundancy_eps=1e-6, pool_kernel=0, max_prompt=0, **_ignored) -> gkv_config:
     """redundancy_lambda=None leaves the redundancy term off; redundancy_recent defaults to the window."""
     use = redundancy_lambda is not None
     return gkv_config(n_layers, batch, h_q, h_kv, d, b, buffer, w, s, alpha, mode,
                       int(fuse_window_scores), int(track_positions), int(use), float(redundancy_lambda if use else 1.0),
                       float(redundancy_threshold), int(w if redundancy_recent is None else redundancy_recent),
-                      float(redundancy_eps), int(pool_kernel))
+                      float(redundancy_eps), int(pool_kernel), int(max_prompt))
 
 
 # ------------------------------------------------------------------ C-ABI calls, same names
@@ -206,6 +207,13 @@ def gkv_get_state(ctx, layer):
     a, b, c = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
     _check(lib().gkv_get_state(ctx, layer, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)), "gkv_get_state")
     return a.value, b.value, c.value
+
+
+def gkv_compress_prompt(ctx, layer, k_prompt, v_prompt, q_window, prompt_len, kept_idx_out=None):
+    """prompt_len: sequence of batch ints (host)."""
+    lens = (ctypes.c_int32 * len(prompt_len))(*[int(x) for x in prompt_len])
+    _check(lib().gkv_compress_prompt(ctx, layer, _ptr(k_prompt), _ptr(v_prompt), _ptr(q_window), lens,
+                                     _ptr(kept_idx_out), _stream()), "gkv_compress_prompt")
 
 
 def gkv_set_eviction_log(ctx, log):
@@ -281,6 +289,9 @@ class GKVCache:
 
     def state(self, layer=0):
         return gkv_get_state(self.ctx, layer)
+
+    def compress_prompt(self, layer, k_prompt, v_prompt, q_window, prompt_len, kept_idx_out=None):
+        gkv_compress_prompt(self.ctx, layer, k_prompt, v_prompt, q_window, prompt_len, kept_idx_out)
 
     def enable_eviction_log(self):
         """Allocates [n_layers][batch][h_kv][buffer] int32 and has every eviction write its evicted tokens there."""

@@ -14,6 +14,7 @@ using namespace gkv;
 namespace {
 
 constexpr int kMaxCapacity = 4096;
+constexpr int kMaxPrompt = 8192;   // longest prompt gkv_compress_prompt takes (its scores stay in shared memory)
 constexpr uint64_t kAlign = 256;
 
 uint64_t align_up(uint64_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -27,6 +28,8 @@ gkv_status check_config(const gkv_config* c) {
     if (!(c->alpha >= 0.f && c->alpha <= 1.f)) return GKV_ERR_INVALID_ARG;
     if (c->mode < GKV_MODE_MAX || c->mode > GKV_MODE_LOCAL) return GKV_ERR_INVALID_ARG;
     if (c->n_q_heads % c->n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
+    if (c->max_prompt < 0) return GKV_ERR_INVALID_ARG;
+    if (c->max_prompt > kMaxPrompt) return GKV_ERR_UNSUPPORTED;
     if (c->pool_kernel < 0 || (c->pool_kernel > 1 && (c->pool_kernel & 1) == 0)) return GKV_ERR_INVALID_ARG;
     if (c->use_redundancy) {
         if (!(c->redundancy_lambda >= 0.f && c->redundancy_lambda <= 1.f)) return GKV_ERR_INVALID_ARG;
@@ -69,6 +72,8 @@ void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     w->kept = off;     off = align_up(off + upl * c->budget * sizeof(int32_t));
     w->fscratch = off; off = align_up(off + upl * C * sizeof(float));
     const uint64_t red = c->use_redundancy ? 1 : 0;   // the redundancy term's scratch exists only when it is on
+    w->prompt_sums = off; off = align_up(off + upl * (uint64_t)c->max_prompt * sizeof(float));
+    w->prompt_len = off;  off = align_up(off + (c->max_prompt > 0 ? B : 0) * sizeof(int32_t));
     const uint64_t sel = (c->use_redundancy || c->pool_kernel > 1) ? 1 : 0;
     w->fsel = off;     off = align_up(off + sel * upl * C * sizeof(float));
     w->inv_norm = off; off = align_up(off + red * L * upl * C * sizeof(float));
@@ -181,6 +186,22 @@ gkv_status launch_redundancy_for(gkv_ctx* ctx, int l0, int nl, cudaStream_t s) {
     return GKV_OK;
 }
 
+// tcgen05 kernel for windows that split into 16-, 32- or 64-row slices; the mma.sync kernel covers the rest.
+gkv_status dispatch_score(gkv_ctx* ctx, const ScoreLaunch& sp, const CUtensorMap& tm_k, cudaStream_t s) {
+    const gkv_config& c = ctx->cfg;
+    const int wk = score_tc_rows_per_cta(ctx->g, c.window);
+    if (wk > 0 && (reinterpret_cast<uintptr_t>(sp.q_win) & 15) == 0) {
+        CUtensorMap tm_q;
+        const uint64_t q_rows = (uint64_t)sp.n_layers * c.batch * c.n_q_heads * c.window;
+        if (encode_map(&tm_q, const_cast<__nv_bfloat16*>(sp.q_win), q_rows, (uint32_t)wk) != GKV_OK) return GKV_ERR_CUDA;
+        if (launch_score_tc(sp, tm_k, tm_q, wk, s) != cudaSuccess) return GKV_ERR_CUDA;
+    } else if (launch_score(sp, tm_k, s) != cudaSuccess) {
+        return GKV_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    return GKV_OK;
+}
+
 gkv_status launch_score_for(gkv_ctx* ctx, int l0, int nl, const void* q_window, cudaStream_t s) {
     ScoreLaunch sp;
     const gkv_config& c = ctx->cfg;
@@ -191,18 +212,7 @@ gkv_status launch_score_for(gkv_ctx* ctx, int l0, int nl, const void* q_window, 
     sp.layer0 = l0; sp.n_layers = nl; sp.batch = c.batch; sp.h_q = c.n_q_heads; sp.h_kv = c.n_kv_heads;
     sp.g = ctx->g; sp.C = ctx->C; sp.w = c.window;
     sp.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
-    // tcgen05 kernel for windows that split into 16-, 32- or 64-row slices; the mma.sync kernel covers the rest
-    const int wk = score_tc_rows_per_cta(ctx->g, c.window);
-    if (wk > 0 && (reinterpret_cast<uintptr_t>(q_window) & 15) == 0) {
-        CUtensorMap tm_q;
-        const uint64_t q_rows = (uint64_t)nl * c.batch * c.n_q_heads * c.window;
-        if (encode_map(&tm_q, const_cast<void*>(q_window), q_rows, (uint32_t)wk) != GKV_OK) return GKV_ERR_CUDA;
-        if (launch_score_tc(sp, ctx->tm_k, tm_q, wk, s) != cudaSuccess) return GKV_ERR_CUDA;
-    } else if (launch_score(sp, ctx->tm_k, s) != cudaSuccess) {
-        return GKV_ERR_CUDA;
-    }
-    ctx->launches += 1;
-    return GKV_OK;
+    return dispatch_score(ctx, sp, ctx->tm_k, s);
 }
 
 // Shared validation of an eviction request. Returns GKV_OK with *noop set when len <= b.
@@ -525,6 +535,79 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
     if (kept_idx_out_host && will_evict &&
         cudaMemcpyAsync(kept_idx_out_host, dkept, kb, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return GKV_ERR_CUDA;
+    return GKV_OK;
+}
+
+gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt, const void* v_prompt,
+                               const void* q_window, const int32_t* prompt_len_host, int32_t* kept_idx_out, void* stream) {
+    if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers || !k_prompt || !v_prompt || !prompt_len_host)
+        return GKV_ERR_INVALID_ARG;
+    const gkv_config& c = ctx->cfg;
+    if (c.max_prompt <= 0) return GKV_ERR_STATE;
+    if ((reinterpret_cast<uintptr_t>(k_prompt) & 15) || (reinterpret_cast<uintptr_t>(v_prompt) & 15)) return GKV_ERR_INVALID_ARG;
+    int longest = 0;
+    bool any_long = false;
+    for (int i = 0; i < c.batch; ++i) {
+        const int n = prompt_len_host[i];
+        if (n < 1 || n > c.max_prompt) return GKV_ERR_INVALID_ARG;
+        any_long |= n > c.budget;
+        const int rows = n > c.budget ? c.budget : n;
+        if (rows > longest) longest = rows;
+    }
+    if (any_long && !q_window) return GKV_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t* d_len = ws_ptr<int32_t>(ctx, ctx->ws.prompt_len);
+    // a copy from pageable host memory has staged its source when the call returns
+    if (cudaMemcpyAsync(d_len, prompt_len_host, sizeof(int32_t) * c.batch, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GKV_ERR_CUDA;
+    }
+    float* sums = ws_ptr<float>(ctx, ctx->ws.prompt_sums);
+    if (any_long) {
+        CUtensorMap tm_kp;
+        const uint64_t rows = (uint64_t)c.batch * c.n_kv_heads * c.max_prompt;
+        if (encode_map(&tm_kp, const_cast<void*>(k_prompt), rows) != GKV_OK) return GKV_ERR_CUDA;
+        ScoreLaunch sp;
+        sp.q_win = static_cast<const __nv_bfloat16*>(q_window);
+        sp.sacc = sums;
+        sp.len = d_len;
+        sp.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
+        sp.layer0 = 0; sp.n_layers = 1; sp.batch = c.batch; sp.h_q = c.n_q_heads; sp.h_kv = c.n_kv_heads;
+        sp.g = ctx->g; sp.C = c.max_prompt; sp.w = c.window;
+        sp.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
+        const gkv_status st = dispatch_score(ctx, sp, tm_kp, s);
+        if (st != GKV_OK) {
+            (void)cudaGetLastError();
+            return st;
+        }
+    }
+    PromptLaunch p;
+    p.k_src = static_cast<const __nv_bfloat16*>(k_prompt);
+    p.v_src = static_cast<const __nv_bfloat16*>(v_prompt);
+    p.k_cache = static_cast<__nv_bfloat16*>(ctx->buf.k);
+    p.v_cache = static_cast<__nv_bfloat16*>(ctx->buf.v);
+    p.f = static_cast<float*>(ctx->buf.f);
+    p.sacc = static_cast<float*>(ctx->buf.sacc);
+    p.pos = static_cast<int32_t*>(ctx->buf.pos);
+    p.len = static_cast<int32_t*>(ctx->buf.len);
+    p.sums = sums;
+    p.prompt_len = d_len;
+    p.seq_done = ws_ptr<int32_t>(ctx, ctx->ws.seq_done);
+    p.kept_out = kept_idx_out;
+    p.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
+    p.layer = layer; p.L_total = c.n_layers; p.batch = c.batch; p.h_kv = c.n_kv_heads; p.C = ctx->C;
+    p.P_max = c.max_prompt; p.b = c.budget; p.w = c.window; p.pool_kernel = c.pool_kernel;
+    if (launch_prompt_compress(p, s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GKV_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    ctx->len[layer] = longest;                       // host counters follow the longest sequence of the layer
+    ctx->n_hist[layer] = any_long ? c.budget - c.window : 0;
+    ctx->since_evict[layer] = 0;
+    ctx->sacc_valid[layer] = 0;
+    ctx->stage_next[layer] = 0;
+    ctx->cbar_valid[layer] = 0;
     return GKV_OK;
 }
 

@@ -232,13 +232,14 @@ constexpr int kCopyStages = 5;
 constexpr int kCopyStageBytes = kCopyRows * kRowBytes * 2;   // K rows then V rows
 constexpr int kCopyRingBytes = kCopyStages * kCopyStageBytes;
 
-__device__ void compact_phase_async(__nv_bfloat16* kbase, __nv_bfloat16* vbase, const int* kept, int b, int r_first,
-                                    uint8_t* ring, int tid) {
+// Source and destination may be the same buffers (compaction in place) or different ones (gather of a prompt).
+__device__ void compact_phase_async(const __nv_bfloat16* ksrc, const __nv_bfloat16* vsrc, __nv_bfloat16* kbase,
+                                    __nv_bfloat16* vbase, const int* kept, int b, int r_first, uint8_t* ring, int tid) {
     constexpr int D = kCopyStages - 2;                        // groups of loads in flight
     const int n_groups = (b - r_first + kCopyRows - 1) / kCopyRows;
     const uint32_t ring_addr = smem_u32(ring);
-    const uint4* k4 = reinterpret_cast<const uint4*>(kbase);
-    const uint4* v4 = reinterpret_cast<const uint4*>(vbase);
+    const uint4* k4 = reinterpret_cast<const uint4*>(ksrc);
+    const uint4* v4 = reinterpret_cast<const uint4*>(vsrc);
     for (int j = 0; j < n_groups + D; ++j) {
         // the stage group j loads into was last read by the store issued two iterations ago
         if (tid == 0) bulk_wait_read<1>();
@@ -370,9 +371,70 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const Ev
     selection_scores(p, u.unit, s_f, s_sel, n, n_c, sh, tid);
     const int r_first = select_phase(s_sel, s_kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
     write_score_state(p, u, s_f, s_kept, s_pos, s_evict, n, tid);
-    compact_phase_async(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
-                        p.b, r_first, evict_smem + ring_offset, tid);
+    __nv_bfloat16* kb = p.k_cache + (size_t)u.unit * p.C * kHeadDim;
+    __nv_bfloat16* vb = p.v_cache + (size_t)u.unit * p.C * kHeadDim;
+    compact_phase_async(kb, vb, kb, vb, s_kept, p.b, r_first, evict_smem + ring_offset, tid);
     publish_state(p, u, p.h_kv, sh, tid);
+}
+
+// ---------------------------------------------------------------------------------------------
+// First compression of a prompt that is longer than the cache (Section 3: "compressed after every s
+// tokens" starts from a prefilled cache; Section 5: the first step uses the normalised local score alone).
+// The prompt's K, V live in the caller's prefill buffers [batch][h_kv][P_max][d] with per-sequence lengths;
+// `sums` holds w * S of the prompt's last w tokens over all its keys (scoring kernel). Per unit: prompts of
+// at most b tokens are copied whole (no history starts); longer ones keep the top-(b-w) candidates by the
+// normalised score (after the optional pooling) plus the window, gathered into cache rows 0..b-1 in
+// ascending position, with F_state = the normalised score of the kept rows and pos = prompt position.
+__global__ void __launch_bounds__(kEvictThreads) gkv_prompt_compress_kernel(const PromptLaunch p, int ring_offset) {
+    extern __shared__ __align__(128) uint8_t evict_smem[];
+    EvictShared* sh = reinterpret_cast<EvictShared*>(evict_smem);
+    float* s_f = reinterpret_cast<float*>(evict_smem + sizeof(EvictShared));   // [P_max]
+    float* s_sel = (p.pool_kernel > 1) ? s_f + p.P_max : s_f;                  // [P_max] pooled scores
+    int* s_kept = reinterpret_cast<int*>(s_f + ((p.pool_kernel > 1) ? 2 : 1) * p.P_max);   // [b]
+    const int tid = threadIdx.x;
+    const int unit_local = blockIdx.x;
+    const int seq = unit_local / p.h_kv;
+    const int lseq_global = p.layer * p.batch + seq;
+    const long unit = (long)lseq_global * p.h_kv + (unit_local - seq * p.h_kv);
+    const int n = min(p.prompt_len[seq], p.P_max);
+    const bool compress = n > p.b;
+    const int rows = compress ? p.b : n;                   // rows of the cache after this call
+    const int n_keep = p.b - p.w;
+    if (compress) {
+        const int n_c = n - p.w;
+        merge_phase(p.sums + (size_t)unit_local * p.P_max, nullptr, s_f, n_c, 0, 0.f, GKV_MODE_LOCAL, sh, tid);
+        if (p.pool_kernel > 1) pool_phase(s_f, s_sel, n_c, p.pool_kernel, tid);
+        select_phase(s_sel, s_kept, nullptr, n_c, n_keep, p.w, sh, tid);
+    } else {
+        for (int r = tid; r < n; r += kEvictThreads) s_kept[r] = r;
+        __syncthreads();
+    }
+    float* f = p.f + (size_t)unit * p.C;
+    float* sacc = p.sacc + (size_t)unit * p.C;
+    for (int r = tid; r < p.C; r += kEvictThreads) {
+        f[r] = (compress && r < n_keep) ? s_f[s_kept[r]] : 0.f;
+        sacc[r] = 0.f;
+    }
+    if (p.pos) {
+        int32_t* pos = p.pos + (size_t)unit * p.C;
+        for (int r = tid; r < rows; r += kEvictThreads) pos[r] = s_kept[r];
+    }
+    if (p.kept_out) {
+        int32_t* ko = p.kept_out + (size_t)unit_local * p.b;
+        for (int r = tid; r < p.b; r += kEvictThreads) ko[r] = (r < rows) ? s_kept[r] : -1;
+    }
+    compact_phase_async(p.k_src + (size_t)unit_local * p.P_max * kHeadDim, p.v_src + (size_t)unit_local * p.P_max * kHeadDim,
+                        p.k_cache + (size_t)unit * p.C * kHeadDim, p.v_cache + (size_t)unit * p.C * kHeadDim, s_kept, rows, 0,
+                        evict_smem + ring_offset, tid);
+    __syncthreads();
+    if (tid == 0) {   // the last CTA of the sequence publishes its length and the rows that carry history
+        const int prev = atomicAdd(&p.seq_done[lseq_global], 1);
+        if (prev == p.h_kv - 1) {
+            p.seq_done[lseq_global] = 0;
+            p.len[lseq_global] = rows;
+            p.len[(size_t)p.L_total * p.batch + lseq_global] = compress ? n_keep : 0;
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -462,6 +524,15 @@ cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s) {
     cudaError_t e = ensure_smem((const void*)gkv_evict_fused_kernel, smem);
     if (e != cudaSuccess) return e;
     gkv_evict_fused_kernel<<<p.n_layers * p.batch * p.h_kv, kEvictThreads, smem, s>>>(p, (int)ring);
+    return cudaGetLastError();
+}
+cudaError_t launch_prompt_compress(const PromptLaunch& p, cudaStream_t s) {
+    const size_t state = sizeof(EvictShared) + sizeof(float) * p.P_max * ((p.pool_kernel > 1) ? 2 : 1) + sizeof(int) * p.b;
+    const size_t ring = (state + 127) & ~size_t(127);
+    const size_t smem = ring + kCopyRingBytes;
+    cudaError_t e = ensure_smem((const void*)gkv_prompt_compress_kernel, smem);
+    if (e != cudaSuccess) return e;
+    gkv_prompt_compress_kernel<<<p.batch * p.h_kv, kEvictThreads, smem, s>>>(p, (int)ring);
     return cudaGetLastError();
 }
 cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s) {

@@ -22,6 +22,8 @@ struct WorkspaceLayout {
     uint64_t logits;      // split-K window steps: per unit C x 8 fp32 scaled logits
     uint64_t kept;        // int32[units_per_layer * b]   kept lists of the staged eviction path
     uint64_t fscratch;    // fp32[units_per_layer * C]    merged scores of the staged eviction path
+    uint64_t prompt_sums; // fp32[units_per_layer * max_prompt]  window sums of a prompt being compressed
+    uint64_t prompt_len;  // int32[batch]                        device copy of the prompt lengths
     uint64_t fsel;        // fp32[units_per_layer * C]    selection scores of the staged path (redundancy term on)
     uint64_t inv_norm;    // fp32[L * units_per_layer * C] 1 / (|K row| + eps)            (redundancy term on)
     uint64_t cbar;        // fp32[L * units_per_layer * C] redundancy level of every row  (redundancy term on)
@@ -71,6 +73,23 @@ struct EvictLaunch {
     int pool_kernel;     // > 1: sequence-wise max-pooling of the score before the selection
 };
 
+struct PromptLaunch {
+    const __nv_bfloat16* k_src;  // [batch][h_kv][P_max][d] prefill keys / values
+    const __nv_bfloat16* v_src;
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    float* f;
+    float* sacc;
+    int32_t* pos;                // may be NULL
+    int32_t* len;                // plane 0; plane 1 follows at len + L_total*batch
+    const float* sums;           // [batch*h_kv][P_max] w * S of the prompt's window
+    const int32_t* prompt_len;   // device [batch]
+    int32_t* seq_done;
+    int32_t* kept_out;           // may be NULL: [batch*h_kv][b], -1 padded
+    int32_t* status;
+    int layer, L_total, batch, h_kv, C, P_max, b, w, pool_kernel;
+};
+
 struct RedundancyLaunch {
     const __nv_bfloat16* k_cache;
     const int32_t* len;
@@ -118,6 +137,7 @@ cudaError_t launch_score(const ScoreLaunch& p, const CUtensorMap& tm_k, cudaStre
 cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s);
 int score_tc_rows_per_cta(int g, int w);
 cudaError_t score_tc_kernel_setup();
+cudaError_t launch_prompt_compress(const PromptLaunch& p, cudaStream_t s);
 cudaError_t launch_keynorm(const RedundancyLaunch& p, cudaStream_t s);
 cudaError_t launch_redundancy(const RedundancyLaunch& p, const CUtensorMap& tm_k, cudaStream_t s);
 cudaError_t redundancy_kernel_setup();
