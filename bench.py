@@ -420,6 +420,70 @@ def run_sweep(args) -> dict:
 
 
 # ------------------------------------------------------------------------------------------
+def run_prompt(args) -> dict:
+    """First compression of a prefilled prompt (one layer of the 7B shape: batch 32, 28 q / 4 kv heads, b = 1024,
+    w = 32) for prompt lengths 2048, 4096 and 8192: scoring of the prompt's window over all its keys, selection
+    and gather into the cache. The JSON line carries the longest prompt; `sweep` every length."""
+    import torch
+    import paper_2512_00504_b200 as gkv
+    from paper_2512_00504_b200 import synth
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    gkv.build_library()
+    sh = {k: v for k, v in synth.CONFIGS[2].items() if k != "steps"}
+    sh["n_layers"] = 1
+    B, Hq, H, b, w = sh["batch"], sh["h_q"], sh["h_kv"], sh["b"], sh["w"]
+    peaks_path = ROOT / "MEASURED_PEAKS.json"
+    peak_gbs = float(json.loads(peaks_path.read_text())["hbm_gbs"]) if peaks_path.exists() else 6650.0
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    reps = max(3, args.steps)
+    cells, launches = [], 0
+    sampler = ClockSampler(0)
+    sampler.start()
+    for P in (2048, 4096, 8192):
+        cfg = gkv.make_config(**sh, fuse_window_scores=True, max_prompt=P)
+        cache = gkv.GKVCache(cfg, dev)
+        gen = torch.Generator(device=dev).manual_seed(synth.BASE_SEED + 9)
+        kp = torch.randn((B, H, P, 128), generator=gen, device=dev).to(torch.bfloat16)
+        vp = torch.randn((B, H, P, 128), generator=gen, device=dev).to(torch.bfloat16)
+        qw = torch.randn((B, Hq, w, 128), generator=gen, device=dev).to(torch.bfloat16)
+        kept = torch.empty((B, H, b), dtype=torch.int32, device=dev)
+        ts = []
+        l0 = gkv.gkv_launch_count(cache.ctx)
+        for it in range(reps + 3):
+            e0, e1 = ev(), ev()
+            e0.record(); cache.compress_prompt(0, kp, vp, qw, [P] * B, kept); e1.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                ts.append(e0.elapsed_time(e1))
+        cache.poll()
+        launches += gkv.gkv_launch_count(cache.ctx) - l0
+        ms = sorted(ts)[len(ts) // 2]
+        units = B * H
+        bytes_ = units * (P * 256 + 2 * b * 256 * 2 + 8 * P)     # K once (second pass from L2), gather of b K and V rows, sums
+        cells.append({"prompt_len": P, "ms": ms, "prompt_tokens_per_s": B * P / (ms * 1e-3), "algorithmic_bytes": bytes_,
+                      "GBps": bytes_ / (ms * 1e-3) / 1e9, "score_flop": 2.0 * 2.0 * units * (Hq // H) * w * 128 * P,
+                      "score_TFLOPs": 2.0 * 2.0 * units * (Hq // H) * w * 128 * P / (ms * 1e-3) / 1e12})
+        del cache, kp, vp, qw, kept
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = cells[-1]
+    return {"metric": "prompt tokens/s compressed into the cache (first compression of a prefilled prompt, one layer)",
+            "value": top["prompt_tokens_per_s"], "unit": "tok/s", "n_gpus": 1, "steps": reps, "warmup": 3,
+            "ms_per_step": top["ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"prompt compression: 1 layer, batch {B}, {Hq} q / {H} kv heads, d 128, b={b}, w={w}, "
+                                   f"prompt {top['prompt_len']} tokens per sequence; step = scoring + selection + gather",
+                       "l2": "the prompt's K (268 MB at 8192 tokens) exceeds L2"},
+            "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+            "roofline": {"kernel": "gkv_score_tc_kernel + gkv_prompt_compress_kernel", "bound": "hbm", "achieved": top["GBps"],
+                         "peak": peak_gbs, "unit": "GB/s", "frac": top["GBps"] / peak_gbs, "traffic": None,
+                         "algorithmic_bytes_per_launch": top["algorithmic_bytes"], "avg_launch_ms": top["ms"]},
+            "sweep": cells}
+
+
+# ------------------------------------------------------------------------------------------
 def cpu_baseline(sh: dict, budget_s: float = 20.0, n_units: int = 64) -> dict:
     """The oracle, as it stands, timed on the host cores on a bounded sample of the workload:
     `n_units` (layer, sequence) pairs, a few decode steps plus one eviction; extrapolated to a period."""
@@ -493,7 +557,7 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "prompt"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiler captures only)")
     ap.add_argument("--ring", type=int, default=0, help="distinct per-step inputs kept on the device (0 = one period)")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -508,11 +572,13 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.workload == "cfg3":
+        if args.workload in ("cfg3", "prompt"):
             args.workload = "cfg2"   # the oracle arm times the default workload only
         res = run_reference(args)
     elif args.workload == "cfg3":
         res = run_sweep(args)
+    elif args.workload == "prompt":
+        res = run_prompt(args)
     else:
         res = run_ours(args)
     if res is not None:
