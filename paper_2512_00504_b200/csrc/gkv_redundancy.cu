@@ -84,6 +84,12 @@ __device__ __forceinline__ void rd_abort(RedundancyTail* tail, int32_t* status, 
         status[2] = blockIdx.x;
     }
 }
+// 1.0f where a >= b, else 0.0f (also for NaN).
+__device__ __forceinline__ float ge_mask(float a, float b) {
+    float m;
+    asm("set.ge.f32.f32 %0, %1, %2;" : "=f"(m) : "f"(a), "f"(b));
+    return m;
+}
 __device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kRdEpiThreads) : "memory"); }
 
 __global__ void __launch_bounds__(kRdThreads, 1)
@@ -229,14 +235,30 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
                 tmem_ld<32>(t_p + (uint32_t)(buf * kRdAccCols + ch * 32), gacc);
                 const float4* iv = reinterpret_cast<const float4*>(s_inv + i * kRdTileKeys + col0 + ch * 32);
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                if (i + 1 < T) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                    const float4 c = iv[j >> 2];       // 0 for keys past the end of the cache: those terms vanish
-                    const float t0 = gacc[j] * c.x, t1 = gacc[j + 1] * c.y, t2 = gacc[j + 2] * c.z, t3 = gacc[j + 3] * c.w;
-                    s0 += (t0 >= thr) ? t0 : 0.f;
-                    s1 += (t1 >= thr) ? t1 : 0.f;
-                    s2 += (t2 >= thr) ? t2 : 0.f;
-                    s3 += (t3 >= thr) ? t3 : 0.f;
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 c = iv[j >> 2];
+                        const float t0 = gacc[j] * c.x, t1 = gacc[j + 1] * c.y, t2 = gacc[j + 2] * c.z, t3 = gacc[j + 3] * c.w;
+                        // one compare (1.0 / 0.0) and one fused multiply-add per element: a compare + select pair would
+                        // put two instructions per element on the ALU pipe, which throttles first
+                        s0 = fmaf(t0, ge_mask(t0, thr), s0);
+                        s1 = fmaf(t1, ge_mask(t1, thr), s1);
+                        s2 = fmaf(t2, ge_mask(t2, thr), s2);
+                        s3 = fmaf(t3, ge_mask(t3, thr), s3);
+                    }
+                } else {
+                    // last tile: columns past the end of the cache hold whatever the rows beyond it contain (possibly
+                    // NaN or Inf bit patterns); their inverse norm is 0 and a select drops them whatever the product is
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 c = iv[j >> 2];
+                        const float t0 = gacc[j] * c.x, t1 = gacc[j + 1] * c.y, t2 = gacc[j + 2] * c.z, t3 = gacc[j + 3] * c.w;
+                        s0 += (c.x != 0.f && t0 >= thr) ? t0 : 0.f;
+                        s1 += (c.y != 0.f && t1 >= thr) ? t1 : 0.f;
+                        s2 += (c.z != 0.f && t2 >= thr) ? t2 : 0.f;
+                        s3 += (c.w != 0.f && t3 >= thr) ? t3 : 0.f;
+                    }
                 }
                 sum += (s0 + s1) + (s2 + s3);
             }

@@ -35,6 +35,7 @@ def run(shape, seed, lam, tau, recent, l=None, n_h=None, staged=False, dup=True)
         noise = torch.randn((B, H, 24, 128), generator=gen, device=DEV) * torch.linspace(0.0, 1.2, 24, device=DEV)[:, None]
         case.k[:, :, dst] = (case.k[:, :, src].float() + noise).to(torch.bfloat16)
     cache.k[0].copy_(case.k); cache.v[0].copy_(case.v); cache.f[0].copy_(case.f_prev); cache.pos[0].copy_(case.pos)
+    cache.k[0, :, :, case.l:] = float("nan")     # rows beyond the cache length may hold anything: they must not leak in
     cache.set_state(0, case.l, case.n_h, cfg.interval, False)
     seqs = list(range(B))
     snap = snapshot(cache, 0, seqs)
