@@ -416,3 +416,71 @@ def test_eviction_log_lists_what_left_the_cache():
         cache.set_state(-1, 90, 0, 32, True)
         cache.evict(-1)
         assert (log == -1).all()
+
+
+def test_config1_full_decode_eviction_loop():
+    """Configuration 1 at full length: 28 q / 4 kv heads, b = 512, buffer = 128, w = 16, 4096 decode steps from an
+    empty cache with the drifting query direction and the intermittently attended planted keys. Every scheduled
+    compression is compared step-wise with the oracle (28 of the 32 evict; the first 4 find at most b tokens);
+    decode outputs are spot-checked; the planted keys' survival under the global score is reported by assertion
+    against the local score on the same stream."""
+    shape = {k: v for k, v in synth.CONFIGS[1].items() if k != "steps"}
+    steps, b, w, s, H = synth.CONFIGS[1]["steps"], 512, 16, 128, 4
+    survivors = {}
+    for mode in (gkv.GKV_MODE_MAX, gkv.GKV_MODE_LOCAL):
+        cfg = gkv.make_config(**shape, mode=mode, fuse_window_scores=True, track_positions=True)
+        cache = gkv.GKVCache(cfg, DEV)
+        stream = synth.DecodeStream(synth.BASE_SEED + 1, n_layers=1, batch=1, h_q=28, h_kv=4, b=b, s=s, device=DEV)
+        planted = sorted(stream.planted_steps)
+        out = torch.empty((1, 1, 28, 128), dtype=torch.bfloat16, device=DEV)
+        kept = torch.empty((1, H, b), dtype=torch.int32, device=DEV)
+        pos_step = torch.zeros((1, H), dtype=torch.int32, device=DEV)
+        real = 0
+        for t in range(steps):
+            q, kn, vn = stream.step()
+            n_before = cache.state(0)[0]
+            cache.decode_attn(0, q[0], kn[0], vn[0], out[0])
+            cache.pos[0, :, :, n_before] = t                      # original position of the appended token
+            if mode == gkv.GKV_MODE_MAX and t % 499 == 0:
+                ref = oracle.decode_batch(synth.bits(q[0]), synth.bits(cache.k[0]), synth.bits(cache.v[0]), n_before + 1)
+                assert np.abs(out[0].float().cpu().numpy() - ref).max() < DECODE_ATOL, t
+            if (t + 1) % s == 0:
+                l, n_h, _ = cache.state(0)
+                snap = snapshot(cache, 0, [0]) if mode == gkv.GKV_MODE_MAX else None
+                cache.evict(0, None, kept)
+                if l > b:
+                    real += 1
+                    if snap is not None:
+                        check_evict_against_oracle(cache, 0, [0], snap, kept.cpu().numpy(), l=l, n_h=n_h)
+        cache.poll()
+        assert real == 28 and cache.state(0) == (b, b - w, 0)
+        final_pos = cache.pos[0, 0, :, :b].cpu().numpy()
+        survivors[mode] = sum(int(np.isin(planted, final_pos[j]).sum()) for j in range(H))
+    # the keys that regain attention only now and then are what the global score is for (Section 4 / 5)
+    assert survivors[gkv.GKV_MODE_MAX] >= survivors[gkv.GKV_MODE_LOCAL]
+    assert survivors[gkv.GKV_MODE_MAX] > 0
+
+
+def test_full_size_config3_largest_cell_sampled():
+    """Largest cell of the configuration-3 sweep (32 q / 8 kv heads, b = 2048, batch 256, w = 64, l = 2176): the
+    step from the window queries (tcgen05 scoring kernel, 2048 units) in the benchmark's launch configuration,
+    sampled units against the oracle and structure for all."""
+    shape = dict(batch=256, h_q=32, h_kv=8, b=2048, buffer=128, w=64, s=128)
+    cfg = gkv.make_config(n_layers=1, **shape, fuse_window_scores=False, track_positions=False)
+    cache = gkv.GKVCache(cfg, DEV)
+    case = synth.eviction_case(synth.BASE_SEED + 3, batch=256, h_q=32, h_kv=8, b=2048, buffer=128, w=64, n_planted=22, device=DEV)
+    cache.k[0].copy_(case.k); cache.v[0].copy_(case.v); cache.f[0].copy_(case.f_prev)
+    cache.set_state(0, case.l, case.n_h, 128, False)
+    seqs = [0, 101, 255]
+    snap = snapshot(cache, 0, seqs)
+    kept = torch.empty((256, 8, 2048), dtype=torch.int32, device=DEV)
+    cache.evict(0, case.q_win, kept)
+    cache.poll()
+    kk = kept.cpu().numpy()
+    check_evict_against_oracle(cache, 0, seqs, snap, kk[seqs], l=case.l, n_h=case.n_h,
+                               q_win=[synth.bits(case.q_win[n]) for n in seqs])
+    assert (np.diff(kk, axis=-1) > 0).all() and (kk[..., 2048 - 64:] == np.arange(2176 - 64, 2176)).all()
+    assert int(cache.len[0].min()) == int(cache.len[0].max()) == 2048
+    for n in seqs:   # the heavy hitters carry e^4 times the weight of ordinary keys: always kept
+        for j in range(8):
+            assert set(case.planted[n, j].tolist()) <= set(kk[n, j].tolist())
