@@ -27,6 +27,7 @@ struct __align__(8) DecodeSmemTail {
     float l[kConsumerWarps][8];
     float fin_m[8];
     float fin_l[8];
+    float wgt[kConsumerWarps][8];
     int abort_flag;
     int issued;
     int is_last;
@@ -316,23 +317,33 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
     }
     __syncthreads();  // [B]
 
-    // CTA-level state: M, L per head and the merged accumulator column of this thread's dim
-    float o[8], M[8], L[8];
+    // CTA-level state: per head the combined (max, sum) of the four warps and each warp's weight ...
+    if (tid < 8) {
+        const int h = tid;
+        float mm = tail->m[0][h];
+#pragma unroll
+        for (int w = 1; w < kConsumerWarps; ++w) mm = fmaxf(mm, tail->m[w][h]);
+        float ll = 0.f;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+            const float wm = tail->m[w][h];
+            const float wgt = (wm == -INFINITY) ? 0.f : fast_exp2(wm - mm);
+            tail->wgt[w][h] = wgt;
+            ll += wgt * tail->l[w][h];
+        }
+        tail->fin_m[h] = mm;
+        tail->fin_l[h] = ll;
+    }
+    __syncthreads();
+    // ... and per thread (one of the 128 dims) the merged accumulator of the 8 heads
+    float o[8];
     if (tid < kHeadDim) {
 #pragma unroll
         for (int h = 0; h < 8; ++h) {
-            float mm = tail->m[0][h];
+            float oo = 0.f;
 #pragma unroll
-            for (int w = 1; w < kConsumerWarps; ++w) mm = fmaxf(mm, tail->m[w][h]);
-            float ll = 0.f, oo = 0.f;
-#pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) {
-                const float wm = tail->m[w][h];
-                const float wgt = (wm == -INFINITY) ? 0.f : fast_exp2(wm - mm);
-                ll += wgt * tail->l[w][h];
-                oo += wgt * s_acc[w * (kHeadDim * 8) + tid * 8 + h];
-            }
-            M[h] = mm; L[h] = ll; o[h] = oo;
+            for (int w = 0; w < kConsumerWarps; ++w) oo += tail->wgt[w][h] * s_acc[w * (kHeadDim * 8) + tid * 8 + h];
+            o[h] = oo;
         }
     }
 
@@ -341,7 +352,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
     if (p.splits > 1) {
         float* mine = p.part + ((size_t)unit_local * p.splits + split) * kPartFloats;
         if (tid < kHeadDim) {
-            if (tid < 8) { mine[tid] = M[tid]; mine[8 + tid] = L[tid]; }
+            if (tid < 8) { mine[tid] = tail->fin_m[tid]; mine[8 + tid] = tail->fin_l[tid]; }
             float4* d4 = reinterpret_cast<float4*>(mine + 16 + tid * 8);
             d4[0] = make_float4(o[0], o[1], o[2], o[3]);
             d4[1] = make_float4(o[4], o[5], o[6], o[7]);
@@ -356,21 +367,43 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
         __syncthreads();
         do_final = tail->is_last != 0;
         if (do_final) {
+            // The last CTA of the unit merges the partials. All loads of a phase are independent, so the merge
+            // costs a few L2 round trips, not one per split: (1) every split's (max, sum) into shared memory,
+            // (2) per head the global max, the splits' weights and the global sum, (3) per dim the weighted sum
+            // of the splits' accumulators.
             __threadfence();
+            const float* base = p.part + (size_t)unit_local * p.splits * kPartFloats;
+            float* s_stat = s_acc;                 // [splits][16]: M[8], L[8]   (the accumulators are in registers now)
+            float* s_w = s_acc + 32 * 16;          // [splits][8] weights
+            for (int idx = tid; idx < p.splits * 16; idx += kDecodeThreads)
+                s_stat[idx] = __ldcg(base + (size_t)(idx >> 4) * kPartFloats + (idx & 15));
+            __syncthreads();
+            if (tid < 8) {
+                const int h = tid;
+                float mm = -INFINITY;
+                for (int sp = 0; sp < p.splits; ++sp) mm = fmaxf(mm, s_stat[sp * 16 + h]);
+                float ll = 0.f;
+                for (int sp = 0; sp < p.splits; ++sp) {
+                    const float wm = s_stat[sp * 16 + h];
+                    const float wgt = (wm == -INFINITY) ? 0.f : fast_exp2(wm - mm);
+                    s_w[sp * 8 + h] = wgt;
+                    ll += wgt * s_stat[sp * 16 + 8 + h];
+                }
+                tail->fin_m[h] = mm;
+                tail->fin_l[h] = ll;
+            }
+            __syncthreads();
             if (tid < kHeadDim) {
-                const float* base = p.part + (size_t)unit_local * p.splits * kPartFloats;
 #pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    float mm = -INFINITY;
-                    for (int sp = 0; sp < p.splits; ++sp) mm = fmaxf(mm, __ldcg(base + sp * kPartFloats + h));
-                    float ll = 0.f, oo = 0.f;
-                    for (int sp = 0; sp < p.splits; ++sp) {
-                        const float wm = __ldcg(base + sp * kPartFloats + h);
-                        const float wgt = (wm == -INFINITY) ? 0.f : fast_exp2(wm - mm);
-                        ll += wgt * __ldcg(base + sp * kPartFloats + 8 + h);
-                        oo += wgt * __ldcg(base + sp * kPartFloats + 16 + tid * 8 + h);
-                    }
-                    M[h] = mm; L[h] = ll; o[h] = oo;
+                for (int h = 0; h < 8; ++h) o[h] = 0.f;
+#pragma unroll 4
+                for (int sp = 0; sp < p.splits; ++sp) {
+                    const float4* a4 = reinterpret_cast<const float4*>(base + (size_t)sp * kPartFloats + 16 + tid * 8);
+                    const float4 a = __ldcg(a4), b = __ldcg(a4 + 1);
+                    const float4 wa = *reinterpret_cast<const float4*>(s_w + sp * 8);
+                    const float4 wb = *reinterpret_cast<const float4*>(s_w + sp * 8 + 4);
+                    o[0] = fmaf(wa.x, a.x, o[0]); o[1] = fmaf(wa.y, a.y, o[1]); o[2] = fmaf(wa.z, a.z, o[2]); o[3] = fmaf(wa.w, a.w, o[3]);
+                    o[4] = fmaf(wb.x, b.x, o[4]); o[5] = fmaf(wb.y, b.y, o[5]); o[6] = fmaf(wb.z, b.z, o[6]); o[7] = fmaf(wb.w, b.w, o[7]);
                 }
             }
         }
@@ -381,8 +414,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
             __nv_bfloat16* orow = p.out + ((size_t)(layer_local * p.batch + seq) * p.h_q + (size_t)head * p.g) * kHeadDim + tid;
 #pragma unroll
             for (int h = 0; h < 8; ++h)
-                if (h < p.g) orow[(size_t)h * kHeadDim] = __float2bfloat16_rn(o[h] / L[h]);
-            if (tid < 8) { tail->fin_m[tid] = M[tid]; tail->fin_l[tid] = L[tid]; }
+                if (h < p.g) orow[(size_t)h * kHeadDim] = __float2bfloat16_rn(o[h] / tail->fin_l[h]);
         }
         if (ACCUM != 0) {
             if (ACCUM == 1) cp_async_wait_all();
