@@ -8,8 +8,6 @@
 // heads of the group on the N side (S^T = K Q^T, O^T = V^T P^T): no padded rows, each K/V byte
 // is read from shared memory exactly once, and the P^T operand comes from the S^T accumulator by
 // an 8x8 register transpose (movmatrix).
-#include <stdlib.h>
-
 #include "gkv_common.cuh"
 #include "gkv_internal.h"
 
@@ -495,15 +493,17 @@ int decode_tmem_cols(int C) {
     return cols;   // C <= 4096 -> at most 256
 }
 
+// Key split of a launch with few units: about two CTAs per SM, so that all of them run in one wave (measured
+// on 4..256 units of 18 tiles: 2 and 3 per SM are equal, 4 and more cost a second wave and 30-50 % more
+// time); the tiles are then spread evenly (no CTA without a tile).
 int decode_pick_splits(int units_in_launch, int C, int sm_count) {
     const int max_tiles = (C + kTileKeys - 1) / kTileKeys;
-    const int want = 4 * sm_count;  // enough CTAs for two per SM, twice over
     if (units_in_launch >= 2 * sm_count) return 1;
-    int s = (want + units_in_launch - 1) / units_in_launch;
-    if (s > max_tiles) s = max_tiles;
-    if (s > 32) s = 32;
-    if (s < 1) s = 1;
-    return s;
+    int s_max = (2 * sm_count) / units_in_launch;
+    if (s_max > 32) s_max = 32;
+    if (s_max < 1) s_max = 1;
+    const int tiles_per_split = (max_tiles + s_max - 1) / s_max;
+    return (max_tiles + tiles_per_split - 1) / tiles_per_split;
 }
 
 // Resident CTAs per SM matter more than ring depth: with four consumer warps per CTA the per-warp
@@ -525,11 +525,6 @@ int decode_pick_stages(int C, int accum, int splits, size_t* smem_bytes) {
             best_score = score;
             best = st;
         }
-    }
-    // tuning knobs for experiments: GKV_DECODE_STAGES (plain steps), GKV_DECODE_STAGES_WINDOW (window steps)
-    if (const char* e = getenv(accum ? "GKV_DECODE_STAGES_WINDOW" : "GKV_DECODE_STAGES")) {
-        const int st = atoi(e);
-        if (st >= 2 && st <= kMaxStages && decode_smem_bytes(C, accum, splits, st) <= cap) best = st;
     }
     if (smem_bytes) *smem_bytes = decode_smem_bytes(C, accum, splits, best);
     return best;

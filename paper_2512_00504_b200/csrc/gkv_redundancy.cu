@@ -14,8 +14,6 @@
 // D[own key][other key] in two 256-column TMEM buffers, and 16 epilogue warps (same roles and
 // barriers as the scoring kernel) scale, threshold and add. The softmax and the max-normalisation
 // of the appendix reduce to exp(cbar - max cbar), which the eviction kernel applies.
-#include <stdlib.h>
-
 #include "gkv_common.cuh"
 #include "gkv_internal.h"
 #include "gkv_tcgen05.cuh"

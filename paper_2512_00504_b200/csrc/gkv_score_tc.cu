@@ -16,8 +16,6 @@
 // tcgen05.ld and do the softmax arithmetic, so copy, tensor work and exponentials overlap; the
 // groups split an accumulator's columns, which keeps four warps per scheduler to hide latencies.
 // Window token k sees the keys t <= n - w + k (its own key included).
-#include <stdlib.h>
-
 #include "gkv_common.cuh"
 #include "gkv_internal.h"
 #include "gkv_tcgen05.cuh"
@@ -368,10 +366,6 @@ cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const
     // the deepest K ring that fits: bytes in flight per SM are what hides the copy latency (one CTA per SM)
     int stages = 2;
     while (stages < kTcMaxStages && score_tc_smem_bytes(p.C, p.g * wk, stages + 1) <= 227 * 1024) ++stages;
-    if (const char* e = getenv("GKV_SCORE_STAGES")) {   // tuning knob for experiments
-        const int st = atoi(e);
-        if (st >= 2 && st <= stages) stages = st;
-    }
     const size_t smem = score_tc_smem_bytes(p.C, p.g * wk, stages);
     if (n_cta > 1) {
         const size_t off = (size_t)p.layer0 * p.batch * p.h_kv * p.C;
