@@ -447,6 +447,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
 #pragma unroll
                 for (int h = 0; h < 8; ++h) c[h] = (h < p.g) ? tail->fin_m[h] + log2f(tail->fin_l[h]) : INFINITY;
                 const float* g_log = p.logits + (size_t)unit_local * p.C * 8;
+#pragma unroll 4   // independent loads: a few L2 round trips for the unit's logits instead of one per iteration
                 for (int t = tid; t < n_keys_all; t += kDecodeThreads) {
                     const float4 x0 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8));
                     const float4 x1 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8 + 4));

@@ -484,3 +484,53 @@ def test_full_size_config3_largest_cell_sampled():
     for n in seqs:   # the heavy hitters carry e^4 times the weight of ordinary keys: always kept
         for j in range(8):
             assert set(case.planted[n, j].tolist()) <= set(kk[n, j].tolist())
+
+
+@pytest.mark.parametrize("shape,kw", [
+    (dict(batch=1, h_q=16, h_kv=2, b=3968, buffer=128, w=64, s=128), dict()),                 # largest cache the library takes (C = 4096), g = 8
+    (dict(batch=2, h_q=4, h_kv=4, b=64, buffer=16, w=16, s=16), dict(alpha=1.0)),              # g = 1, interval = window, no decay
+    (dict(batch=2, h_q=2, h_kv=1, b=33, buffer=9, w=32, s=32, ), dict(n_h=1)),                 # keeps a single candidate (b - w = 1); buffer < s is refused
+    (dict(batch=1, h_q=8, h_kv=1, b=100, buffer=50, w=1, s=50), dict(alpha=0.0, mode=gkv.GKV_MODE_SUM)),  # one-token window, history switched off
+])
+def test_evict_edge_shapes(shape, kw):
+    if shape["s"] > shape["buffer"]:
+        with pytest.raises(gkv.GKVError) as e:
+            gkv.GKVCache(gkv.make_config(n_layers=1, **shape), DEV)
+        assert e.value.status == gkv.GKV_ERR_INVALID_ARG
+        shape = dict(shape, buffer=shape["s"])
+    run_single_eviction(shape, synth.BASE_SEED + 90 + shape["w"], **kw)
+    run_single_eviction(shape, synth.BASE_SEED + 91 + shape["w"], recompute=False, **kw)
+
+
+def test_decode_at_maximum_capacity_with_window_accumulation():
+    """C = 4096 rows (the largest capacity), g = 8: the last window of a period, split and unsplit launches,
+    against the oracle; the cache ends completely full."""
+    for batch in (1, 40):                                           # 2 units (key split) and 80 units x 4 heads = 320 (one CTA per unit)
+        shape = dict(batch=batch, h_q=32, h_kv=4 if batch > 1 else 2, b=3968, buffer=128, w=16, s=128)
+        shape["h_q"] = shape["h_kv"] * 8
+        cfg = gkv.make_config(n_layers=1, **shape, fuse_window_scores=True)
+        cache = gkv.GKVCache(cfg, DEV)
+        B, Hq, H, C, w = batch, shape["h_q"], shape["h_kv"], 4096, 16
+        gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 95)
+        rnd = lambda *sh: torch.randn(*sh, generator=gen, device=DEV).to(torch.bfloat16)
+        start = C - w
+        cache.k[0, :, :, :start] = rnd(B, H, start, 128)
+        cache.v[0, :, :, :start] = rnd(B, H, start, 128)
+        cache.set_state(0, start, 3952, 128 - w)
+        sel = [0] if B == 1 else [0, B - 1]
+        out = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device=DEV)
+        sacc = np.zeros((len(sel), H, C), np.float64)
+        for t in range(w):
+            q, kn, vn = rnd(B, Hq, 128), rnd(B, H, 128), rnd(B, H, 128)
+            cache.decode_attn(0, q, kn, vn, out)
+            if t in (0, w - 1):
+                ref = oracle.decode_batch(synth.bits(q)[sel], synth.bits(cache.k[0])[sel], synth.bits(cache.v[0])[sel],
+                                          start + t + 1, Sacc=None)
+                assert np.abs(out.float().cpu().numpy()[sel] - ref).max() < DECODE_ATOL
+            oracle.decode_batch(synth.bits(q)[sel], synth.bits(cache.k[0])[sel], synth.bits(cache.v[0])[sel], start + t + 1, Sacc=sacc)
+        cache.poll()
+        assert cache.state(0) == (C, 3952, 128)
+        np.testing.assert_allclose(cache.sacc[0].cpu().numpy()[sel], sacc, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+        with pytest.raises(gkv.GKVError) as e:
+            cache.decode_attn(0, q, kn, vn, out)
+        assert e.value.status == gkv.GKV_ERR_CAPACITY
