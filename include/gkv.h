@@ -165,7 +165,11 @@ gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const voi
 /* Same operations with HOST buffers: inputs are copied to the staging buffer on `stream`, the
  * kernels run, and the result is copied back, all asynchronously on `stream` (synchronise the
  * stream before reading out / kept_idx_out). Require buffers.staging.
- * Errors: as the device calls; INVALID_ARG when no staging buffer was given. */
+ * gkv_decode_attn_host takes a faster route when all four of its buffers are page-locked and mapped
+ * (cudaHostAlloc, cudaHostRegister, a pinned torch tensor): the kernel reads and writes them in place
+ * across the bus (zero copy, no staging buffer needed), which overlaps the transfers with the
+ * attention. The result is again complete once `stream` has been synchronised.
+ * Errors: as the device calls; INVALID_ARG when staging is needed and no staging buffer was given. */
 gkv_status gkv_decode_attn_host(gkv_ctx* ctx, int32_t layer, const void* q_host, const void* k_new_host,
                                 const void* v_new_host, void* out_host, void* stream);
 gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host,

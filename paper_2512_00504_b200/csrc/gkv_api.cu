@@ -491,9 +491,27 @@ gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const voi
     return GKV_OK;
 }
 
+// Device alias of a host pointer when the memory is page-locked and mapped into the device's address space
+// (cudaHostAlloc / cudaHostRegister, torch's pin_memory()); NULL for pageable memory.
+static void* mapped_alias(const void* host_ptr) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host_ptr) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    return (at.type == cudaMemoryTypeHost) ? at.devicePointer : nullptr;
+}
+
 gkv_status gkv_decode_attn_host(gkv_ctx* ctx, int32_t layer, const void* q_host, const void* k_new_host,
                                 const void* v_new_host, void* out_host, void* stream) {
     if (!ctx || !layer_ok(ctx, layer) || !q_host || !k_new_host || !v_new_host || !out_host) return GKV_ERR_INVALID_ARG;
+    {
+        // Zero copy: with page-locked, mapped host buffers the kernel itself reads q / k_new / v_new and writes out
+        // across the bus, so the transfers of one unit overlap the attention of the others instead of being
+        // serialised before and after the launch.
+        void *aq = mapped_alias(q_host), *ak = mapped_alias(k_new_host), *av = mapped_alias(v_new_host), *ao = mapped_alias(out_host);
+        if (aq && ak && av && ao) return gkv_decode_attn(ctx, layer, aq, ak, av, ao, stream);
+    }
     if (!ctx->buf.staging) return GKV_ERR_INVALID_ARG;
     int l0, nl;
     layer_range(ctx, layer, &l0, &nl);

@@ -534,3 +534,37 @@ def test_decode_at_maximum_capacity_with_window_accumulation():
         with pytest.raises(gkv.GKVError) as e:
             cache.decode_attn(0, q, kn, vn, out)
         assert e.value.status == gkv.GKV_ERR_CAPACITY
+
+
+@pytest.mark.parametrize("pinned", [False, True])
+def test_host_buffer_entry_points_equal_the_device_calls(pinned):
+    """gkv_decode_attn_host / gkv_evict_host with pageable host buffers (staged copies) and with page-locked
+    mapped ones (the decode kernel then reads and writes them in place): bit-equal to the device-pointer calls."""
+    shape = dict(n_layers=2, batch=3, h_q=8, h_kv=2, b=96, buffer=32, w=8, s=32)
+    caches = [gkv.GKVCache(gkv.make_config(**shape, fuse_window_scores=True), DEV, staging=True) for _ in range(2)]
+    dev_c, host_c = caches
+    gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 97)
+    rnd = lambda *sh: torch.randn(*sh, generator=gen, device=DEV).to(torch.bfloat16)
+    k0, v0 = rnd(2, 3, 2, 100, 128), rnd(2, 3, 2, 100, 128)
+    for c in caches:
+        c.k[:, :, :, :100] = k0; c.v[:, :, :, :100] = v0
+        c.set_state(-1, 100, 0, 4)
+    mk = (lambda t: t.cpu().pin_memory()) if pinned else (lambda t: t.cpu())
+    out_d = torch.empty((2, 3, 8, 128), dtype=torch.bfloat16, device=DEV)
+    out_h = mk(torch.zeros((2, 3, 8, 128), dtype=torch.bfloat16))
+    for t in range(28):                                              # through the window steps up to the compression
+        q, kn, vn = rnd(2, 3, 8, 128), rnd(2, 3, 2, 128), rnd(2, 3, 2, 128)
+        dev_c.decode_attn(-1, q, kn, vn, out_d)
+        gkv.gkv_decode_attn_host(host_c.ctx, -1, mk(q), mk(kn), mk(vn), out_h)
+        torch.cuda.synchronize()
+        assert torch.equal(out_d.cpu(), out_h), t
+    assert torch.equal(dev_c.k, host_c.k) and torch.equal(dev_c.sacc, host_c.sacc)
+    kept_d = torch.empty((2, 3, 2, 96), dtype=torch.int32, device=DEV)
+    kept_h = mk(torch.zeros((2, 3, 2, 96), dtype=torch.int32))
+    dev_c.evict(-1, None, kept_d)
+    gkv.gkv_evict_host(host_c.ctx, -1, None, kept_h)
+    torch.cuda.synchronize()
+    assert torch.equal(kept_d.cpu(), kept_h) and torch.equal(dev_c.k[..., :96, :], host_c.k[..., :96, :])
+    assert dev_c.state(0) == host_c.state(0) == (96, 88, 0)
+    for c in caches:
+        c.poll()
