@@ -163,6 +163,14 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
                 }
             }
         }
+        // The current token's row lands in the last tile; the warp that will append it fetches its 16 bytes per lane
+        // now (lanes 0-15 of k_new, 16-31 of v_new), so that the load's latency -- a bus round trip when the inputs
+        // are mapped host memory -- is long over when the row is needed.
+        uint4 new_row = make_uint4(0u, 0u, 0u, 0u);
+        if (warp == ((len_old & (kTileKeys - 1)) >> 4) && (len_old / kTileKeys) >= t_begin && (len_old / kTileKeys) < t_end) {
+            const size_t src = ((size_t)(layer_local * p.batch + seq) * p.h_kv + head) * kHeadDim + (lane & 15) * 8;
+            new_row = *reinterpret_cast<const uint4*>((lane < 16 ? p.k_new : p.v_new) + src);
+        }
         const int krow = warp * 16 + (mat & 1) * 8 + r_in;   // K ldmatrix: row this lane addresses
         const int kch = mat >> 1;                             //   and which 16-byte chunk of the k step
         const int vrow = warp * 16 + (mat >> 1) * 8 + r_in;   // V ldmatrix (transposed)
@@ -185,16 +193,13 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
                 if (len_old >= key0 && len_old < key0 + 16) {
                     const int lr = len_old - it * kTileKeys;          // row inside the tile
                     const int c = lane & 15;
-                    const size_t src = ((size_t)(layer_local * p.batch + seq) * p.h_kv + head) * kHeadDim + c * 8;
                     const size_t dstg = ((size_t)unit * p.C + len_old) * kHeadDim + c * 8;
                     if (lane < 16) {
-                        const uint4 x = *reinterpret_cast<const uint4*>(p.k_new + src);
-                        *reinterpret_cast<uint4*>(kt + tile_off(lr, c)) = x;
-                        *reinterpret_cast<uint4*>(p.k_cache + dstg) = x;
+                        *reinterpret_cast<uint4*>(kt + tile_off(lr, c)) = new_row;
+                        *reinterpret_cast<uint4*>(p.k_cache + dstg) = new_row;
                     } else {
-                        const uint4 x = *reinterpret_cast<const uint4*>(p.v_new + src);
-                        *reinterpret_cast<uint4*>(vt + tile_off(lr, c)) = x;
-                        *reinterpret_cast<uint4*>(p.v_cache + dstg) = x;
+                        *reinterpret_cast<uint4*>(vt + tile_off(lr, c)) = new_row;
+                        *reinterpret_cast<uint4*>(p.v_cache + dstg) = new_row;
                     }
                     fence_proxy_async_smem();
                 }
