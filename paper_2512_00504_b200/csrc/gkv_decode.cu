@@ -17,8 +17,9 @@ constexpr int kConsumerWarps = 4;
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 constexpr int kMaxStages = 6;
 constexpr int kPartFloats = 16 + kHeadDim * 8;  // M[8], L[8], acc[128][8]
+constexpr int kQRowBytes = 272;                 // 256 bytes of a query row + 16 of padding
 
-struct __align__(8) DecodeSmemTail {
+struct __align__(16) DecodeSmemTail {
     uint64_t full_bar[kMaxStages];
     uint64_t empty_bar[kMaxStages];
     float m[kConsumerWarps][8];
@@ -26,6 +27,7 @@ struct __align__(8) DecodeSmemTail {
     float fin_m[8];
     float fin_l[8];
     float wgt[kConsumerWarps][8];
+    alignas(16) uint8_t q_rows[8 * 272];   // the group's query rows, 272 bytes apart
     int abort_flag;
     int issued;
     int is_last;
@@ -149,15 +151,25 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
         const int r_in = lane & 7, mat = lane >> 3;
         const int hq = lane >> 2;                     // head whose Q row this lane holds (B operand)
         // Q^T fragments: B[k = d][n = head], two packed bf16 pairs per 16-wide k step
+        // The group's g query rows come in once per CTA with 16-byte loads (warp w fetches heads w and w + 4, one
+        // row per half warp) and are re-read from shared memory in fragment order: one bus or L2 transaction per
+        // 16 bytes instead of four copies of it in 4-byte pieces. Rows are 272 bytes apart: conflict-free reads.
         uint32_t qf[8][2];
         {
-            const __nv_bfloat16* qrow =
-                p.q + ((size_t)(layer_local * p.batch + seq) * p.h_q + (size_t)head * p.g + hq) * kHeadDim;
+            const int hl = warp + (lane >> 4) * kConsumerWarps;          // head this half warp fetches
+            if (hl < p.g) {
+                const __nv_bfloat16* qrow =
+                    p.q + ((size_t)(layer_local * p.batch + seq) * p.h_q + (size_t)head * p.g + hl) * kHeadDim;
+                *reinterpret_cast<uint4*>(tail->q_rows + hl * kQRowBytes + (lane & 15) * 16) =
+                    *reinterpret_cast<const uint4*>(qrow + (lane & 15) * 8);
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");   // the four consumer warps only
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 if (hq < p.g) {
-                    qf[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + (lane & 3) * 2);
-                    qf[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + (lane & 3) * 2 + 8);
+                    const uint8_t* row = tail->q_rows + hq * kQRowBytes + ks * 32 + (lane & 3) * 4;
+                    qf[ks][0] = *reinterpret_cast<const uint32_t*>(row);
+                    qf[ks][1] = *reinterpret_cast<const uint32_t*>(row + 16);
                 } else {
                     qf[ks][0] = qf[ks][1] = 0u;
                 }
