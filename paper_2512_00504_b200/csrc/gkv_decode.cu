@@ -425,11 +425,19 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
     }
 
     if (do_final) {
+        // out = o / L as bf16, transposed through shared memory (the query rows' slot is free by now) so that it
+        // leaves in 16-byte pieces, 256 contiguous bytes per head: one row per half warp.
         if (tid < kHeadDim) {
-            __nv_bfloat16* orow = p.out + ((size_t)(layer_local * p.batch + seq) * p.h_q + (size_t)head * p.g) * kHeadDim + tid;
 #pragma unroll
             for (int h = 0; h < 8; ++h)
-                if (h < p.g) orow[(size_t)h * kHeadDim] = __float2bfloat16_rn(o[h] / tail->fin_l[h]);
+                if (h < p.g)
+                    *reinterpret_cast<__nv_bfloat16*>(tail->q_rows + h * kQRowBytes + tid * 2) = __float2bfloat16_rn(o[h] / tail->fin_l[h]);
+        }
+        __syncthreads();
+        if (tid < p.g * 16) {
+            const int h = tid >> 4, c = tid & 15;
+            __nv_bfloat16* orow = p.out + ((size_t)(layer_local * p.batch + seq) * p.h_q + (size_t)head * p.g + h) * kHeadDim;
+            *reinterpret_cast<uint4*>(orow + c * 8) = *reinterpret_cast<const uint4*>(tail->q_rows + h * kQRowBytes + c * 16);
         }
         if (ACCUM != 0) {
             if (ACCUM == 1) cp_async_wait_all();
