@@ -310,7 +310,8 @@ gkv_status gkv_init(gkv_ctx** out, const gkv_config* cfg, const gkv_buffers* b, 
                  redundancy_kernel_setup() == cudaSuccess;
     if (ok) {
         const uint64_t rows = (uint64_t)cfg->n_layers * ctx->units_per_layer * ctx->C;
-        ok = encode_map(&ctx->tm_k, b->k, rows) == GKV_OK && encode_map(&ctx->tm_v, b->v, rows) == GKV_OK;
+        ok = encode_map(&ctx->tm_k, b->k, rows) == GKV_OK && encode_map(&ctx->tm_v, b->v, rows) == GKV_OK &&
+             encode_map(&ctx->tm_k16, b->k, rows, 16) == GKV_OK && encode_map(&ctx->tm_v16, b->v, rows, 16) == GKV_OK;
     }
     if (!ok) {
         (void)cudaGetLastError();
@@ -385,7 +386,8 @@ gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const voi
     p.splits = decode_pick_splits(nl * ctx->units_per_layer, ctx->C, ctx->sm_count);
     p.stages = decode_pick_stages(ctx->C, p.accum, p.splits, nullptr);
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
-    if (launch_decode(p, ctx->tm_k, ctx->tm_v, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    const DecodeMaps maps = {ctx->tm_k, ctx->tm_v, ctx->tm_k16, ctx->tm_v16};
+    if (launch_decode(p, maps, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return GKV_ERR_CUDA;
     }

@@ -50,8 +50,7 @@ __host__ __device__ constexpr size_t decode_sum_bytes(int C, int accum_mode) {
 // ACCUM = 2: window step with the keys split over several CTAs, logits in the workspace.
 template <int ACCUM>
 __global__ void __launch_bounds__(kDecodeThreads)
-gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k,
-                  const __grid_constant__ CUtensorMap tm_v) {
+gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment for the swizzled TMA boxes
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -122,8 +121,12 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            prefetch_tensormap(&tm_k);
-            prefetch_tensormap(&tm_v);
+            prefetch_tensormap(&maps.k64);
+            prefetch_tensormap(&maps.v64);
+            if (n & (kTileKeys - 1)) {
+                prefetch_tensormap(&maps.k16);
+                prefetch_tensormap(&maps.v16);
+            }
             for (int it = t_begin; it < t_end; ++it) {
                 const int j = it - t_begin;
                 const int s = j % stages;
@@ -138,11 +141,26 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ CUtensorMap tm_k
                 const uint32_t bar = smem_u32(&tail->full_bar[s]);
                 const uint32_t dst = smem_u32(stage_base + (size_t)s * kStageBytes);
                 const int y = row0 + it * kTileKeys;
-                mbar_arrive_expect_tx(bar, kStageBytes);
-                tma_load_2d(dst, &tm_k, 0, y, bar);
-                tma_load_2d(dst + kBoxBytes, &tm_k, 64, y, bar);
-                tma_load_2d(dst + kTileBytes, &tm_v, 0, y, bar);
-                tma_load_2d(dst + kTileBytes + kBoxBytes, &tm_v, 64, y, bar);
+                const int rows_left = n - it * kTileKeys;       // keys of this tile that exist
+                if (rows_left > kTileKeys - 16) {
+                    mbar_arrive_expect_tx(bar, kStageBytes);
+                    tma_load_2d(dst, &maps.k64, 0, y, bar);
+                    tma_load_2d(dst + kBoxBytes, &maps.k64, 64, y, bar);
+                    tma_load_2d(dst + kTileBytes, &maps.v64, 0, y, bar);
+                    tma_load_2d(dst + kTileBytes + kBoxBytes, &maps.v64, 64, y, bar);
+                } else {
+                    // ragged last tile: only the 16-row pieces that hold keys (a 16-row piece of a 128-byte-swizzled
+                    // 64-row box is 2 KB at row offset 16 * piece; the swizzle pattern repeats every 8 rows)
+                    const int pieces = (rows_left + 15) >> 4;
+                    mbar_arrive_expect_tx(bar, (uint32_t)pieces * 4 * 2048);
+                    for (int pc = 0; pc < pieces; ++pc) {
+                        const uint32_t o = (uint32_t)pc * 2048;
+                        tma_load_2d(dst + o, &maps.k16, 0, y + pc * 16, bar);
+                        tma_load_2d(dst + kBoxBytes + o, &maps.k16, 64, y + pc * 16, bar);
+                        tma_load_2d(dst + kTileBytes + o, &maps.v16, 0, y + pc * 16, bar);
+                        tma_load_2d(dst + kTileBytes + kBoxBytes + o, &maps.v16, 64, y + pc * 16, bar);
+                    }
+                }
                 *(volatile int*)&tail->issued = it + 1;
             }
         }
@@ -564,14 +582,14 @@ cudaError_t decode_kernel_setup() {
     return cudaFuncSetAttribute(gkv_decode_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }
 
-cudaError_t launch_decode(const DecodeLaunch& p_in, const CUtensorMap& tm_k, const CUtensorMap& tm_v, cudaStream_t s) {
+cudaError_t launch_decode(const DecodeLaunch& p_in, const DecodeMaps& maps, cudaStream_t s) {
     DecodeLaunch p = p_in;
     p.tmem_cols = decode_tmem_cols(p.C);
     const size_t smem = decode_smem_bytes(p.C, p.accum, p.splits, p.stages);
     const int grid = p.n_layers * p.batch * p.h_kv * p.splits;
-    if (!p.accum) gkv_decode_kernel<0><<<grid, kDecodeThreads, smem, s>>>(p, tm_k, tm_v);
-    else if (p.splits == 1) gkv_decode_kernel<1><<<grid, kDecodeThreads, smem, s>>>(p, tm_k, tm_v);
-    else gkv_decode_kernel<2><<<grid, kDecodeThreads, smem, s>>>(p, tm_k, tm_v);
+    if (!p.accum) gkv_decode_kernel<0><<<grid, kDecodeThreads, smem, s>>>(p, maps);
+    else if (p.splits == 1) gkv_decode_kernel<1><<<grid, kDecodeThreads, smem, s>>>(p, maps);
+    else gkv_decode_kernel<2><<<grid, kDecodeThreads, smem, s>>>(p, maps);
     return cudaGetLastError();
 }
 

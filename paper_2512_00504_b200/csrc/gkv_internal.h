@@ -50,6 +50,13 @@ struct DecodeLaunch {
     float scale_log2;    // log2(e) / sqrt(d)
 };
 
+// Tensor maps of the decode kernel: K and V as [rows][128] bf16 with 64-row boxes (full tiles) and with 16-row
+// boxes (the ragged last tile of a unit is fetched in 16-row pieces, so at most 15 rows past the cache's end
+// cross the memory bus instead of up to 63).
+struct DecodeMaps {
+    CUtensorMap k64, v64, k16, v16;
+};
+
 struct EvictLaunch {
     __nv_bfloat16* k_cache;
     __nv_bfloat16* v_cache;
@@ -117,7 +124,8 @@ struct gkv_ctx {
     gkv::WorkspaceLayout ws;
     int C, g, units_per_layer;
     int device, sm_count;
-    CUtensorMap tm_k, tm_v;
+    CUtensorMap tm_k, tm_v;   // 64-row boxes
+    CUtensorMap tm_k16, tm_v16;   // 16-row boxes
     std::vector<int32_t> len, n_hist, since_evict, sacc_valid, stage_next, cbar_valid;
     int64_t launches;
     int32_t* evict_log;  // caller's device buffer for the eviction log, or NULL
@@ -128,7 +136,7 @@ namespace gkv {
 
 int decode_pick_splits(int units_in_launch, int C, int sm_count);
 int decode_pick_stages(int C, int accum, int splits, size_t* smem_bytes);
-cudaError_t launch_decode(const DecodeLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_v, cudaStream_t s);
+cudaError_t launch_decode(const DecodeLaunch& p, const DecodeMaps& maps, cudaStream_t s);
 cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s);
 cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s);
 cudaError_t launch_evict_select(const EvictLaunch& p, cudaStream_t s);

@@ -73,8 +73,8 @@ typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// [rows][128] bf16 view in 64 x 64 boxes with the 128-byte swizzle the decode kernel expects.
-bool encode_rows(CUtensorMap* map, void* base, uint64_t rows) {
+// [rows][128] bf16 view in boxes of box_rows rows x 64 elements with the 128-byte swizzle the decode kernel expects.
+bool encode_rows(CUtensorMap* map, void* base, uint64_t rows, uint32_t box_rows) {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
@@ -82,7 +82,7 @@ bool encode_rows(CUtensorMap* map, void* base, uint64_t rows) {
         return false;
     const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kTileKeys};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return reinterpret_cast<EncodeFn>(sym)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
                                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -115,8 +115,10 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     DecodeLaunch p;
     p.splits = decode_pick_splits((int)units, capacity, sm);
     if (units * p.splits > kStaticMaxCtas) return GKV_ERR_SCRATCH_LIMIT;
-    CUtensorMap tm_k, tm_v;
-    if (!encode_rows(&tm_k, k_cache, (uint64_t)units * capacity) || !encode_rows(&tm_v, v_cache, (uint64_t)units * capacity))
+    DecodeMaps maps;
+    const uint64_t rows = (uint64_t)units * capacity;
+    if (!encode_rows(&maps.k64, k_cache, rows, kTileKeys) || !encode_rows(&maps.v64, v_cache, rows, kTileKeys) ||
+        !encode_rows(&maps.k16, k_cache, rows, 16) || !encode_rows(&maps.v16, v_cache, rows, 16))
         return GKV_ERR_CUDA;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -145,7 +147,7 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     p.accum = 0;
     p.stages = decode_pick_stages(capacity, 0, p.splits, nullptr);
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
-    if (launch_decode(p, tm_k, tm_v, s) != cudaSuccess) {
+    if (launch_decode(p, maps, s) != cudaSuccess) {
         (void)cudaGetLastError();
         return GKV_ERR_CUDA;
     }
