@@ -123,7 +123,7 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tail->d_full[b]), 1);
-            mbar_init(smem_u32(&tail->d_empty[b]), kRdEpiThreads / 32);
+            mbar_init(smem_u32(&tail->d_empty[b]), kRdEpiThreads / 64);   // the eight warps that read this accumulator
         }
         mbar_init(smem_u32(&tail->drain), 1);
         tail->abort_flag = 0;
@@ -213,18 +213,21 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
         const int q4 = warp & 3;
         const int L = q4 * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q4 * 32) << 16);
-        // two row tiles: two groups per tile, 64 columns each; one tile: four groups, 32 columns each
-        const int rl = (MT == 2) ? (wg >> 1) * 128 + L : L;
-        const int col0 = (MT == 2) ? (wg & 1) * 64 : wg * 32;
-        const int nch = (MT == 2) ? 2 : 1;
-        const uint32_t t_p = t_lane + (uint32_t)((MT == 2) ? (wg >> 1) * 128 + col0 : col0);
+        // Groups 0, 1 take the even key tiles (accumulator 0), groups 2, 3 the odd ones (accumulator 1), so two tiles
+        // are in the epilogue at any time and one pair's TMEM loads overlap the other pair's arithmetic. Within a
+        // pair: two row tiles -> one each, all 128 columns; one row tile -> 64 columns each.
+        const int parity = wg >> 1, sub = wg & 1;
+        const int rl = (MT == 2) ? sub * 128 + L : L;
+        const int col0 = (MT == 2) ? 0 : sub * 64;
+        const int nch = (MT == 2) ? 4 : 2;
+        const uint32_t t_p = t_lane + (uint32_t)((MT == 2) ? sub * 128 : col0);
         const int row = a0 + rl;                       // the key this thread sums for
         const float inv_r = (row < n) ? s_inv[row] : 0.f;
         const float thr = (row < n) ? __fdiv_rn(p.tau, inv_r) : INFINITY;   // Cm >= tau  <=>  G * inv_col >= tau / inv_row
         float sum = 0.f;
         bool ok = true;
-        for (int i = 0; i < T; ++i) {
-            const int buf = i & 1;
+        for (int i = parity; i < T; i += 2) {
+            const int buf = parity;
             ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (i >> 1) & 1, &tail->abort_flag));
             if (!ok) { rd_abort(tail, p.status, 35); break; }
             tmem_fence_after_sync();
@@ -266,9 +269,9 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
         }
         s_part[wg * 128 + L] = sum;
         epilogue_bar_sync();
-        if (ok && !*(volatile int*)&tail->abort_flag && ((MT == 2) ? (wg & 1) == 0 : wg == 0) && row < n) {
-            float tot;
-            if (MT == 2) tot = s_part[wg * 128 + L] + s_part[(wg + 1) * 128 + L];
+        if (!*(volatile int*)&tail->abort_flag && ((MT == 2) ? parity == 0 : wg == 0) && row < n) {
+            float tot;   // even-tile and odd-tile partials (and, with one row tile, the two column halves), fixed order
+            if (MT == 2) tot = s_part[sub * 128 + L] + s_part[(2 + sub) * 128 + L];
             else tot = (s_part[L] + s_part[128 + L]) + (s_part[256 + L] + s_part[384 + L]);
             p.cbar[(size_t)unit * p.C + row] = (row < n - p.recent) ? tot * inv_r : 0.f;   // recent tokens: column zeroed
         }
