@@ -154,9 +154,12 @@ gkv_status gkv_evict(gkv_ctx* ctx, int32_t layer, const void* q_window, int32_t*
                      void* stream);
 
 /* The stages of gkv_evict as separate launches, for timing them one by one. They communicate
- * through the workspace and must be called in order SCORE (only with q_window) -> MERGE ->
- * SELECT -> COMPACT on one layer (or -1); after COMPACT the state equals that after gkv_evict.
- * Results are identical to gkv_evict. Errors: as gkv_evict; STATE for an out-of-order stage. */
+ * through the workspace and must be called in order SCORE (only with q_window) -> REDUNDANCY (only
+ * with use_redundancy, then required) -> MERGE -> SELECT -> COMPACT on ONE layer (layer = -1 is
+ * UNSUPPORTED: the staged scratch holds one layer); after COMPACT the state equals that after
+ * gkv_evict. Results are identical to gkv_evict. kept_idx_out is taken by SELECT.
+ * Errors: as gkv_evict; STATE for an out-of-order stage; INVALID_ARG for an unknown stage, SCORE
+ * without q_window, or REDUNDANCY with the term off. */
 typedef enum { GKV_STAGE_SCORE = 0, GKV_STAGE_MERGE = 1, GKV_STAGE_SELECT = 2, GKV_STAGE_COMPACT = 3,
                GKV_STAGE_REDUNDANCY = 4 /* only with use_redundancy: after SCORE (if any), before MERGE */ } gkv_stage;
 gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const void* q_window,

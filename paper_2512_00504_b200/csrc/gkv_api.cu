@@ -437,7 +437,7 @@ gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const voi
                            void* stream) {
     int l0, nl;
     bool noop;
-    if (stage < GKV_STAGE_SCORE || stage > GKV_STAGE_REDUNDANCY) return GKV_ERR_INVALID_ARG;
+    if (!ctx || stage < GKV_STAGE_SCORE || stage > GKV_STAGE_REDUNDANCY) return GKV_ERR_INVALID_ARG;
     if (stage == GKV_STAGE_REDUNDANCY && !ctx->cfg.use_redundancy) return GKV_ERR_INVALID_ARG;
     gkv_status st = evict_precheck(ctx, layer, false, &l0, &nl, &noop);
     if (st != GKV_OK) return st;
