@@ -31,11 +31,11 @@ METRIC = "decode tok/s over the compressed cache incl. eviction (attention + evi
 UNIT = "tok/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
-# summarised in profiles/decode_kernel_cfg2.md: measured on a 4-layer stack (512 units) as 1.040 (plain
-# steps) and 1.029 (window steps) x the algorithmic bytes of the captured launches, i.e. 1.037 over a
+# summarised in profiles/decode_kernel_cfg2.md: measured on a 4-layer stack (512 units) as 1.011 (plain
+# steps) and 1.014 (window steps) x the algorithmic bytes of the captured launches, i.e. 1.012 over a
 # period, scaled to the full 3584-unit launch at the period's average length (traffic grows in
 # proportion to units). None where no capture exists.
-NCU_TRAFFIC_BYTES = {"cfg2": 1.037 * 2.022e9, "cfg1": None, "cfg4": None}
+NCU_TRAFFIC_BYTES = {"cfg2": 1.012 * 2.022e9, "cfg1": None, "cfg4": None}
 
 
 def workload_shape(name: str) -> dict:
@@ -420,6 +420,84 @@ def run_sweep(args) -> dict:
 
 
 # ------------------------------------------------------------------------------------------
+def run_perlayer(args) -> dict:
+    """Decode attention launched one layer at a time, the way a model calls it (7B head geometry, b = 1024, w = 32,
+    cache at 1064 tokens): the 28 per-layer launches of a step are captured in a CUDA graph and replayed, so the
+    figure is device time per launch without host issue overhead. Batch 1, 8, 32, 128; plain and window steps."""
+    import torch
+    import paper_2512_00504_b200 as gkv
+    from paper_2512_00504_b200 import synth
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    gkv.build_library()
+    base = {k: v for k, v in synth.CONFIGS[2].items() if k != "steps"}
+    peaks_path = ROOT / "MEASURED_PEAKS.json"
+    peak_gbs = float(json.loads(peaks_path.read_text())["hbm_gbs"]) if peaks_path.exists() else 6650.0
+    reps = max(3, args.steps)
+    cells, launches = [], 0
+    sampler = ClockSampler(0)
+    sampler.start()
+    for batch in (1, 8, 32, 128):
+        sh = dict(base, batch=batch)
+        L, B, Hq, H, d, b, w, s = (sh[k] for k in ("n_layers", "batch", "h_q", "h_kv", "d", "b", "w", "s"))
+        cache = gkv.GKVCache(gkv.make_config(**sh, fuse_window_scores=True), dev)
+        gen = torch.Generator(device=dev).manual_seed(synth.BASE_SEED + 11)
+        cache.k.copy_(torch.randn(cache.k.shape, generator=gen, device=dev).to(torch.bfloat16))
+        cache.v.copy_(torch.randn(cache.v.shape, generator=gen, device=dev).to(torch.bfloat16))
+        q = torch.randn((L, B, Hq, d), generator=gen, device=dev).to(torch.bfloat16)
+        kn = torch.randn((L, B, H, d), generator=gen, device=dev).to(torch.bfloat16)
+        vn = torch.randn((L, B, H, d), generator=gen, device=dev).to(torch.bfloat16)
+        out = torch.empty_like(q)
+        cell = {"batch": batch, "units_per_launch": B * H}
+        for name, since in (("plain", 40), ("window", s - w)):
+            n0 = b + since
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                cache.set_state(-1, n0, b - w, since)
+                for layer in range(L):                              # warm-up outside the capture
+                    cache.decode_attn(layer, q[layer], kn[layer], vn[layer], out[layer])
+                cache.set_state(-1, n0, b - w, since)
+                side.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for layer in range(L):
+                        cache.decode_attn(layer, q[layer], kn[layer], vn[layer], out[layer])
+            launches += 2 * L
+            ts = []
+            for _ in range(reps + 3):
+                cache.set_state(-1, n0, b - w, since)               # the replay advances the device lengths only
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); graph.replay(); e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1) / L)
+            launches += (reps + 3) * L
+            ms = sorted(ts[3:])[len(ts[3:]) // 2]
+            cell[name + "_us"] = ms * 1e3
+            cell[name + "_GBps"] = algorithmic_bytes(dict(sh, n_layers=1), n0 + 1, name == "window") / (ms * 1e-3) / 1e9
+        cache.poll()
+        cells.append(cell)
+        del cache, graph
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = cells[2]
+    L = base["n_layers"]
+    return {"metric": "decode tok/s with attention launched one layer at a time (28 launches per token step, attention only)",
+            "value": top["batch"] / (L * top["plain_us"] * 1e-6), "unit": "tok/s", "n_gpus": 1, "steps": reps, "warmup": 3,
+            "ms_per_step": L * top["plain_us"] * 1e-3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "per-layer decode launches: 28 layers, 28 q / 4 kv heads, d 128, b=1024, w=32, cache at 1064 "
+                                   "tokens; headline cell batch 32 (128 units per launch); step = the 28 launches of one token step",
+                       "l2": "the 28 layers' K+V (0.55 MB per unit) exceed L2 from batch 8 on; each launch reads its own layer"},
+            "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+            "roofline": {"kernel": "gkv_decode_kernel (key split)", "bound": "hbm", "achieved": top["plain_GBps"], "peak": peak_gbs,
+                         "unit": "GB/s", "frac": top["plain_GBps"] / peak_gbs, "traffic": None,
+                         "avg_launch_ms": top["plain_us"] * 1e-3},
+            "sweep": cells}
+
+
+# ------------------------------------------------------------------------------------------
 def run_prompt(args) -> dict:
     """First compression of a prefilled prompt (one layer of the 7B shape: batch 32, 28 q / 4 kv heads, b = 1024,
     w = 32) for prompt lengths 2048, 4096 and 8192: scoring of the prompt's window over all its keys, selection
@@ -557,7 +635,7 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "prompt"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "prompt", "perlayer"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiler captures only)")
     ap.add_argument("--ring", type=int, default=0, help="distinct per-step inputs kept on the device (0 = one period)")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -572,13 +650,15 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.workload in ("cfg3", "prompt"):
+        if args.workload in ("cfg3", "prompt", "perlayer"):
             args.workload = "cfg2"   # the oracle arm times the default workload only
         res = run_reference(args)
     elif args.workload == "cfg3":
         res = run_sweep(args)
     elif args.workload == "prompt":
         res = run_prompt(args)
+    elif args.workload == "perlayer":
+        res = run_perlayer(args)
     else:
         res = run_ours(args)
     if res is not None:
