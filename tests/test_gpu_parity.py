@@ -568,3 +568,20 @@ def test_host_buffer_entry_points_equal_the_device_calls(pinned):
     assert dev_c.state(0) == host_c.state(0) == (96, 88, 0)
     for c in caches:
         c.poll()
+
+
+def test_latched_device_status_is_reported_once():
+    """A kernel whose bounded wait expires latches a code in the status word at the start of the workspace. No wait
+    is made to expire here (that would need a broken copy); the latch is planted from the host instead, and the
+    poll must report it once and clear it."""
+    cfg = gkv.make_config(n_layers=1, batch=1, h_q=8, h_kv=2, b=96, buffer=32, w=8, s=32)
+    cache = gkv.GKVCache(cfg, DEV)
+    cache.poll()
+    cache.workspace[:16].view(torch.int32)[:3] = torch.tensor([1, 2, 77], dtype=torch.int32, device=DEV)   # code, where, block
+    with pytest.raises(gkv.GKVError) as e:
+        cache.poll()
+    assert e.value.status == gkv.GKV_ERR_TIMEOUT and "wait" in gkv.gkv_strerror(gkv.GKV_ERR_TIMEOUT)
+    cache.poll()                                                   # cleared by the first poll
+    x = torch.zeros((1, 8, 128), dtype=torch.bfloat16, device=DEV)
+    cache.decode_attn(0, x, x[:, :2].contiguous(), x[:, :2].contiguous(), x.clone())   # the context stays usable
+    cache.poll()
