@@ -237,17 +237,18 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
                 const float4* iv = reinterpret_cast<const float4*>(s_inv + i * kRdTileKeys + col0 + ch * 32);
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
                 if (i + 1 < T) {
+                    // per element one compare (1.0 / 0.0) and half a packed multiply and half a packed multiply-add: a
+                    // compare + select pair would put two instructions per element on the ALU pipe, which throttles first
+                    float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
                         const float4 c = iv[j >> 2];
-                        const float t0 = gacc[j] * c.x, t1 = gacc[j + 1] * c.y, t2 = gacc[j + 2] * c.z, t3 = gacc[j + 3] * c.w;
-                        // one compare (1.0 / 0.0) and one fused multiply-add per element: a compare + select pair would
-                        // put two instructions per element on the ALU pipe, which throttles first
-                        s0 = fmaf(t0, ge_mask(t0, thr), s0);
-                        s1 = fmaf(t1, ge_mask(t1, thr), s1);
-                        s2 = fmaf(t2, ge_mask(t2, thr), s2);
-                        s3 = fmaf(t3, ge_mask(t3, thr), s3);
+                        const float2 ta = mul_f32x2(make_float2(gacc[j], gacc[j + 1]), make_float2(c.x, c.y));
+                        const float2 tb = mul_f32x2(make_float2(gacc[j + 2], gacc[j + 3]), make_float2(c.z, c.w));
+                        sa = fma_f32x2(ta, make_float2(ge_mask(ta.x, thr), ge_mask(ta.y, thr)), sa);
+                        sb = fma_f32x2(tb, make_float2(ge_mask(tb.x, thr), ge_mask(tb.y, thr)), sb);
                     }
+                    s0 = sa.x; s1 = sa.y; s2 = sb.x; s3 = sb.y;
                 } else {
                     // last tile: columns past the end of the cache hold whatever the rows beyond it contain (possibly
                     // NaN or Inf bit patterns); their inverse norm is 0 and a select drops them whatever the product is
