@@ -585,3 +585,46 @@ def test_latched_device_status_is_reported_once():
     x = torch.zeros((1, 8, 128), dtype=torch.bfloat16, device=DEV)
     cache.decode_attn(0, x, x[:, :2].contiguous(), x[:, :2].contiguous(), x.clone())   # the context stays usable
     cache.poll()
+
+
+def test_config2_full_length_run_sampled():
+    """Configuration 2 end to end: 28 layers x batch 32, 16384 generated tokens from an empty cache with the drifting
+    synthetic stream (128 scheduled compressions, 120 of which evict). Sampled (layer, sequence) pairs are compared
+    with the oracle step-wise at a few compressions spread over the run, decode outputs are spot-checked, and the
+    schedule state is checked throughout."""
+    shape = {k: v for k, v in synth.CONFIGS[2].items() if k != "steps"}
+    steps = synth.CONFIGS[2]["steps"]
+    L, B, Hq, H, b, w, s = 28, 32, 28, 4, 1024, 32, 128
+    cfg = gkv.make_config(**shape, fuse_window_scores=True)
+    cache = gkv.GKVCache(cfg, DEV)
+    stream = synth.DecodeStream(synth.BASE_SEED + 2, n_layers=L, batch=B, h_q=Hq, h_kv=H, b=b, s=s, device=DEV)
+    out = torch.empty((L, B, Hq, 128), dtype=torch.bfloat16, device=DEV)
+    kept = torch.empty((L, B, H, b), dtype=torch.int32, device=DEV)
+    sample = [(0, 0), (11, 19), (27, 31)]
+    check_at = {8, 9, 40, 127}                                       # compression numbers (0-based) that are verified
+    real = 0
+    for t in range(steps):
+        q, kn, vn = stream.step()
+        cache.decode_attn(-1, q, kn, vn, out)
+        if t in (5, 1100, 9000, steps - 1):
+            n = cache.state(0)[0]
+            for layer, seq in sample[:2]:
+                ref = oracle.decode_attention(synth.bits(q[layer, seq]), synth.bits(cache.k[layer, seq]),
+                                              synth.bits(cache.v[layer, seq]), n)
+                assert np.abs(out[layer, seq].float().cpu().numpy() - ref).max() < DECODE_ATOL, t
+        if (t + 1) % s == 0:
+            c = (t + 1) // s - 1
+            l, n_h, since = cache.state(0)
+            assert since == s and l == min(b, (t + 1 - s)) + s if c >= 8 else l == t + 1
+            snaps = {ls: snapshot(cache, ls[0], [ls[1]]) for ls in sample} if c in check_at else None
+            cache.evict(-1, None, kept)
+            if l > b:
+                real += 1
+                if snaps is not None:
+                    for layer, seq in sample:
+                        check_evict_against_oracle(cache, layer, [seq], snaps[(layer, seq)],
+                                                   kept[layer, seq:seq + 1].cpu().numpy(), l=l, n_h=n_h)
+            assert cache.state(L - 1) == (min(l, b), b - w if l > b else 0, 0)
+    cache.poll()
+    assert real == 120
+    assert int(cache.len[0].min()) == int(cache.len[0].max()) == b and int(cache.len[1].min()) == b - w
