@@ -190,8 +190,8 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
  * keeps track of `len` itself (it is passed by value, nothing is read back).
  * The split-K partials, completion counters, length words and status word live in an array of about
  * 4.1 MiB that is part of the library's device image: every GPU that loads the library holds it until
- * the process exits. Limits: batch <= 1024, batch * n_kv_heads <= 1024, and (units x key splits) <=
- * 1024 CTAs; beyond them the call returns GKV_ERR_SCRATCH_LIMIT and launches nothing.
+ * the process exits. Limits: batch <= 1024 and batch * n_kv_heads <= 1024; beyond them the call returns
+ * GKV_ERR_SCRATCH_LIMIT and launches nothing. (Split-K is planned within the array's 1024 partial slots.)
  * All calls on a device share that array and it keeps the previous call's contents; each call clears
  * the words that must start at zero. Calls that overlap on the GPU (two streams, or unordered host
  * threads) race on the array and produce wrong results: keep them ordered.

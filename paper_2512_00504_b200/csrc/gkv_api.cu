@@ -44,9 +44,6 @@ gkv_status check_config(const gkv_config* c) {
     return GKV_OK;
 }
 
-// Split factor of a decode launch over `units` units; 148 SMs assumed when no device is known.
-int splits_for(int units, int C, int sm_count) { return decode_pick_splits(units, C, sm_count > 0 ? sm_count : 148); }
-
 void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     const uint64_t L = c->n_layers, B = c->batch, H = c->n_kv_heads;
     const uint64_t C = c->budget + c->buffer;
@@ -55,17 +52,20 @@ void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     w->status = off;    off = align_up(off + 64 * sizeof(int32_t));
     w->seq_done = off;  off = align_up(off + L * B * sizeof(int32_t));
     w->unit_done = off; off = align_up(off + L * upl * sizeof(int32_t));
-    // split-K scratch: sized for the larger of a one-layer launch and an all-layer launch
+    // split-K scratch of the decode kernel: the larger of a one-layer launch and an all-layer launch, plain or
+    // window step
     uint64_t part = 0, logits = 0;
-    const int cases[2] = {(int)upl, (int)(upl * L)};
-    for (int i = 0; i < 2; ++i) {
-        const int sp = splits_for(cases[i], (int)C, sm_count);
-        if (sp > 1) {
-            const uint64_t pb = (uint64_t)cases[i] * sp * (16 + kHeadDim * 8) * sizeof(float);
-            const uint64_t lb = (uint64_t)cases[i] * C * 8 * sizeof(float);
-            if (pb > part) part = pb;
-            if (lb > logits) logits = lb;
-        }
+    for (int i = 0; i < 4; ++i) {
+        DecodeLaunch d = {};
+        d.n_layers = (i & 1) ? (int)L : 1; d.batch = (int)B; d.h_kv = (int)H; d.C = (int)C;
+        d.accum = i >> 1;
+        d.sm_count = sm_count;
+        decode_plan(&d, 0);
+        const uint64_t split_units = d.splits > 1 ? (uint64_t)d.n_layers * upl : 0;
+        const uint64_t pb = split_units * d.splits * (16 + kHeadDim * 8) * sizeof(float);
+        const uint64_t lb = d.accum ? split_units * C * 8 * sizeof(float) : 0;
+        if (pb > part) part = pb;
+        if (lb > logits) logits = lb;
     }
     w->part = off;     off = align_up(off + part);
     w->logits = off;   off = align_up(off + logits);
@@ -383,8 +383,9 @@ gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const voi
     p.layer0 = l0; p.n_layers = nl; p.batch = c.batch; p.h_q = c.n_q_heads; p.h_kv = c.n_kv_heads;
     p.g = ctx->g; p.C = ctx->C;
     p.accum = (c.fuse_window_scores && ctx->since_evict[l0] >= c.interval - c.window) ? 1 : 0;
-    p.splits = decode_pick_splits(nl * ctx->units_per_layer, ctx->C, ctx->sm_count);
-    p.stages = decode_pick_stages(ctx->C, p.accum, p.splits, nullptr);
+    p.sm_count = ctx->sm_count;
+    p.work_next = p.status + 32;
+    decode_plan(&p, 0);
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
     const DecodeMaps maps = {ctx->tm_k, ctx->tm_v, ctx->tm_k16, ctx->tm_v16};
     if (launch_decode(p, maps, static_cast<cudaStream_t>(stream)) != cudaSuccess) {

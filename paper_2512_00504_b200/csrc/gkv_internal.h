@@ -44,9 +44,13 @@ struct DecodeLaunch {
     float* part;
     float* logits;
     int32_t* status;
+    int32_t* work_next;  // two zeroed words: the next item's number minus the grid size, and the CTAs that are done
     int layer0, n_layers, batch, h_q, h_kv, g, C;
-    int splits, stages, accum;
-    int tmem_cols;       // filled in by launch_decode
+    int accum;           // 1 on window steps
+    int sm_count;        // SMs of the device (sizes the persistent grid)
+    // filled in by decode_plan():
+    int splits;          // every unit is `splits` work items, each a contiguous share of the keys
+    int stages, grid, tmem_cols;
     float scale_log2;    // log2(e) / sqrt(d)
 };
 
@@ -135,7 +139,7 @@ struct gkv_ctx {
 namespace gkv {
 
 int decode_pick_splits(int units_in_launch, int C, int sm_count);
-int decode_pick_stages(int C, int accum, int splits, size_t* smem_bytes);
+void decode_plan(DecodeLaunch* p, int max_pieces);
 cudaError_t launch_decode(const DecodeLaunch& p, const DecodeMaps& maps, cudaStream_t s);
 cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s);
 cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s);

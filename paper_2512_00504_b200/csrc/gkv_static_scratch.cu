@@ -25,7 +25,7 @@ using namespace gkv;
 
 constexpr int kStaticMaxSeq = 1024;            // batch
 constexpr int kStaticMaxUnits = 1024;          // batch * n_kv_heads
-constexpr int kStaticMaxCtas = 1024;           // units * splits
+constexpr int kStaticMaxCtas = 1024;           // split-K pieces of a launch
 constexpr size_t kPartBytesPerCta = (16 + kHeadDim * 8) * sizeof(float);
 constexpr size_t kOffStatus = 0;                                   // int32[64]
 constexpr size_t kOffLen = 256;                                    // int32[kStaticMaxSeq]
@@ -113,8 +113,10 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
         return GKV_ERR_CUDA;
 
     DecodeLaunch p;
-    p.splits = decode_pick_splits((int)units, capacity, sm);
-    if (units * p.splits > kStaticMaxCtas) return GKV_ERR_SCRATCH_LIMIT;
+    p.n_layers = 1; p.batch = batch; p.h_kv = n_kv_heads; p.C = capacity;
+    p.accum = 0;
+    p.sm_count = sm;
+    decode_plan(&p, kStaticMaxCtas);   // at most that many split-K pieces
     DecodeMaps maps;
     const uint64_t rows = (uint64_t)units * capacity;
     if (!encode_rows(&maps.k64, k_cache, rows, kTileKeys) || !encode_rows(&maps.v64, v_cache, rows, kTileKeys) ||
@@ -142,10 +144,9 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     p.part = reinterpret_cast<float*>(scratch + kOffPart);
     p.logits = nullptr;
     p.status = reinterpret_cast<int32_t*>(scratch + kOffStatus);
+    p.work_next = p.status + 32;
     p.layer0 = 0; p.n_layers = 1; p.batch = batch; p.h_q = n_q_heads; p.h_kv = n_kv_heads;
     p.g = n_q_heads / n_kv_heads; p.C = capacity;
-    p.accum = 0;
-    p.stages = decode_pick_stages(capacity, 0, p.splits, nullptr);
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
     if (launch_decode(p, maps, s) != cudaSuccess) {
         (void)cudaGetLastError();

@@ -31,6 +31,8 @@ def load_case(cache, case, layer=0, window_scores=None):
     dict(batch=1, h_q=8, h_kv=2, b=160, buffer=40, w=8, s=40),      # split-K path, C = 200 (ragged tiles)
     dict(batch=2, h_q=28, h_kv=4, b=96, buffer=32, w=16, s=32),     # g = 7
     dict(batch=80, h_q=16, h_kv=4, b=130, buffer=30, w=8, s=30),    # 320 units: one CTA per unit, no split
+    # 528 units, more than the 3 x 148 CTAs of the persistent grid: CTAs take a second item from the work counter
+    dict(batch=66, h_q=16, h_kv=8, b=130, buffer=30, w=8, s=30),
 ])
 def test_decode_attention_matches_oracle(shape):
     cfg = gkv.make_config(n_layers=1, **shape, fuse_window_scores=False)
@@ -49,7 +51,7 @@ def test_decode_attention_matches_oracle(shape):
             q, kn, vn = rnd(B, Hq, 128), rnd(B, H, 128), rnd(B, H, 128)
             cache.decode_attn(0, q, kn, vn, out)
             K[:, :, t], V[:, :, t] = synth.bits(kn), synth.bits(vn)
-            sel = np.arange(B) if B <= 4 else np.array([0, 1, B // 2, B - 1])
+            sel = np.arange(B) if B <= 4 else np.array(sorted({0, 1, B // 2, (5 * B) // 6, B - 1}))
             ref = oracle.decode_batch(synth.bits(q)[sel], K[sel], V[sel], t + 1)
             got = out.float().cpu().numpy()[sel]
             assert np.abs(got - ref).max() < DECODE_ATOL, (start, t)
@@ -65,7 +67,8 @@ def test_decode_attention_matches_oracle(shape):
 
 @pytest.mark.parametrize("shape", [
     dict(batch=1, h_q=8, h_kv=2, b=150, buffer=50, w=16, s=50),     # split-K + window accumulation
-    dict(batch=75, h_q=28, h_kv=4, b=100, buffer=40, w=8, s=40),    # 300 units, shared-memory logits
+    dict(batch=75, h_q=28, h_kv=4, b=100, buffer=40, w=8, s=40),    # 300 units, logits in tensor memory
+    dict(batch=66, h_q=16, h_kv=8, b=100, buffer=40, w=8, s=40),    # 528 units: more items than resident CTAs
 ])
 def test_window_accumulation_matches_recomputed_local_score(shape):
     """Fused window sums from w decode steps vs Eq. 1-2 recomputed by the oracle from the stored
@@ -87,7 +90,7 @@ def test_window_accumulation_matches_recomputed_local_score(shape):
         qs.append(q)
     assert cache.state(0) == (C, 0, s)
     q_win = torch.stack(qs, dim=2).contiguous()           # [B][Hq][w][d], oldest first
-    sel = list(range(B)) if B <= 4 else [0, B // 2, B - 1]
+    sel = list(range(B)) if B <= 4 else sorted({0, B // 2, (5 * B) // 6, B - 1})
     K = synth.bits(cache.k[0])
     sacc = cache.sacc[0].cpu().numpy()
     for n in sel:
