@@ -32,10 +32,10 @@ UNIT = "tok/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture
 # summarised in profiles/decode_kernel_cfg2.md: measured on a 4-layer stack (512 units) as 1.012 (plain
-# steps) and 1.014 (window steps) x the algorithmic bytes of the captured launches, i.e. 1.012 over a
+# steps) and 1.015 (window steps) x the algorithmic bytes of the captured launches, i.e. 1.013 over a
 # period, scaled to the full 3584-unit launch at the period's average length (traffic grows in
 # proportion to units). None where no capture exists.
-NCU_TRAFFIC_BYTES = {"cfg2": 1.012 * 2.022e9, "cfg1": None, "cfg4": None}
+NCU_TRAFFIC_BYTES = {"cfg2": 1.013 * 2.022e9, "cfg1": None, "cfg4": None}
 
 
 def workload_shape(name: str) -> dict:

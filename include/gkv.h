@@ -129,9 +129,9 @@ gkv_status gkv_set_state(gkv_ctx* ctx, int32_t layer, int32_t len, int32_t n_his
  * included); len += 1. With fuse_window_scores, the last w steps before a scheduled compression
  * also add max over the group of the final attention weights to sacc (this token's row of the
  * group max that Eq. 2 averages). layer = -1 runs all layers in one launch with every tensor
- * argument carrying a leading [n_layers] dimension.
+ * argument carrying a leading [n_layers] dimension. q, k_new, v_new and out are 16-byte aligned.
  * Errors: CAPACITY (len == C, nothing launched); STATE (fuse_window_scores and a compression is
- * due: since_evict == interval); INVALID_ARG; CUDA. */
+ * due: since_evict == interval); INVALID_ARG (NULL or misaligned pointer, bad layer); CUDA. */
 gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const void* k_new,
                            const void* v_new, void* out, void* stream);
 

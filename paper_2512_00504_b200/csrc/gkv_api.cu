@@ -359,6 +359,10 @@ gkv_status gkv_set_state(gkv_ctx* ctx, int32_t layer, int32_t len, int32_t n_his
 gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const void* k_new, const void* v_new,
                            void* out, void* stream) {
     if (!ctx || !layer_ok(ctx, layer) || !q || !k_new || !v_new || !out) return GKV_ERR_INVALID_ARG;
+    // 16-byte vector accesses and, for q, bulk copies
+    if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
+         reinterpret_cast<uintptr_t>(out)) % 16 != 0)
+        return GKV_ERR_INVALID_ARG;
     int l0, nl;
     layer_range(ctx, layer, &l0, &nl);
     if (!uniform(ctx->len, l0, nl) || !uniform(ctx->since_evict, l0, nl)) return GKV_ERR_STATE;

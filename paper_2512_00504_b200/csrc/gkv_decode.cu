@@ -21,7 +21,6 @@ constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 constexpr int kMaxStages = 6;
 constexpr int kPartFloats = 16 + kHeadDim * 8;  // M[8], L[8], acc[128][8]
-constexpr int kQRowBytes = 272;                 // 256 bytes of a query row + 16 of padding
 
 struct __align__(16) DecodeSmemTail {
     uint64_t full_bar[kMaxStages];
@@ -31,15 +30,20 @@ struct __align__(16) DecodeSmemTail {
     float fin_m[8];
     float fin_l[8];
     float wgt[kConsumerWarps][8];
-    // One scratch slot with three lives per item: the group's query rows (272 bytes apart) while the fragments are
-    // loaded, then the cross-warp merge of the output accumulators (64 dims x 8 heads fp32 at a time; with key split
-    // the splits' statistics and weights), then the bf16 output rows on their way out.
-    alignas(16) uint8_t scratch[3072];
+    uint64_t q_full;    // the item's query rows have landed in q_rows (one bulk copy by the producer lane)
+    uint64_t q_empty;   // the four consumer warps have the item's query fragments in registers
+    // The group's g query rows, contiguous as in global memory, and the current token's k and v rows.
+    alignas(16) uint8_t q_rows[8 * 256];
+    alignas(16) uint8_t new_rows[2 * 256];
+    // Scratch slot of the per-item epilogue: the cross-warp merge of the output accumulators (64 dims x 8 heads fp32
+    // at a time; with key split the splits' statistics and weights), then the bf16 output rows on their way out.
+    alignas(16) uint8_t scratch[8 * 256];
     int item_ids[8];   // work items in the order the producer took them (a ring: the producer is < 8 items ahead)
     int cur_item;      // the item the consumers are on, or -1: no more
     int abort_flag;
     int abort_seen;   // the abort flag as consumer thread 0 saw it between two barriers of the epilogue
     int issued;
+    int q_issued;     // bulk copies of query rows started (the last one may be in flight at an abort)
     int is_last;
     uint32_t tmem_base;
 };
@@ -120,6 +124,9 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
             mbar_init(smem_u32(&tail->full_bar[s]), 1);
             mbar_init(smem_u32(&tail->empty_bar[s]), kConsumerWarps);
         }
+        mbar_init(smem_u32(&tail->q_full), 1);
+        mbar_init(smem_u32(&tail->q_empty), kConsumerWarps);
+        tail->q_issued = 0;
         tail->abort_flag = 0;
         tail->abort_seen = 0;
         tail->cur_item = -1;
@@ -157,6 +164,27 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                 DecodeItem d;
                 if (more) {
                     d = decode_item(p, item);
+                    // The group's query rows, one bulk copy, started the moment the item is known: about two tiles
+                    // before the consumers get to it, so the rows' latency -- microseconds when q is mapped host
+                    // memory and the bus is busy -- is over by then. The buffer is free once the consumers have
+                    // the previous item's fragments in registers, which they take at the start of an item.
+                    if (k > 0 && !decode_wait(smem_u32(&tail->q_empty), (k - 1) & 1, &tail->abort_flag)) {
+                        if (!*(volatile int*)&tail->abort_flag) latch_timeout(p.status, 4);
+                        tail->abort_flag = 1;
+                        break;
+                    }
+                    const uint32_t qbar = smem_u32(&tail->q_full);
+                    const bool appends = d.len_old / kTileKeys >= d.t_begin && d.len_old / kTileKeys < d.t_end;
+                    mbar_arrive_expect_tx(qbar, (uint32_t)p.g * 256u + (appends ? 512u : 0u));
+                    bulk_load(smem_u32(tail->q_rows),
+                              p.q + ((size_t)(d.layer_local * p.batch + d.seq) * p.h_q + (size_t)d.head * p.g) * kHeadDim,
+                              (uint32_t)p.g * 256u, qbar);
+                    if (appends) {   // this item holds the tile that the current token's row goes into
+                        const size_t src = ((size_t)(d.layer_local * p.batch + d.seq) * p.h_kv + d.head) * kHeadDim;
+                        bulk_load(smem_u32(tail->new_rows), p.k_new + src, 256u, qbar);
+                        bulk_load(smem_u32(tail->new_rows + 256), p.v_new + src, 256u, qbar);
+                    }
+                    *(volatile int*)&tail->q_issued = k + 1;
                 } else {
                     d.t_begin = d.t_end = 0; d.slot_end = 1; d.n = 0; d.row0 = 0;
                 }
@@ -219,9 +247,17 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
             // where the previous item's use of the scratch slot, the statistics and the window sums has ended.
             if (tid == 0) {
                 int next = -1;
+                bool timed_out = false;
                 if (decode_wait(smem_u32(&tail->full_bar[s]), round & 1, &tail->abort_flag)) {
                     next = *(volatile int*)&tail->item_ids[k & 7];
+                    if (next >= 0 && !decode_wait(smem_u32(&tail->q_full), k & 1, &tail->abort_flag)) {
+                        next = -1;
+                        timed_out = true;
+                    }
                 } else {
+                    timed_out = true;
+                }
+                if (timed_out) {
                     if (!*(volatile int*)&tail->abort_flag) latch_timeout(p.status, 3);
                     tail->abort_flag = 1;
                 }
@@ -233,38 +269,27 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
             const DecodeItem d = decode_item(p, item);
             const int n = d.n, len_old = d.len_old;
 
-            // The group's g query rows come in once per item with 16-byte loads (warp w fetches heads w and w + 4,
-            // one row per half warp) and are re-read from shared memory in fragment order: one bus or L2 transaction
-            // per 16 bytes instead of four copies of it in 4-byte pieces. Rows are 272 bytes apart: conflict-free.
+            // The group's g query rows are in q_rows (thread 0 has seen the copy complete; the wait below passes at
+            // once and makes the copied bytes visible to this thread). Fragment order: B[k = d][n = head].
             uint32_t qf[8][2];
-            {
-                const int hl = warp + (lane >> 4) * kConsumerWarps;          // head this half warp fetches
-                if (hl < p.g) {
-                    const __nv_bfloat16* qrow =
-                        p.q + ((size_t)(d.layer_local * p.batch + d.seq) * p.h_q + (size_t)d.head * p.g + hl) * kHeadDim;
-                    *reinterpret_cast<uint4*>(tail->scratch + hl * kQRowBytes + (lane & 15) * 16) =
-                        *reinterpret_cast<const uint4*>(qrow + (lane & 15) * 8);
-                }
-                consumer_bar_sync();
+            (void)decode_wait(smem_u32(&tail->q_full), k & 1, &tail->abort_flag);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    if (hq < p.g) {
-                        const uint8_t* row = tail->scratch + hq * kQRowBytes + ks * 32 + (lane & 3) * 4;
-                        qf[ks][0] = *reinterpret_cast<const uint32_t*>(row);
-                        qf[ks][1] = *reinterpret_cast<const uint32_t*>(row + 16);
-                    } else {
-                        qf[ks][0] = qf[ks][1] = 0u;
-                    }
+            for (int ks = 0; ks < 8; ++ks) {
+                if (hq < p.g) {
+                    const uint8_t* row = tail->q_rows + hq * 256 + ks * 32 + (lane & 3) * 4;
+                    qf[ks][0] = *reinterpret_cast<const uint32_t*>(row);
+                    qf[ks][1] = *reinterpret_cast<const uint32_t*>(row + 16);
+                } else {
+                    qf[ks][0] = qf[ks][1] = 0u;
                 }
             }
-            // The current token's row lands in the last tile; the warp that will append it fetches its 16 bytes per
-            // lane now (lanes 0-15 of k_new, 16-31 of v_new), so that the load's latency -- a bus round trip when the
-            // inputs are mapped host memory -- is long over when the row is needed.
+            // The current token's row lands in the last tile; the warp that will append it takes its 16 bytes per lane
+            // now (lanes 0-15 of the k row, 16-31 of the v row).
             uint4 new_row = make_uint4(0u, 0u, 0u, 0u);
-            if (warp == ((len_old & (kTileKeys - 1)) >> 4) && (len_old / kTileKeys) >= d.t_begin && (len_old / kTileKeys) < d.t_end) {
-                const size_t src = ((size_t)(d.layer_local * p.batch + d.seq) * p.h_kv + d.head) * kHeadDim + (lane & 15) * 8;
-                new_row = *reinterpret_cast<const uint4*>((lane < 16 ? p.k_new : p.v_new) + src);
-            }
+            if (warp == ((len_old & (kTileKeys - 1)) >> 4) && (len_old / kTileKeys) >= d.t_begin && (len_old / kTileKeys) < d.t_end)
+                new_row = *reinterpret_cast<const uint4*>(tail->new_rows + (lane >> 4) * 256 + (lane & 15) * 16);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tail->q_empty));
             // Window steps: the unit's current window sums start their way into shared memory now and are needed only
             // in the epilogue; the updated sums go back with plain coalesced stores. (One atomic per key is measurably
             // slower: the L2 atomic units saturate at ~4 M reductions a launch.)
@@ -465,8 +490,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                     // of the splits' accumulators.
                     __threadfence();
                     const float* base = p.part + (size_t)d.unit_local * p.splits * kPartFloats;
-                    float* s_stat = reinterpret_cast<float*>(tail->scratch);   // [splits <= 32][16]: M[8], L[8]
-                    float* s_w = s_stat + 32 * 16;                              // [splits][8] weights
+                    float* s_stat = reinterpret_cast<float*>(tail->scratch);   // [splits <= 32][16]: M[8] (then the weights), L[8]
                     for (int idx = tid; idx < p.splits * 16; idx += kConsumerThreads)
                         s_stat[idx] = __ldcg(base + (size_t)(idx >> 4) * kPartFloats + (idx & 15));
                     consumer_bar_sync();
@@ -478,7 +502,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                         for (int sp = 0; sp < p.splits; ++sp) {
                             const float wm = s_stat[sp * 16 + h];
                             const float wgt = (wm == -INFINITY) ? 0.f : fast_exp2(wm - mm);
-                            s_w[sp * 8 + h] = wgt;
+                            s_stat[sp * 16 + h] = wgt;   // over the maximum it came from: only this thread reads that word
                             ll += wgt * s_stat[sp * 16 + 8 + h];
                         }
                         tail->fin_m[h] = mm;
@@ -491,8 +515,8 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                     for (int sp = 0; sp < p.splits; ++sp) {
                         const float4* a4 = reinterpret_cast<const float4*>(base + (size_t)sp * kPartFloats + 16 + tid * 8);
                         const float4 a = __ldcg(a4), b = __ldcg(a4 + 1);
-                        const float4 wa = *reinterpret_cast<const float4*>(s_w + sp * 8);
-                        const float4 wb = *reinterpret_cast<const float4*>(s_w + sp * 8 + 4);
+                        const float4 wa = *reinterpret_cast<const float4*>(s_stat + sp * 16);
+                        const float4 wb = *reinterpret_cast<const float4*>(s_stat + sp * 16 + 4);
                         o[0] = fmaf(wa.x, a.x, o[0]); o[1] = fmaf(wa.y, a.y, o[1]); o[2] = fmaf(wa.z, a.z, o[2]); o[3] = fmaf(wa.w, a.w, o[3]);
                         o[4] = fmaf(wb.x, b.x, o[4]); o[5] = fmaf(wb.y, b.y, o[5]); o[6] = fmaf(wb.z, b.z, o[6]); o[7] = fmaf(wb.w, b.w, o[7]);
                     }
@@ -506,12 +530,12 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
 #pragma unroll
                 for (int h = 0; h < 8; ++h)
                     if (h < p.g)
-                        *reinterpret_cast<__nv_bfloat16*>(tail->scratch + h * kQRowBytes + tid * 2) = __float2bfloat16_rn(o[h] / tail->fin_l[h]);
+                        *reinterpret_cast<__nv_bfloat16*>(tail->scratch + h * 256 + tid * 2) = __float2bfloat16_rn(o[h] / tail->fin_l[h]);
                 consumer_bar_sync();
                 if (tid < p.g * 16) {
                     const int h = tid >> 4, c = tid & 15;
                     __nv_bfloat16* orow = p.out + ((size_t)(d.layer_local * p.batch + d.seq) * p.h_q + (size_t)d.head * p.g + h) * kHeadDim;
-                    *reinterpret_cast<uint4*>(orow + c * 8) = *reinterpret_cast<const uint4*>(tail->scratch + h * kQRowBytes + c * 16);
+                    *reinterpret_cast<uint4*>(orow + c * 8) = *reinterpret_cast<const uint4*>(tail->scratch + h * 256 + c * 16);
                 }
                 if (ACCUM != 0) {
                     // Sacc[t] += max over the group of the final weights = exp2(max_h (z_h[t] - M_h - log2 L_h)).
@@ -577,6 +601,8 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
         const int issued = *(volatile int*)&tail->issued;
         for (int j = max(0, issued - stages); j < issued; ++j)
             mbar_wait_bounded(smem_u32(&tail->full_bar[j % stages]), (j / stages) & 1);
+        const int q_issued = *(volatile int*)&tail->q_issued;
+        if (q_issued > 0) mbar_wait_bounded(smem_u32(&tail->q_full), (q_issued - 1) & 1);
     }
     if (ACCUM == 1) cp_async_wait_all();
     __syncthreads();

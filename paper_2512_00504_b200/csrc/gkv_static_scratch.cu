@@ -99,7 +99,9 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     if (batch <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || capacity <= 0 || len < 0) return GKV_ERR_INVALID_ARG;
     if (n_q_heads % n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
     if (n_q_heads / n_kv_heads > kMaxGroup || capacity > 4096) return GKV_ERR_UNSUPPORTED;
-    if ((reinterpret_cast<uintptr_t>(k_cache) | reinterpret_cast<uintptr_t>(v_cache)) % 16 != 0) return GKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(k_cache) | reinterpret_cast<uintptr_t>(v_cache) | reinterpret_cast<uintptr_t>(q) |
+         reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(out)) % 16 != 0)
+        return GKV_ERR_INVALID_ARG;
     if (len >= capacity) return GKV_ERR_CAPACITY;
     const long units = (long)batch * n_kv_heads;
     if (batch > kStaticMaxSeq || units > kStaticMaxUnits) return GKV_ERR_SCRATCH_LIMIT;
