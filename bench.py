@@ -500,8 +500,8 @@ def run_perlayer(args) -> dict:
 # ------------------------------------------------------------------------------------------
 def run_prompt(args) -> dict:
     """First compression of a prefilled prompt (one layer of the 7B shape: batch 32, 28 q / 4 kv heads, b = 1024,
-    w = 32) for prompt lengths 2048, 4096 and 8192: scoring of the prompt's window over all its keys, selection
-    and gather into the cache. The JSON line carries the longest prompt; `sweep` every length."""
+    w = 32) for prompt lengths 2048, 4096, 8192 and 32768: scoring of the prompt's window over all its keys,
+    selection and gather into the cache. The JSON line carries the longest prompt; `sweep` every length."""
     import torch
     import paper_2512_00504_b200 as gkv
     from paper_2512_00504_b200 import synth
@@ -519,7 +519,7 @@ def run_prompt(args) -> dict:
     cells, launches = [], 0
     sampler = ClockSampler(0)
     sampler.start()
-    for P in (2048, 4096, 8192):
+    for P in (2048, 4096, 8192, 32768):
         cfg = gkv.make_config(**sh, fuse_window_scores=True, max_prompt=P)
         cache = gkv.GKVCache(cfg, dev)
         gen = torch.Generator(device=dev).manual_seed(synth.BASE_SEED + 9)
@@ -553,7 +553,7 @@ def run_prompt(args) -> dict:
             "data": "synthetic",
             "config": {"workload": f"prompt compression: 1 layer, batch {B}, {Hq} q / {H} kv heads, d 128, b={b}, w={w}, "
                                    f"prompt {top['prompt_len']} tokens per sequence; step = scoring + selection + gather",
-                       "l2": "the prompt's K (268 MB at 8192 tokens) exceeds L2"},
+                       "l2": "the prompt's K (268 MB at 8192 tokens, 1.07 GB at 32768) exceeds L2"},
             "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
             "roofline": {"kernel": "gkv_score_tc_kernel + gkv_prompt_compress_kernel", "bound": "hbm", "achieved": top["GBps"],
                          "peak": peak_gbs, "unit": "GB/s", "frac": top["GBps"] / peak_gbs, "traffic": None,

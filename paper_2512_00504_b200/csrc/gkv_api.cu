@@ -14,7 +14,8 @@ using namespace gkv;
 namespace {
 
 constexpr int kMaxCapacity = 4096;
-constexpr int kMaxPrompt = 8192;   // longest prompt gkv_compress_prompt takes (its scores stay in shared memory)
+constexpr int kMaxPromptShared = 8192;   // up to here a prompt's scores stay in shared memory during the selection
+constexpr int kMaxPrompt = 65536;        // longest prompt gkv_compress_prompt takes (16-bit counts in the selection's scan)
 constexpr uint64_t kAlign = 256;
 
 uint64_t align_up(uint64_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -30,6 +31,11 @@ gkv_status check_config(const gkv_config* c) {
     if (c->n_q_heads % c->n_kv_heads != 0) return GKV_ERR_INVALID_ARG;
     if (c->max_prompt < 0) return GKV_ERR_INVALID_ARG;
     if (c->max_prompt > kMaxPrompt) return GKV_ERR_UNSUPPORTED;
+    // beyond the cache sizes only the tensor-core scoring kernel passes its window sums through in chunks
+    if (c->max_prompt > kMaxPromptShared && c->n_kv_heads > 0 &&
+        score_tc_rows_per_cta(c->n_q_heads / c->n_kv_heads, c->window) == 0)
+        return GKV_ERR_UNSUPPORTED;
+    if ((uint64_t)c->batch * c->n_kv_heads * (uint64_t)c->max_prompt >= (1ull << 31)) return GKV_ERR_UNSUPPORTED;
     if (c->pool_kernel < 0 || (c->pool_kernel > 1 && (c->pool_kernel & 1) == 0)) return GKV_ERR_INVALID_ARG;
     if (c->use_redundancy) {
         if (!(c->redundancy_lambda >= 0.f && c->redundancy_lambda <= 1.f)) return GKV_ERR_INVALID_ARG;
@@ -74,6 +80,8 @@ void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     const uint64_t red = c->use_redundancy ? 1 : 0;   // the redundancy term's scratch exists only when it is on
     w->prompt_sums = off; off = align_up(off + upl * (uint64_t)c->max_prompt * sizeof(float));
     w->prompt_len = off;  off = align_up(off + (c->max_prompt > 0 ? B : 0) * sizeof(int32_t));
+    const uint64_t long_arrays = c->max_prompt > kMaxPromptShared ? (c->pool_kernel > 1 ? 2 : 1) : 0;
+    w->prompt_f = off;    off = align_up(off + long_arrays * upl * (uint64_t)c->max_prompt * sizeof(float));
     const uint64_t sel = (c->use_redundancy || c->pool_kernel > 1) ? 1 : 0;
     w->fsel = off;     off = align_up(off + sel * upl * C * sizeof(float));
     w->inv_norm = off; off = align_up(off + red * L * upl * C * sizeof(float));
@@ -195,6 +203,8 @@ gkv_status dispatch_score(gkv_ctx* ctx, const ScoreLaunch& sp, const CUtensorMap
         const uint64_t q_rows = (uint64_t)sp.n_layers * c.batch * c.n_q_heads * c.window;
         if (encode_map(&tm_q, const_cast<__nv_bfloat16*>(sp.q_win), q_rows, (uint32_t)wk) != GKV_OK) return GKV_ERR_CUDA;
         if (launch_score_tc(sp, tm_k, tm_q, wk, s) != cudaSuccess) return GKV_ERR_CUDA;
+    } else if (sp.C > kMaxPromptShared) {
+        return GKV_ERR_INVALID_ARG;   // a long prompt with misaligned window queries: the other kernel holds all sums on chip
     } else if (launch_score(sp, tm_k, s) != cudaSuccess) {
         return GKV_ERR_CUDA;
     }
@@ -616,6 +626,7 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
     p.pos = static_cast<int32_t*>(ctx->buf.pos);
     p.len = static_cast<int32_t*>(ctx->buf.len);
     p.sums = sums;
+    p.f_long = c.max_prompt > kMaxPromptShared ? ws_ptr<float>(ctx, ctx->ws.prompt_f) : nullptr;
     p.prompt_len = d_len;
     p.seq_done = ws_ptr<int32_t>(ctx, ctx->ws.seq_done);
     p.kept_out = kept_idx_out;

@@ -388,11 +388,16 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const Ev
 __global__ void __launch_bounds__(kEvictThreads) gkv_prompt_compress_kernel(const PromptLaunch p, int ring_offset) {
     extern __shared__ __align__(128) uint8_t evict_smem[];
     EvictShared* sh = reinterpret_cast<EvictShared*>(evict_smem);
-    float* s_f = reinterpret_cast<float*>(evict_smem + sizeof(EvictShared));   // [P_max]
-    float* s_sel = (p.pool_kernel > 1) ? s_f + p.P_max : s_f;                  // [P_max] pooled scores
-    int* s_kept = reinterpret_cast<int*>(s_f + ((p.pool_kernel > 1) ? 2 : 1) * p.P_max);   // [b]
     const int tid = threadIdx.x;
     const int unit_local = blockIdx.x;
+    // The unit's scores [P_max] (and the pooled ones) live in shared memory, or, for prompts too long for it, in the
+    // workspace: the phases below only need a pointer, and a CTA-wide barrier orders global accesses as well.
+    const int n_arrays = (p.pool_kernel > 1) ? 2 : 1;
+    float* s_f = p.f_long ? p.f_long + (size_t)unit_local * n_arrays * p.P_max
+                          : reinterpret_cast<float*>(evict_smem + sizeof(EvictShared));
+    float* s_sel = (p.pool_kernel > 1) ? s_f + p.P_max : s_f;                  // [P_max] pooled scores
+    int* s_kept = p.f_long ? reinterpret_cast<int*>(evict_smem + sizeof(EvictShared))
+                           : reinterpret_cast<int*>(s_f + n_arrays * p.P_max);   // [b]
     const int seq = unit_local / p.h_kv;
     const int lseq_global = p.layer * p.batch + seq;
     const long unit = (long)lseq_global * p.h_kv + (unit_local - seq * p.h_kv);
@@ -527,7 +532,8 @@ cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s) {
     return cudaGetLastError();
 }
 cudaError_t launch_prompt_compress(const PromptLaunch& p, cudaStream_t s) {
-    const size_t state = sizeof(EvictShared) + sizeof(float) * p.P_max * ((p.pool_kernel > 1) ? 2 : 1) + sizeof(int) * p.b;
+    const size_t scores = p.f_long ? 0 : sizeof(float) * p.P_max * ((p.pool_kernel > 1) ? 2 : 1);
+    const size_t state = sizeof(EvictShared) + scores + sizeof(int) * p.b;
     const size_t ring = (state + 127) & ~size_t(127);
     const size_t smem = ring + kCopyRingBytes;
     cudaError_t e = ensure_smem((const void*)gkv_prompt_compress_kernel, smem);

@@ -24,6 +24,7 @@ struct WorkspaceLayout {
     uint64_t fscratch;    // fp32[units_per_layer * C]    merged scores of the staged eviction path
     uint64_t prompt_sums; // fp32[units_per_layer * max_prompt]  window sums of a prompt being compressed
     uint64_t prompt_len;  // int32[batch]                        device copy of the prompt lengths
+    uint64_t prompt_f;    // fp32[(1 or 2) * units_per_layer * max_prompt]  scores of long prompts (max_prompt > 8192)
     uint64_t fsel;        // fp32[units_per_layer * C]    selection scores of the staged path (redundancy term on)
     uint64_t inv_norm;    // fp32[L * units_per_layer * C] 1 / (|K row| + eps)            (redundancy term on)
     uint64_t cbar;        // fp32[L * units_per_layer * C] redundancy level of every row  (redundancy term on)
@@ -94,6 +95,8 @@ struct PromptLaunch {
     int32_t* pos;                // may be NULL
     int32_t* len;                // plane 0; plane 1 follows at len + L_total*batch
     const float* sums;           // [batch*h_kv][P_max] w * S of the prompt's window
+    float* f_long;               // NULL, or [batch*h_kv][P_max] (pooling: twice that): the scores of a prompt too long
+                                 // for shared memory are kept here
     const int32_t* prompt_len;   // device [batch]
     int32_t* seq_done;
     int32_t* kept_out;           // may be NULL: [batch*h_kv][b], -1 padded

@@ -32,6 +32,7 @@ constexpr int kTcMaxRows = 256;
 constexpr int kTcQBytes = kTcMaxRows * kRowBytes;            // 64 KB: d-low half (32 KB) then d-high half
 constexpr int kTcAccCols = 256;                              // TMEM columns of one accumulator
 constexpr uint32_t kTcTmemCols = 512;
+constexpr int kTcChunkKeys = 8192;                           // keys whose window sums are held in shared memory at a time
 
 struct __align__(8) ScoreTcTail {
     uint64_t q_full;
@@ -40,6 +41,7 @@ struct __align__(8) ScoreTcTail {
     uint64_t d_full[2];
     uint64_t d_empty[2];
     uint64_t drain;
+    uint64_t chunk_bar;   // the softmax warps meet here when the window sums move on to the next chunk of keys
     uint32_t tmem_base;
     int abort_flag;
     int issued;
@@ -70,10 +72,12 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
     float* s_c = reinterpret_cast<float*>(k_smem + stages * kTcKStageBytes);      // [256] m + log2 l of every local row
     float* s_pm = s_c + kTcMaxRows;                                               // [groups][128] partial row maxima
     float* s_pl = s_pm + kTcGroups * 128;                                         // [groups][128] partial row sums
-    // [2][C] window sums of this CTA's rows: two groups add into each plane, so every sum has two addends and
-    // the result does not depend on the order in which the groups arrive
+    // [2][c_pad] window sums of this CTA's rows: two groups add into each plane, so every sum has two addends and
+    // the result does not depend on the order in which the groups arrive. Caches hold at most kTcChunkKeys rows and
+    // fit whole; a longer key range (a prompt being compressed) passes through in chunks of kTcChunkKeys keys, each
+    // written out when pass 2, which walks the tiles from the last to the first, leaves it.
     float* s_sum = s_pl + kTcGroups * 128;
-    const int c_pad = (p.C + 63) & ~63;
+    const int c_pad = min((p.C + 63) & ~63, kTcChunkKeys);
     ScoreTcTail* tail = reinterpret_cast<ScoreTcTail*>(s_sum + 2 * c_pad);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -99,6 +103,7 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
             mbar_init(smem_u32(&tail->d_empty[b]), kTcSoftmaxThreads / 32);   // one arrival per softmax warp
         }
         mbar_init(smem_u32(&tail->drain), 1);
+        mbar_init(smem_u32(&tail->chunk_bar), kTcSoftmaxThreads / 32);
         tail->abort_flag = 0;
         tail->issued = 0;
         fence_mbar_init();
@@ -276,8 +281,37 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
         softmax_bar_sync();
 
         // ---- pass 2: this thread owns key `tile * 128 + L`; group wg covers window rows k0 + wg*HW .. + HW - 1
+        float* out = p.sacc + (size_t)unit * p.C;
+        // window sums of keys [lo, lo + c_pad) leave shared memory (which is zeroed for the next chunk)
+        auto flush_chunk = [&](int lo) {
+            const int hi = min(lo + c_pad, p.C);
+            for (int t = lo + stid; t < hi; t += kTcSoftmaxThreads) {
+                const float v = s_sum[t - lo] + s_sum[c_pad + t - lo];
+                s_sum[t - lo] = 0.f;
+                s_sum[c_pad + t - lo] = 0.f;
+                if (n_cta == 1) out[t] = (t < n) ? v : 0.f;
+                else if (t < n) atomicAdd(&out[t], v);   // buffer zeroed by the host
+            }
+        };
+        uint32_t chunk_phase = 0;
+        int chunk_lo = T > 0 ? ((T - 1) * kTcTileKeys / c_pad) * c_pad : 0;
         for (int i = T; i < total; ++i) {
             const int buf = i & 1;
+            const int tile_lo = ((total - 1 - i) * kTcTileKeys / c_pad) * c_pad;
+            if (tile_lo != chunk_lo) {
+                // Every softmax warp has added its part of the chunk; then the chunk is written and cleared; then all
+                // go on. mbarrier waits, not bar.sync: a warp that gives up (abort flag) must not leave the others at
+                // a barrier it will never reach.
+                for (int step = 0; ok && step < 2; ++step) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&tail->chunk_bar));
+                    ok = __all_sync(0xffffffffu, tc_wait(smem_u32(&tail->chunk_bar), chunk_phase & 1, &tail->abort_flag));
+                    ++chunk_phase;
+                    if (ok && step == 0) flush_chunk(chunk_lo);
+                }
+                if (!ok) { tc_abort(tail, p.status, 27); break; }
+                chunk_lo = tile_lo;
+            }
             ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (i >> 1) & 1, &tail->abort_flag));
             if (!ok) { tc_abort(tail, p.status, 26); break; }
             tmem_fence_after_sync();
@@ -309,17 +343,15 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                     s0 += (j >= first_k) ? fast_exp2(v[j]) : 0.f;
                     s1 += (j + 1 >= first_k) ? fast_exp2(v[j + 1]) : 0.f;
                 }
-                atomicAdd(&s_sum[(wg >> 1) * c_pad + key], s0 + s1);
+                atomicAdd(&s_sum[(wg >> 1) * c_pad + key - chunk_lo], s0 + s1);
             }
         }
         softmax_bar_sync();
         if (ok && !*(volatile int*)&tail->abort_flag) {
-            float* out = p.sacc + (size_t)unit * p.C;
-            if (n_cta == 1) {
-                for (int t = stid; t < p.C; t += kTcSoftmaxThreads) out[t] = (t < n) ? s_sum[t] + s_sum[c_pad + t] : 0.f;
-            } else {
-                for (int t = stid; t < n; t += kTcSoftmaxThreads) atomicAdd(&out[t], s_sum[t] + s_sum[c_pad + t]);   // buffer zeroed by the host
-            }
+            flush_chunk(chunk_lo);   // the chunk of the first tile, walked last
+            // rows past the chunk that holds the last key were never in shared memory
+            if (n_cta == 1)
+                for (int t = (T > 0 ? ((T - 1) * kTcTileKeys / c_pad + 1) * c_pad : 0) + stid; t < p.C; t += kTcSoftmaxThreads) out[t] = 0.f;
         }
     }
 
@@ -341,7 +373,7 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
 static size_t score_tc_smem_bytes(int C, int rows, int stages) {
     (void)rows;
     return 1024 + (size_t)kTcQBytes + (size_t)stages * kTcKStageBytes +
-           sizeof(float) * (kTcMaxRows + 2 * kTcGroups * 128 + 2 * ((C + 63) & ~63)) + sizeof(ScoreTcTail);
+           sizeof(float) * (kTcMaxRows + 2 * kTcGroups * 128 + 2 * min((C + 63) & ~63, kTcChunkKeys)) + sizeof(ScoreTcTail);
 }
 
 // Window rows per CTA for this shape, or 0 when the shape is left to the mma.sync kernel.

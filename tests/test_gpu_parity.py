@@ -261,6 +261,15 @@ def test_evict_noop_and_state_errors():
     with pytest.raises(gkv.GKVError) as e:
         cache.decode_attn(-1, x, x[:, :, :2].contiguous(), x[:, :, :2].contiguous(), x.clone())
     assert e.value.status == gkv.GKV_ERR_STATE
+    cache.set_state(-1, 100, 0, 5)
+    flat = torch.zeros(x.numel() + 8, dtype=torch.bfloat16, device=DEV)
+    q_off = flat[1: 1 + x.numel()].view(x.shape)              # 2 bytes off a 16-byte boundary: rejected, nothing launched
+    kn = x[:, :, :2].contiguous()
+    for args in ((q_off, kn, kn, x.clone()), (x, kn, kn, q_off)):
+        with pytest.raises(gkv.GKVError) as e:
+            cache.decode_attn(-1, *args)
+        assert e.value.status == gkv.GKV_ERR_INVALID_ARG
+    assert cache.state(0) == (100, 0, 5)
     cache.poll()
 
 

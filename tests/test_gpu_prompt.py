@@ -112,6 +112,47 @@ def test_prompt_compression_and_ragged_loop(w, h_q, h_kv, pool):
             check_evict_against_oracle(cache, layer, [n], one, kept2[n:n + 1], l=cur[n], n_h=nh[n])
 
 
+@pytest.mark.parametrize("w,h_q,h_kv,pool,lens", [
+    (16, 8, 2, 0, [20000, 9000, 300, 8193]),     # one CTA per unit scores all window rows; 3, 2 and 2 chunks of 8192 keys
+    (64, 28, 4, 5, [12288, 8200, 100]),          # the window split over two CTAs per unit (sums meet in global memory), pooling
+])
+def test_long_prompt_compression(w, h_q, h_kv, pool, lens):
+    """Prompts longer than 8192 tokens: their window sums pass through the scoring kernel's shared memory in chunks and
+    their scores stay in the workspace during the selection. Same checks as for short prompts."""
+    b, buffer, s = 512, 64, 64
+    P_max = max(lens)
+    B = len(lens)
+    cfg = gkv.make_config(n_layers=1, batch=B, h_q=h_q, h_kv=h_kv, b=b, buffer=buffer, w=w, s=s, fuse_window_scores=True,
+                          track_positions=True, max_prompt=P_max, pool_kernel=pool)
+    cache = gkv.GKVCache(cfg, DEV)
+    kp, vp, qw = make_prompt(synth.BASE_SEED + 90 + w, B, h_q, h_kv, w, P_max, lens)
+    kept = torch.full((B, h_kv, b), -7, dtype=torch.int32, device=DEV)
+    cache.compress_prompt(0, kp, vp, qw, lens, kept)
+    cache.poll()
+    kept = kept.cpu().numpy()
+    Kp, Vp = synth.bits(kp), synth.bits(vp)
+    K_c, V_c = synth.bits(cache.k[0]), synth.bits(cache.v[0])
+    F_c, pos_c = cache.f[0].cpu().numpy(), cache.pos[0].cpu().numpy()
+    dev_len, dev_nh = cache.len[0, 0].cpu().numpy(), cache.len[1, 0].cpu().numpy()
+    for n in range(B):
+        P = lens[n]
+        if P <= b:
+            assert dev_len[n] == P and dev_nh[n] == 0
+            assert (K_c[n, :, :P] == Kp[n, :, :P]).all() and (kept[n, :, :P] == np.arange(P)).all()
+            continue
+        assert dev_len[n] == b and dev_nh[n] == b - w
+        ref = oracle.evict_step_full(synth.bits(qw[n]), None, Kp[n], Vp[n], None, np.zeros((h_kv, P_max), np.float32),
+                                     l=P, n_h=0, b=b, w=w, alpha=0.8, mode=oracle.MODE_MAX, pool_kernel=max(pool, 1))
+        for j in range(h_kv):
+            assert_kept_matches(kept[n, j], ref["Fsel"][j], b, w, f"seq {n} head {j}")
+            k = kept[n, j]
+            assert (np.diff(k) > 0).all() and (k[b - w:] == np.arange(P - w, P)).all()
+            assert (K_c[n, j, :b] == Kp[n, j, k]).all() and (V_c[n, j, :b] == Vp[n, j, k]).all()
+            assert (pos_c[n, j, :b] == k).all()
+            np.testing.assert_allclose(F_c[n, j, : b - w], ref["F"][j, k[: b - w]], rtol=SCORE_RTOL, atol=SCORE_ATOL)
+    assert cache.state(0) == (b, b - w, 0) and float(cache.sacc[0].abs().max()) == 0.0
+
+
 def test_prompt_call_errors():
     cfg = gkv.make_config(n_layers=1, batch=2, h_q=8, h_kv=2, b=64, buffer=16, w=8, s=16)
     cache = gkv.GKVCache(cfg, DEV)
@@ -125,6 +166,12 @@ def test_prompt_call_errors():
         with pytest.raises(gkv.GKVError) as e:
             cache.compress_prompt(0, x, x, q, lens)
         assert e.value.status == gkv.GKV_ERR_INVALID_ARG
+    for bad in (dict(max_prompt=65537), dict(max_prompt=9000, w=8)):   # too long; long prompts need a window of 16 k rows
+        kw = dict(n_layers=1, batch=2, h_q=8, h_kv=2, b=64, buffer=16, w=16, s=16)
+        kw.update(bad)
+        with pytest.raises(gkv.GKVError) as e:
+            gkv.GKVCache(gkv.make_config(**kw), DEV)
+        assert e.value.status == gkv.GKV_ERR_UNSUPPORTED
     cache.compress_prompt(0, x, x, None, [10, 64])                 # no prompt longer than b: no queries needed
     cache.poll()
     assert cache.state(0) == (64, 0, 0) and cache.len[0, 0].cpu().numpy().tolist() == [10, 64]
