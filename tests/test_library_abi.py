@@ -55,6 +55,9 @@ def base(**over):
     (dict(d=64), gkv.GKV_ERR_UNSUPPORTED),
     (dict(h_q=32), gkv.GKV_ERR_UNSUPPORTED),         # g = 16 > 8
     (dict(b=4000, buffer=200, s=128), gkv.GKV_ERR_UNSUPPORTED),
+    (dict(max_prompt=65537), gkv.GKV_ERR_UNSUPPORTED),          # longest prompt the first compression takes
+    (dict(max_prompt=9000, w=24), gkv.GKV_ERR_UNSUPPORTED),     # above 8192 tokens the window is a multiple of 16
+    (dict(max_prompt=-1), gkv.GKV_ERR_INVALID_ARG),
 ])
 def test_config_validation(over, status):
     with pytest.raises(gkv.GKVError) as e:
@@ -77,6 +80,21 @@ def test_query_sizes_layout():
     # the 32B-shaped stress configuration keeps ~77 GB of K+V resident
     huge = gkv.gkv_query_sizes(gkv.make_config(n_layers=64, batch=128, h_q=64, h_kv=8, b=2048, buffer=256, w=64, s=256))
     assert abs((huge.k + huge.v) / 1e9 - 77.3) < 0.1
+
+
+def test_workspace_grows_with_the_prompt_limit():
+    """The workspace holds the window sums of a prompt being compressed (4 bytes per token and KV head) and, above
+    8192 tokens, the prompt's scores as well (once more, twice with pooling): then they no longer fit a CTA's shared
+    memory."""
+    upl = 3 * 2
+    w0 = gkv.gkv_query_sizes(base()).workspace
+    w8 = gkv.gkv_query_sizes(base(max_prompt=8192)).workspace
+    w64 = gkv.gkv_query_sizes(base(max_prompt=65536)).workspace
+    w64p = gkv.gkv_query_sizes(base(max_prompt=65536, pool_kernel=5)).workspace
+    near = lambda got, want: abs(got - want) <= 4096            # 256-byte alignment of a few regions
+    assert near(w8 - w0, upl * 8192 * 4)
+    assert near(w64 - w0, 2 * upl * 65536 * 4)
+    assert w64p - w64 >= upl * 65536 * 4                       # pooled scores (+ the cache-sized selection scratch)
 
 
 def test_memory_model_reproduces_the_papers_appendix():
