@@ -96,8 +96,8 @@ typedef struct {
      * gives no kernel size and reports that pooling does not help at decode time. */
     int32_t pool_kernel;
     /* Longest prompt gkv_compress_prompt will be given (rows per head of its K / V buffers); 0 = that call is
-     * not used. At most 65536; above 8192 the window must be a multiple of 16 (UNSUPPORTED otherwise) and q_window
-     * 16-byte aligned. Sizes part of the workspace (4 bytes per prompt token and KV head, twice or three times
+     * not used. At most 65536; above 8192 the window must be a multiple of 16 and use_redundancy off (UNSUPPORTED
+     * otherwise) and q_window 16-byte aligned. Sizes part of the workspace (4 bytes per prompt token and KV head, twice or three times
      * that above 8192). */
     int32_t max_prompt;
 } gkv_config;
@@ -214,8 +214,8 @@ gkv_status gkv_decode_attn_static(const void* q, const void* k_new, const void* 
  * q_window: device, [batch][n_q_heads][w][128], the queries of each prompt's last w tokens, oldest first
  * (may be NULL when no prompt is longer than b). Per sequence and KV head: a prompt of at most b tokens is
  * copied whole into cache rows 0..len-1 (n_hist = 0); a longer one keeps the top-(b-w) of its first
- * len - w tokens by the max-normalised window score (Eq. 1-2, after the optional pooling; the redundancy
- * term is not applied to prompts) plus the last w tokens, in ascending position, in rows 0..b-1, with F of
+ * len - w tokens by the max-normalised window score (Eq. 1-2, after the optional pooling and, with
+ * use_redundancy, the redundancy term over the prompt's keys) plus the last w tokens, in ascending position, in rows 0..b-1, with F of
  * the kept rows recorded and pos = position in the prompt (with track_positions). sacc of the layer is
  * cleared, since_evict = 0. kept_idx_out (optional, device [batch][n_kv_heads][b]) receives the kept
  * prompt positions, -1 padded. One layer per call (prefill proceeds layer by layer).

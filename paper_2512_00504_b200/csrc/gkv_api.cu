@@ -36,6 +36,8 @@ gkv_status check_config(const gkv_config* c) {
         score_tc_rows_per_cta(c->n_q_heads / c->n_kv_heads, c->window) == 0)
         return GKV_ERR_UNSUPPORTED;
     if ((uint64_t)c->batch * c->n_kv_heads * (uint64_t)c->max_prompt >= (1ull << 31)) return GKV_ERR_UNSUPPORTED;
+    // the redundancy kernel keeps a unit's inverse key norms in shared memory
+    if (c->use_redundancy && c->max_prompt > kMaxPromptShared) return GKV_ERR_UNSUPPORTED;
     if (c->pool_kernel < 0 || (c->pool_kernel > 1 && (c->pool_kernel & 1) == 0)) return GKV_ERR_INVALID_ARG;
     if (c->use_redundancy) {
         if (!(c->redundancy_lambda >= 0.f && c->redundancy_lambda <= 1.f)) return GKV_ERR_INVALID_ARG;
@@ -84,8 +86,10 @@ void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     w->prompt_f = off;    off = align_up(off + long_arrays * upl * (uint64_t)c->max_prompt * sizeof(float));
     const uint64_t sel = (c->use_redundancy || c->pool_kernel > 1) ? 1 : 0;
     w->fsel = off;     off = align_up(off + sel * upl * C * sizeof(float));
-    w->inv_norm = off; off = align_up(off + red * L * upl * C * sizeof(float));
-    w->cbar = off;     off = align_up(off + red * L * upl * C * sizeof(float));
+    // per cached row of every layer, or per token of a prompt being compressed, whichever is more
+    const uint64_t red_rows = L * upl * C > upl * (uint64_t)c->max_prompt ? L * upl * C : upl * (uint64_t)c->max_prompt;
+    w->inv_norm = off; off = align_up(off + red * red_rows * sizeof(float));
+    w->cbar = off;     off = align_up(off + red * red_rows * sizeof(float));
     w->total = off;
 }
 
@@ -615,6 +619,23 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
             (void)cudaGetLastError();
             return st;
         }
+        if (c.use_redundancy) {
+            // redundancy level of every prompt key, in the scratch the cached layers' levels use as well
+            RedundancyLaunch rp;
+            rp.k_cache = static_cast<const __nv_bfloat16*>(k_prompt);
+            rp.len = d_len;
+            rp.inv_norm = ws_ptr<float>(ctx, ctx->ws.inv_norm);
+            rp.cbar = ws_ptr<float>(ctx, ctx->ws.cbar);
+            rp.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
+            rp.layer0 = 0; rp.n_layers = 1; rp.batch = c.batch; rp.h_kv = c.n_kv_heads; rp.C = c.max_prompt;
+            rp.recent = c.redundancy_recent; rp.tau = c.redundancy_threshold; rp.eps = c.redundancy_eps;
+            if (launch_keynorm(rp, s) != cudaSuccess || launch_redundancy(rp, tm_kp, s) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return GKV_ERR_CUDA;
+            }
+            ctx->launches += 2;
+            for (int i = 0; i < c.n_layers; ++i) ctx->cbar_valid[i] = 0;
+        }
     }
     PromptLaunch p;
     p.k_src = static_cast<const __nv_bfloat16*>(k_prompt);
@@ -627,6 +648,8 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
     p.len = static_cast<int32_t*>(ctx->buf.len);
     p.sums = sums;
     p.f_long = c.max_prompt > kMaxPromptShared ? ws_ptr<float>(ctx, ctx->ws.prompt_f) : nullptr;
+    p.cbar = (c.use_redundancy && any_long) ? ws_ptr<float>(ctx, ctx->ws.cbar) : nullptr;
+    p.lambda = c.redundancy_lambda;
     p.prompt_len = d_len;
     p.seq_done = ws_ptr<int32_t>(ctx, ctx->ws.seq_done);
     p.kept_out = kept_idx_out;
@@ -712,7 +735,7 @@ const char* gkv_strerror(gkv_status status) {
         case GKV_ERR_CAPACITY: return "cache full: evict before decoding further";
         case GKV_ERR_CUDA: return "CUDA call failed";
         case GKV_ERR_TIMEOUT: return "a bounded device-side wait expired";
-        case GKV_ERR_UNSUPPORTED: return "configuration not supported by this build";
+        case GKV_ERR_UNSUPPORTED: return "configuration not supported by this library";
         case GKV_ERR_SCRATCH_LIMIT: return "problem exceeds the library's built-in scratch array";
         default: return "unknown status";
     }

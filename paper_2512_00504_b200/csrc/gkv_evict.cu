@@ -392,10 +392,10 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_prompt_compress_kernel(cons
     const int unit_local = blockIdx.x;
     // The unit's scores [P_max] (and the pooled ones) live in shared memory, or, for prompts too long for it, in the
     // workspace: the phases below only need a pointer, and a CTA-wide barrier orders global accesses as well.
-    const int n_arrays = (p.pool_kernel > 1) ? 2 : 1;
+    const int n_arrays = (p.pool_kernel > 1 || p.cbar) ? 2 : 1;
     float* s_f = p.f_long ? p.f_long + (size_t)unit_local * n_arrays * p.P_max
                           : reinterpret_cast<float*>(evict_smem + sizeof(EvictShared));
-    float* s_sel = (p.pool_kernel > 1) ? s_f + p.P_max : s_f;                  // [P_max] pooled scores
+    float* s_sel = (n_arrays == 2) ? s_f + p.P_max : s_f;                      // [P_max] the scores the selection runs on
     int* s_kept = p.f_long ? reinterpret_cast<int*>(evict_smem + sizeof(EvictShared))
                            : reinterpret_cast<int*>(s_f + n_arrays * p.P_max);   // [b]
     const int seq = unit_local / p.h_kv;
@@ -409,6 +409,8 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_prompt_compress_kernel(cons
         const int n_c = n - p.w;
         merge_phase(p.sums + (size_t)unit_local * p.P_max, nullptr, s_f, n_c, 0, 0.f, GKV_MODE_LOCAL, sh, tid);
         if (p.pool_kernel > 1) pool_phase(s_f, s_sel, n_c, p.pool_kernel, tid);
+        if (p.cbar)
+            combine_phase(p.cbar + (size_t)unit_local * p.P_max, (p.pool_kernel > 1) ? s_sel : s_f, s_sel, n, n_c, p.lambda, sh, tid);
         select_phase(s_sel, s_kept, nullptr, n_c, n_keep, p.w, sh, tid);
     } else {
         for (int r = tid; r < n; r += kEvictThreads) s_kept[r] = r;
@@ -532,7 +534,7 @@ cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s) {
     return cudaGetLastError();
 }
 cudaError_t launch_prompt_compress(const PromptLaunch& p, cudaStream_t s) {
-    const size_t scores = p.f_long ? 0 : sizeof(float) * p.P_max * ((p.pool_kernel > 1) ? 2 : 1);
+    const size_t scores = p.f_long ? 0 : sizeof(float) * p.P_max * ((p.pool_kernel > 1 || p.cbar) ? 2 : 1);
     const size_t state = sizeof(EvictShared) + scores + sizeof(int) * p.b;
     const size_t ring = (state + 127) & ~size_t(127);
     const size_t smem = ring + kCopyRingBytes;

@@ -95,6 +95,8 @@ struct PromptLaunch {
     int32_t* pos;                // may be NULL
     int32_t* len;                // plane 0; plane 1 follows at len + L_total*batch
     const float* sums;           // [batch*h_kv][P_max] w * S of the prompt's window
+    const float* cbar;           // NULL, or [batch*h_kv][P_max] redundancy level of the prompt's keys
+    float lambda;                // weight of the score against the redundancy term
     float* f_long;               // NULL, or [batch*h_kv][P_max] (pooling: twice that): the scores of a prompt too long
                                  // for shared memory are kept here
     const int32_t* prompt_len;   // device [batch]

@@ -153,6 +153,46 @@ def test_long_prompt_compression(w, h_q, h_kv, pool, lens):
     assert cache.state(0) == (b, b - w, 0) and float(cache.sacc[0].abs().max()) == 0.0
 
 
+@pytest.mark.parametrize("pool", [0, 5])
+def test_prompt_compression_with_redundancy_term(pool):
+    """With use_redundancy the first compression selects on lambda * F - (1 - lambda) * R' like every later one; the
+    redundancy level comes from the prompt's own keys (cosine similarities above the threshold, the most recent
+    columns zeroed). The heavy hitters of the synthetic prompt share a direction, so they are mutually redundant."""
+    w, h_q, h_kv, b, buffer, s, P_max = 16, 8, 2, 256, 32, 32, 1500
+    lam, tau, recent = 0.7, 0.3, 16
+    lens = [1500, 200, 777]
+    B = len(lens)
+    cfg = gkv.make_config(n_layers=1, batch=B, h_q=h_q, h_kv=h_kv, b=b, buffer=buffer, w=w, s=s, fuse_window_scores=True,
+                          track_positions=True, max_prompt=P_max, pool_kernel=pool, redundancy_lambda=lam,
+                          redundancy_threshold=tau, redundancy_recent=recent)
+    cache = gkv.GKVCache(cfg, DEV)
+    kp, vp, qw = make_prompt(synth.BASE_SEED + 120 + pool, B, h_q, h_kv, w, P_max, lens)
+    kept = torch.full((B, h_kv, b), -7, dtype=torch.int32, device=DEV)
+    cache.compress_prompt(0, kp, vp, qw, lens, kept)
+    cache.poll()
+    kept = kept.cpu().numpy()
+    Kp, Vp = synth.bits(kp), synth.bits(vp)
+    K_c, F_c = synth.bits(cache.k[0]), cache.f[0].cpu().numpy()
+    differs = 0
+    for n in range(B):
+        P = lens[n]
+        if P <= b:
+            assert (kept[n, :, :P] == np.arange(P)).all() and (K_c[n, :, :P] == Kp[n, :, :P]).all()
+            continue
+        args = (synth.bits(qw[n]), None, Kp[n], Vp[n], None, np.zeros((h_kv, P_max), np.float32))
+        kw = dict(l=P, n_h=0, b=b, w=w, alpha=0.8, mode=oracle.MODE_MAX, pool_kernel=max(pool, 1))
+        ref = oracle.evict_step_full(*args, **kw, lam=lam, tau=tau, recent=recent, eps=1e-6)
+        plain = oracle.evict_step_full(*args, **kw)
+        for j in range(h_kv):
+            assert_kept_matches(kept[n, j], ref["Fsel"][j], b, w, f"seq {n} head {j}")
+            k = kept[n, j]
+            assert (K_c[n, j, :b] == Kp[n, j, k]).all()
+            # what is recorded is F itself, not the score the selection ran on
+            np.testing.assert_allclose(F_c[n, j, : b - w], ref["F"][j, k[: b - w]], rtol=SCORE_RTOL, atol=SCORE_ATOL)
+            differs += int(set(ref["kept"][j].tolist()) != set(plain["kept"][j].tolist()))
+    assert differs > 0            # the term changed at least one head's selection: the case exercises it
+
+
 def test_prompt_call_errors():
     cfg = gkv.make_config(n_layers=1, batch=2, h_q=8, h_kv=2, b=64, buffer=16, w=8, s=16)
     cache = gkv.GKVCache(cfg, DEV)
