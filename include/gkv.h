@@ -255,7 +255,10 @@ gkv_status gkv_get_state(const gkv_ctx* ctx, int32_t layer, int32_t* len, int32_
 int64_t gkv_launch_count(const gkv_ctx* ctx);
 
 /* Synchronises `stream` and returns GKV_ERR_TIMEOUT if any kernel latched an expired bounded
- * wait since the last poll (the latch is then cleared), GKV_ERR_CUDA on a CUDA error, else OK. */
+ * wait since the last poll, GKV_ERR_CUDA on a CUDA error, else OK. On TIMEOUT the latch and the
+ * kernels' completion and work counters in the workspace are cleared, so the context can be used
+ * again; what the kernel that gave up had written (outputs, cache rows, lengths) is undefined:
+ * declare the state anew with gkv_set_state before going on. */
 gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream);
 
 /* Memory model of the paper's appendix "Memory Analysis": bytes of the full KV cache at

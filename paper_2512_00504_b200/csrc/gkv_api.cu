@@ -707,7 +707,9 @@ gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream) {
     if (cudaMemcpyAsync(h, d, sizeof h, cudaMemcpyDeviceToHost, s) != cudaSuccess) return GKV_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return GKV_ERR_CUDA;
     if (h[0] != 0) {
-        if (cudaMemsetAsync(d, 0, sizeof h, s) != cudaSuccess) return GKV_ERR_CUDA;
+        // A kernel that gave up may have left its completion and work counters part-way (they are returned to zero
+        // by the last CTA of a launch that runs to its end): clear them together with the latch.
+        if (cudaMemsetAsync(d, 0, ctx->ws.part - ctx->ws.status, s) != cudaSuccess) return GKV_ERR_CUDA;
         return GKV_ERR_TIMEOUT;
     }
     return GKV_OK;

@@ -589,14 +589,22 @@ def test_latched_device_status_is_reported_once():
     cfg = gkv.make_config(n_layers=1, batch=1, h_q=8, h_kv=2, b=96, buffer=32, w=8, s=32)
     cache = gkv.GKVCache(cfg, DEV)
     cache.poll()
-    cache.workspace[:16].view(torch.int32)[:3] = torch.tensor([1, 2, 77], dtype=torch.int32, device=DEV)   # code, where, block
+    words = cache.workspace[:256].view(torch.int32)
+    words[:3] = torch.tensor([1, 2, 77], dtype=torch.int32, device=DEV)   # code, where, block
+    words[32:34] = torch.tensor([5, 1], dtype=torch.int32, device=DEV)    # a work counter left part-way by that kernel
     with pytest.raises(gkv.GKVError) as e:
         cache.poll()
     assert e.value.status == gkv.GKV_ERR_TIMEOUT and "wait" in gkv.gkv_strerror(gkv.GKV_ERR_TIMEOUT)
     cache.poll()                                                   # cleared by the first poll
-    x = torch.zeros((1, 8, 128), dtype=torch.bfloat16, device=DEV)
-    cache.decode_attn(0, x, x[:, :2].contiguous(), x[:, :2].contiguous(), x.clone())   # the context stays usable
+    assert int(words[:64].abs().max()) == 0                        # and the counters with it
+    # the context stays usable: a decode step after the poll gives the single cached token's value row
+    gen = torch.Generator(device=DEV).manual_seed(3)
+    x = torch.randn((1, 8, 128), generator=gen, device=DEV).to(torch.bfloat16)
+    kn, vn = x[:, :2].contiguous(), x[:, 2:4].contiguous()
+    out = torch.empty_like(x)
+    cache.decode_attn(0, x, kn, vn, out)
     cache.poll()
+    assert torch.equal(out.view(1, 2, 4, 128), vn.view(1, 2, 1, 128).expand(1, 2, 4, 128))
 
 
 def test_config2_full_length_run_sampled():
