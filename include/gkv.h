@@ -190,10 +190,10 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
  * all bf16. Semantics are those of gkv_decode_attn without window-score accumulation: k_new, v_new are
  * written to row `len` of every head's cache and out is the attention over rows 0..len; the caller
  * keeps track of `len` itself (it is passed by value, nothing is read back).
- * The split-K partials, completion counters, length words and status word live in an array of about
- * 4.1 MiB that is part of the library's device image: every GPU that loads the library holds it until
- * the process exits. Limits: batch <= 1024 and batch * n_kv_heads <= 1024; beyond them the call returns
- * GKV_ERR_SCRATCH_LIMIT and launches nothing. (Split-K is planned within the array's 1024 partial slots.)
+ * The length words, completion and work counters and the status word live in an array of 8.25 KiB
+ * that is part of the library's device image: every GPU that loads the library holds it until the
+ * process exits. Limit: batch <= 1024 (one length word and one counter per sequence); beyond it the
+ * call returns GKV_ERR_SCRATCH_LIMIT and launches nothing.
  * All calls on a device share that array and it keeps the previous call's contents; each call clears
  * the words that must start at zero. Calls that overlap on the GPU (two streams, or unordered host
  * threads) race on the array and produce wrong results: keep them ordered.

@@ -32,6 +32,7 @@ struct __align__(16) DecodeSmemTail {
     float wgt[kConsumerWarps][8];
     uint64_t q_full;    // the item's query rows have landed in q_rows (one bulk copy by the producer lane)
     uint64_t q_empty;   // the four consumer warps have the item's query fragments in registers
+    uint64_t cl_bar;    // key split: the other CTAs of the cluster arrive here when their partial results are in rx
     // The group's g query rows, contiguous as in global memory, and the current token's k and v rows.
     alignas(16) uint8_t q_rows[8 * 256];
     alignas(16) uint8_t new_rows[2 * 256];
@@ -126,6 +127,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
         }
         mbar_init(smem_u32(&tail->q_full), 1);
         mbar_init(smem_u32(&tail->q_empty), kConsumerWarps);
+        if (p.splits > 1) mbar_init(smem_u32(&tail->cl_bar), (uint32_t)p.splits - 1);
         tail->q_issued = 0;
         tail->abort_flag = 0;
         tail->abort_seen = 0;
@@ -140,6 +142,9 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
         tmem_fence_before_sync();
     }
     __syncthreads();
+    // Key split: the CTAs of a unit form a cluster (launched so); none may reach into another's shared memory or
+    // barriers before all have initialised theirs.
+    if (p.splits > 1) cluster_sync_all();
     if (use_tmem) tmem_fence_after_sync();
     const uint32_t tmem_warp = use_tmem ? (*(volatile uint32_t*)&tail->tmem_base + ((uint32_t)(warp & 3) << 21)) : 0u;
 
@@ -227,7 +232,8 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                     if (++s == stages) { s = 0; ++round; }
                 }
                 if (!more) break;
-                item = (int)gridDim.x + atomicAdd(p.work_next, 1);
+                // a split launch has one CTA per item (the cluster's ranks are the unit's pieces)
+                item = (p.splits > 1) ? total_items : (int)gridDim.x + atomicAdd(p.work_next, 1);
             }
         }
     } else {
@@ -469,30 +475,45 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
 
             bool do_final = true;          // this CTA writes the output (always true without split)
             if (p.splits > 1) {
-                float* mine = p.part + ((size_t)d.unit_local * p.splits + d.split) * kPartFloats;
-                if (tid < 8) { mine[tid] = tail->fin_m[tid]; mine[8 + tid] = tail->fin_l[tid]; }
-                float4* d4 = reinterpret_cast<float4*>(mine + 16 + tid * 8);
-                d4[0] = make_float4(o[0], o[1], o[2], o[3]);
-                d4[1] = make_float4(o[4], o[5], o[6], o[7]);
-                __threadfence();
-                consumer_bar_sync();
-                if (tid == 0) {
-                    const int prev = atomicAdd(&p.unit_done[d.unit], 1);
-                    tail->is_last = (prev == p.splits - 1);
-                    if (prev == p.splits - 1) p.unit_done[d.unit] = 0;   // self-reset for the next launch
+                // The pieces of a unit are the CTAs of one cluster. Every CTA stores its (max, sum) per head and its
+                // accumulators into slot `rank` of the receive buffer in the shared memory of the cluster's first CTA
+                // (distributed shared memory: no trip through L2, no completion counter in global memory), then
+                // arrives on that CTA's mbarrier and is done. The first CTA waits for the others and merges.
+                float* rx = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(tail) + sizeof(DecodeSmemTail));   // [splits][kPartFloats]
+                const uint32_t slot = cluster_map_shared(smem_u32(rx + (size_t)d.split * kPartFloats), 0);
+                if (tid < 8) {
+                    st_cluster_f32(slot + 4u * tid, tail->fin_m[tid]);
+                    st_cluster_f32(slot + 4u * (8 + tid), tail->fin_l[tid]);
                 }
+                st_cluster_f32x4(slot + 4u * (16 + tid * 8), o[0], o[1], o[2], o[3]);
+                st_cluster_f32x4(slot + 4u * (16 + tid * 8 + 4), o[4], o[5], o[6], o[7]);
+                fence_acq_rel_cluster();
                 consumer_bar_sync();
-                do_final = tail->is_last != 0;
-                if (do_final) {
-                    // The last CTA of the unit merges the partials. All loads of a phase are independent, so the merge
-                    // costs a few L2 round trips, not one per split: (1) every split's (max, sum) into shared memory,
-                    // (2) per head the global max, the splits' weights and the global sum, (3) per dim the weighted sum
-                    // of the splits' accumulators.
-                    __threadfence();
-                    const float* base = p.part + (size_t)d.unit_local * p.splits * kPartFloats;
-                    float* s_stat = reinterpret_cast<float*>(tail->scratch);   // [splits <= 32][16]: M[8] (then the weights), L[8]
+                do_final = d.split == 0;
+                if (!do_final) {
+                    if (tid == 0) mbar_arrive_cluster(cluster_map_shared(smem_u32(&tail->cl_bar), 0));
+                } else {
+                    if (tid == 0) {
+                        bool ok = false;
+                        for (uint32_t i = 0; i < kWaitSpins && !ok; ++i) {
+                            ok = mbar_try_wait_cluster(smem_u32(&tail->cl_bar), 0);
+                            if (!ok && *(volatile int*)&tail->abort_flag) break;
+                            if (!ok && i > 64) __nanosleep(64);
+                        }
+                        if (!ok) {
+                            if (!*(volatile int*)&tail->abort_flag) latch_timeout(p.status, 5);
+                            tail->abort_flag = 1;
+                        }
+                        tail->is_last = ok;
+                    }
+                    consumer_bar_sync();
+                    if (!tail->is_last) break;   // all four warps: the cluster did not deliver
+                    fence_acq_rel_cluster();
+                    // (1) per head the global max, the pieces' weights and the global sum, (2) per dim the weighted sum
+                    // of the pieces' accumulators
+                    float* s_stat = reinterpret_cast<float*>(tail->scratch);   // [splits <= 8][16]: M[8] (then the weights), L[8]
                     for (int idx = tid; idx < p.splits * 16; idx += kConsumerThreads)
-                        s_stat[idx] = __ldcg(base + (size_t)(idx >> 4) * kPartFloats + (idx & 15));
+                        s_stat[idx] = rx[(size_t)(idx >> 4) * kPartFloats + (idx & 15)];
                     consumer_bar_sync();
                     if (tid < 8) {
                         const int h = tid;
@@ -513,8 +534,8 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                     for (int h = 0; h < 8; ++h) o[h] = 0.f;
 #pragma unroll 4
                     for (int sp = 0; sp < p.splits; ++sp) {
-                        const float4* a4 = reinterpret_cast<const float4*>(base + (size_t)sp * kPartFloats + 16 + tid * 8);
-                        const float4 a = __ldcg(a4), b = __ldcg(a4 + 1);
+                        const float4* a4 = reinterpret_cast<const float4*>(rx + (size_t)sp * kPartFloats + 16 + tid * 8);
+                        const float4 a = a4[0], b = a4[1];
                         const float4 wa = *reinterpret_cast<const float4*>(s_stat + sp * 16);
                         const float4 wb = *reinterpret_cast<const float4*>(s_stat + sp * 16 + 4);
                         o[0] = fmaf(wa.x, a.x, o[0]); o[1] = fmaf(wa.y, a.y, o[1]); o[2] = fmaf(wa.z, a.z, o[2]); o[3] = fmaf(wa.w, a.w, o[3]);
@@ -622,8 +643,11 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
 }
 
 // ---------------------------------------------------------------------------------------------
-static size_t decode_smem_bytes(int C, int accum, int stages) {
-    return 1024 + (size_t)stages * kStageBytes + decode_sum_bytes(C, accum ? 1 : 0) + sizeof(DecodeSmemTail);
+constexpr int kMaxSplits = 8;   // a unit's pieces are one thread-block cluster (portable size limit)
+
+static size_t decode_smem_bytes(int C, int accum, int stages, int splits) {
+    const size_t rx = splits > 1 ? (size_t)splits * kPartFloats * sizeof(float) : 0;   // the cluster's receive buffer
+    return 1024 + (size_t)stages * kStageBytes + decode_sum_bytes(C, accum ? 1 : 0) + sizeof(DecodeSmemTail) + rx;
 }
 
 // TMEM columns a window-step CTA allocates for its logits: 4 per 64-key tile, a power of two >= 32.
@@ -636,12 +660,13 @@ int decode_tmem_cols(int C) {
 
 // Key split of `units` units that would leave most of the device idle: about two CTAs per SM, so that all pieces
 // run at once (measured on 4..256 units of 18 tiles: 2 and 3 per SM are equal, 4 and more cost a second wave and
-// 30-50 % more time); the tiles are then spread evenly (no piece without a tile at full length).
+// 30-50 % more time), at most kMaxSplits pieces per unit; the tiles are then spread evenly (no piece without a
+// tile at full length).
 int decode_pick_splits(int units, int C, int sm_count) {
     const int max_tiles = (C + kTileKeys - 1) / kTileKeys;
     if (units <= 0 || units >= 2 * sm_count) return 1;
     int s_max = (2 * sm_count) / units;
-    if (s_max > 32) s_max = 32;
+    if (s_max > kMaxSplits) s_max = kMaxSplits;
     if (s_max < 1) s_max = 1;
     const int tiles_per_split = (max_tiles + s_max - 1) / s_max;
     return (max_tiles + tiles_per_split - 1) / tiles_per_split;
@@ -650,22 +675,22 @@ int decode_pick_splits(int units, int C, int sm_count) {
 // CTAs of a given shape that one SM holds (shared memory decides; 160 threads x 128 registers allow 3).
 // Window steps hold TMEM: resident CTAs x columns must stay within the SM's 512 columns, so that no CTA
 // ever waits for its allocation.
-static int decode_ctas_per_sm(int C, int accum, int stages) {
+static int decode_ctas_per_sm(int C, int accum, int stages, int splits) {
     const size_t cap = 227 * 1024;
     const int cta_cap = accum ? min(3, 512 / decode_tmem_cols(C)) : 3;
-    int ctas = (int)(cap / (decode_smem_bytes(C, accum, stages) + 1024));  // 1 KB per-CTA reservation
+    int ctas = (int)(cap / (decode_smem_bytes(C, accum, stages, splits) + 1024));  // 1 KB per-CTA reservation
     return ctas > cta_cap ? cta_cap : ctas;
 }
 
 // Resident CTAs per SM matter more than ring depth: with four consumer warps per CTA the per-warp
 // dependent chain (ldmatrix -> mma -> shuffles -> exp2 -> mma) needs >= 8-12 warps per SM to hide, so take
 // the stage count that allows the most CTAs per SM (up to 3), then the deepest ring that still fits.
-static int decode_pick_stages(int C, int accum) {
+static int decode_pick_stages(int C, int accum, int splits) {
     const size_t cap = 227 * 1024;
     int best = 2, best_score = -1;
     for (int st = 2; st <= kMaxStages; ++st) {
-        if (decode_smem_bytes(C, accum, st) > cap) break;
-        const int score = decode_ctas_per_sm(C, accum, st) * 100 + st;
+        if (decode_smem_bytes(C, accum, st, splits) > cap) break;
+        const int score = decode_ctas_per_sm(C, accum, st, splits) * 100 + st;
         if (score > best_score) {
             best_score = score;
             best = st;
@@ -676,20 +701,20 @@ static int decode_pick_stages(int C, int accum) {
 
 // Work plan of a launch. The grid is persistent (at most the CTAs the device holds at once) and hands out items
 // first come, first served. Units are whole items; only a launch so small that whole units would leave most SMs
-// idle is split over the keys, so that about two CTAs per SM run. (Splitting the last units of a large launch into
-// pieces of a few tiles, to even out the end, was measured and lost: a piece's epilogue -- partials to the
-// workspace, the completion count, the merge -- costs as much time as three tiles.) `max_pieces` > 0 bounds the
-// split scratch.
+// idle is split over the keys, so that about two CTAs per SM run: then the grid is one CTA per piece and the
+// pieces of a unit form a thread-block cluster. (Splitting the last units of a large launch into pieces of a few
+// tiles, to even out the end, was measured and lost: a piece's epilogue costs as much time as three tiles.)
+// `max_pieces` > 0 bounds the number of pieces.
 void decode_plan(DecodeLaunch* p, int max_pieces) {
     const int sm = p->sm_count > 0 ? p->sm_count : 148;
     const int units = p->n_layers * p->batch * p->h_kv;
-    p->stages = decode_pick_stages(p->C, p->accum);
     p->tmem_cols = decode_tmem_cols(p->C);
-    const int resident = decode_ctas_per_sm(p->C, p->accum, p->stages) * sm;
     p->splits = decode_pick_splits(units, p->C, sm);
     if (max_pieces > 0 && (long)units * p->splits > max_pieces) p->splits = 1;   // whole units still fit one wave
+    p->stages = decode_pick_stages(p->C, p->accum, p->splits);
+    const int resident = decode_ctas_per_sm(p->C, p->accum, p->stages, p->splits) * sm;
     const long items = (long)units * p->splits;
-    p->grid = (int)(items < resident ? items : resident);
+    p->grid = (int)((p->splits > 1 || items < resident) ? items : resident);
 }
 
 cudaError_t decode_kernel_setup() {
@@ -700,10 +725,27 @@ cudaError_t decode_kernel_setup() {
 
 // `p` must have been through decode_plan().
 cudaError_t launch_decode(const DecodeLaunch& p, const DecodeMaps& maps, cudaStream_t s) {
-    const size_t smem = decode_smem_bytes(p.C, p.accum, p.stages);
-    if (!p.accum) gkv_decode_kernel<0><<<p.grid, kDecodeThreads, smem, s>>>(p, maps);
-    else gkv_decode_kernel<1><<<p.grid, kDecodeThreads, smem, s>>>(p, maps);
-    return cudaGetLastError();
+    const size_t smem = decode_smem_bytes(p.C, p.accum, p.stages, p.splits);
+    if (p.splits == 1) {
+        if (!p.accum) gkv_decode_kernel<0><<<p.grid, kDecodeThreads, smem, s>>>(p, maps);
+        else gkv_decode_kernel<1><<<p.grid, kDecodeThreads, smem, s>>>(p, maps);
+        return cudaGetLastError();
+    }
+    // key split: clusters of p.splits CTAs, one per unit (grid = units x splits)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(kDecodeThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)p.splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (!p.accum) return cudaLaunchKernelEx(&cfg, gkv_decode_kernel<0>, p, maps);
+    return cudaLaunchKernelEx(&cfg, gkv_decode_kernel<1>, p, maps);
 }
 
 }  // namespace gkv

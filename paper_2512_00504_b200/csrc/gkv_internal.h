@@ -17,8 +17,6 @@ namespace gkv {
 struct WorkspaceLayout {
     uint64_t status;      // int32[64]   latched device status + diagnostics
     uint64_t seq_done;    // int32[L*batch]         CTA completion counters per (layer, sequence)
-    uint64_t unit_done;   // int32[L*batch*h_kv]    split completion counters per unit
-    uint64_t part;        // split-K partials: per (unit, split) M[8], L[8], acc[128][8] fp32
     uint64_t logits;      // split-K window steps: per unit C x 8 fp32 scaled logits
     uint64_t kept;        // int32[units_per_layer * b]   kept lists of the staged eviction path
     uint64_t fscratch;    // fp32[units_per_layer * C]    merged scores of the staged eviction path
@@ -41,8 +39,6 @@ struct DecodeLaunch {
     float* sacc;
     int32_t* len;        // plane 0 of the len buffer
     int32_t* seq_done;
-    int32_t* unit_done;
-    float* part;
     float* logits;
     int32_t* status;
     int32_t* work_next;  // two zeroed words: the next item's number minus the grid size, and the CTAs that are done
@@ -50,7 +46,8 @@ struct DecodeLaunch {
     int accum;           // 1 on window steps
     int sm_count;        // SMs of the device (sizes the persistent grid)
     // filled in by decode_plan():
-    int splits;          // every unit is `splits` work items, each a contiguous share of the keys
+    int splits;          // every unit is `splits` work items, each a contiguous share of the keys; > 1: the kernel is
+                         // launched in clusters of `splits` CTAs, one cluster per unit
     int stages, grid, tmem_cols;
     float scale_log2;    // log2(e) / sqrt(d)
 };

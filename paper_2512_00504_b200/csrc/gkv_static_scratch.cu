@@ -1,7 +1,8 @@
 // gkv_decode_attn_static: one decode-attention step that needs no buffer beyond its inputs and
-// outputs. The split-K partial results, the completion counters, the per-sequence length words and
-// the status word that the context-based call keeps in a caller-allocated workspace live here in a
-// fixed array inside the library's own device image.
+// outputs. The per-sequence length words, the completion and work counters and the status word that
+// the context-based call keeps in a caller-allocated workspace live here in a fixed array inside the
+// library's own device image. (The partial results of units split over the keys need no global
+// scratch: they meet in the shared memory of a thread-block cluster.)
 //
 // It exists for callers that cannot obtain device memory at the point of the call: code running
 // after an application has handed its whole memory budget to a pool it does not control (a plug-in
@@ -24,15 +25,10 @@ namespace {
 using namespace gkv;
 
 constexpr int kStaticMaxSeq = 1024;            // batch
-constexpr int kStaticMaxUnits = 1024;          // batch * n_kv_heads
-constexpr int kStaticMaxCtas = 1024;           // split-K pieces of a launch
-constexpr size_t kPartBytesPerCta = (16 + kHeadDim * 8) * sizeof(float);
-constexpr size_t kOffStatus = 0;                                   // int32[64]
+constexpr size_t kOffStatus = 0;                                   // int32[64]: status word, work counters
 constexpr size_t kOffLen = 256;                                    // int32[kStaticMaxSeq]
 constexpr size_t kOffSeqDone = kOffLen + 4 * kStaticMaxSeq;        // int32[kStaticMaxSeq]
-constexpr size_t kOffUnitDone = kOffSeqDone + 4 * kStaticMaxSeq;   // int32[kStaticMaxUnits]
-constexpr size_t kOffPart = kOffUnitDone + 4 * kStaticMaxUnits;    // split-K partials
-constexpr size_t kStaticScratchBytes = kOffPart + kStaticMaxCtas * kPartBytesPerCta;   // ~4.1 MiB
+constexpr size_t kStaticScratchBytes = kOffSeqDone + 4 * kStaticMaxSeq;   // 8.25 KiB
 
 // In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -104,7 +100,7 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
         return GKV_ERR_INVALID_ARG;
     if (len >= capacity) return GKV_ERR_CAPACITY;
     const long units = (long)batch * n_kv_heads;
-    if (batch > kStaticMaxSeq || units > kStaticMaxUnits) return GKV_ERR_SCRATCH_LIMIT;
+    if (batch > kStaticMaxSeq) return GKV_ERR_SCRATCH_LIMIT;
 
     unsigned char* scratch = nullptr;
     gkv_status st = scratch_for_current_device(&scratch);
@@ -118,9 +114,10 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     p.n_layers = 1; p.batch = batch; p.h_kv = n_kv_heads; p.C = capacity;
     p.accum = 0;
     p.sm_count = sm;
-    decode_plan(&p, kStaticMaxCtas);   // at most that many split-K pieces
+    decode_plan(&p, 0);
     DecodeMaps maps;
     const uint64_t rows = (uint64_t)units * capacity;
+    if (rows >= (1ull << 31)) return GKV_ERR_UNSUPPORTED;   // TMA row coordinate is a signed 32-bit integer
     if (!encode_rows(&maps.k64, k_cache, rows, kTileKeys) || !encode_rows(&maps.v64, v_cache, rows, kTileKeys) ||
         !encode_rows(&maps.k16, k_cache, rows, 16) || !encode_rows(&maps.v16, v_cache, rows, 16))
         return GKV_ERR_CUDA;
@@ -128,7 +125,7 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // The array keeps whatever the previous call left: status word and counters must start at zero,
     // and every sequence's length word is set to this call's `len`.
-    if (cudaMemsetAsync(scratch, 0, kOffPart, s) != cudaSuccess) return GKV_ERR_CUDA;
+    if (cudaMemsetAsync(scratch, 0, kStaticScratchBytes, s) != cudaSuccess) return GKV_ERR_CUDA;
     int32_t* d_len = reinterpret_cast<int32_t*>(scratch + kOffLen);
     gkv_static_fill_len<<<(batch + 255) / 256, 256, 0, s>>>(d_len, batch, len);
     if (cudaGetLastError() != cudaSuccess) return GKV_ERR_CUDA;
@@ -142,8 +139,6 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     p.sacc = nullptr;
     p.len = d_len;
     p.seq_done = reinterpret_cast<int32_t*>(scratch + kOffSeqDone);
-    p.unit_done = reinterpret_cast<int32_t*>(scratch + kOffUnitDone);
-    p.part = reinterpret_cast<float*>(scratch + kOffPart);
     p.logits = nullptr;
     p.status = reinterpret_cast<int32_t*>(scratch + kOffStatus);
     p.work_next = p.status + 32;
