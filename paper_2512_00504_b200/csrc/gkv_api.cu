@@ -59,19 +59,7 @@ void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     uint64_t off = 0;
     w->status = off;    off = align_up(off + 64 * sizeof(int32_t));
     w->seq_done = off;  off = align_up(off + L * B * sizeof(int32_t));
-    // logits of window steps whose units are split over the keys: the larger of a one-layer launch and an all-layer
-    // launch (the partial results of a split unit meet in shared memory, not here)
-    uint64_t logits = 0;
-    for (int i = 0; i < 2; ++i) {
-        DecodeLaunch d = {};
-        d.n_layers = i ? (int)L : 1; d.batch = (int)B; d.h_kv = (int)H; d.C = (int)C;
-        d.accum = 1;
-        d.sm_count = sm_count;
-        decode_plan(&d, 0);
-        const uint64_t lb = d.splits > 1 ? (uint64_t)d.n_layers * upl * C * 8 * sizeof(float) : 0;
-        if (lb > logits) logits = lb;
-    }
-    w->logits = off;   off = align_up(off + logits);
+    (void)sm_count;   // the decode kernel keeps nothing else here: split units merge in shared memory, logits stay in TMEM
     w->kept = off;     off = align_up(off + upl * c->budget * sizeof(int32_t));
     w->fscratch = off; off = align_up(off + upl * C * sizeof(float));
     const uint64_t red = c->use_redundancy ? 1 : 0;   // the redundancy term's scratch exists only when it is on
@@ -389,7 +377,6 @@ gkv_status gkv_decode_attn(gkv_ctx* ctx, int32_t layer, const void* q, const voi
     p.sacc = static_cast<float*>(ctx->buf.sacc);
     p.len = static_cast<int32_t*>(ctx->buf.len);
     p.seq_done = ws_ptr<int32_t>(ctx, ctx->ws.seq_done);
-    p.logits = ws_ptr<float>(ctx, ctx->ws.logits);
     p.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
     p.layer0 = l0; p.n_layers = nl; p.batch = c.batch; p.h_q = c.n_q_heads; p.h_kv = c.n_kv_heads;
     p.g = ctx->g; p.C = ctx->C;
@@ -702,7 +689,7 @@ gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream) {
     if (h[0] != 0) {
         // A kernel that gave up may have left its completion and work counters part-way (they are returned to zero
         // by the last CTA of a launch that runs to its end): clear them together with the latch.
-        if (cudaMemsetAsync(d, 0, ctx->ws.logits - ctx->ws.status, s) != cudaSuccess) return GKV_ERR_CUDA;
+        if (cudaMemsetAsync(d, 0, ctx->ws.kept - ctx->ws.status, s) != cudaSuccess) return GKV_ERR_CUDA;
         return GKV_ERR_TIMEOUT;
     }
     return GKV_OK;

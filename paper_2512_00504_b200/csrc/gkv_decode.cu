@@ -29,10 +29,13 @@ struct __align__(16) DecodeSmemTail {
     float l[kConsumerWarps][8];
     float fin_m[8];
     float fin_l[8];
+    float fin_c[8];     // fin_m + log2 fin_l of the whole unit: what a window step subtracts from its parked logits
     float wgt[kConsumerWarps][8];
     uint64_t q_full;    // the item's query rows have landed in q_rows (one bulk copy by the producer lane)
     uint64_t q_empty;   // the four consumer warps have the item's query fragments in registers
-    uint64_t cl_bar;    // key split: the other CTAs of the cluster arrive here when their partial results are in rx
+    // Key split. First CTA of the cluster: the others arrive here when their partial results are in rx. Other CTAs
+    // (window steps): the first CTA arrives here when it has stored the unit's fin_c into this CTA's shared memory.
+    uint64_t cl_bar;
     // The group's g query rows, contiguous as in global memory, and the current token's k and v rows.
     alignas(16) uint8_t q_rows[8 * 256];
     alignas(16) uint8_t new_rows[2 * 256];
@@ -98,8 +101,7 @@ __device__ __forceinline__ DecodeItem decode_item(const DecodeLaunch& p, int ite
     return d;
 }
 
-// ACCUM = 0: plain step. ACCUM = 1: window step; without key split the logits are parked in TMEM, with it they
-// go through the workspace.
+// ACCUM = 0: plain step. ACCUM = 1: window step (the logits are parked in TMEM until the unit's normaliser is known).
 template <int ACCUM>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
 gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps) {
@@ -110,7 +112,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
     uint8_t* stage_base = smem;
     float* s_sum = reinterpret_cast<float*>(smem + (size_t)stages * kStageBytes);   // [C] window sums, window steps only
     DecodeSmemTail* tail = reinterpret_cast<DecodeSmemTail*>(smem + (size_t)stages * kStageBytes + decode_sum_bytes(p.C, ACCUM));
-    // Window steps without key split keep the scaled logits [key][head] on chip until the row's
+    // Window steps keep the scaled logits [key][head] on chip until the row's
     // normaliser is final. They live in tensor memory, not shared memory: a consumer thread parks
     // the 4 values it owns of every tile in 4 columns of its own TMEM lane and reads them back
     // itself in the epilogue, so shared memory (and with it the number of resident CTAs) is nearly the
@@ -127,7 +129,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
         }
         mbar_init(smem_u32(&tail->q_full), 1);
         mbar_init(smem_u32(&tail->q_empty), kConsumerWarps);
-        if (p.splits > 1) mbar_init(smem_u32(&tail->cl_bar), (uint32_t)p.splits - 1);
+        if (p.splits > 1) mbar_init(smem_u32(&tail->cl_bar), (blockIdx.x % p.splits == 0) ? (uint32_t)p.splits - 1 : 1u);
         tail->q_issued = 0;
         tail->abort_flag = 0;
         tail->abort_seen = 0;
@@ -299,9 +301,10 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
             // Window steps: the unit's current window sums start their way into shared memory now and are needed only
             // in the epilogue; the updated sums go back with plain coalesced stores. (One atomic per key is measurably
             // slower: the L2 atomic units saturate at ~4 M reductions a launch.)
-            if (ACCUM == 1 && p.splits == 1) {
+            if (ACCUM == 1) {
                 const float* gsum = p.sacc + (size_t)d.unit * p.C;
-                for (int t = tid; t < n; t += kConsumerThreads) cp_async_4(smem_u32(s_sum + t), gsum + t);
+                const int k_hi = min(d.t_end * kTileKeys, n);      // this item's keys: [t_begin * 64, k_hi)
+                for (int t = d.t_begin * kTileKeys + tid; t < k_hi; t += kConsumerThreads) cp_async_4(smem_u32(s_sum + t), gsum + t);
                 cp_async_commit();
             }
 
@@ -361,13 +364,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                     float s2 = (sa[2] + sb[2]) * p.scale_log2, s3 = (sa[3] + sb[3]) * p.scale_log2;
                     if (key_a >= n) s0 = s1 = -INFINITY;
                     if (key_b >= n) s2 = s3 = -INFINITY;
-                    if (ACCUM == 1 && p.splits == 1) {
-                        tmem_st4(tmem_warp + 4u * (uint32_t)it, s0, s1, s2, s3);
-                    } else if (ACCUM == 1) {
-                        float* g_log = p.logits + (size_t)d.unit_local * p.C * 8;
-                        if (key_a < n) *reinterpret_cast<float2*>(g_log + key_a * 8 + h0) = make_float2(s0, s1);
-                        if (key_b < n) *reinterpret_cast<float2*>(g_log + key_b * 8 + h0) = make_float2(s2, s3);
-                    }
+                    if (ACCUM == 1) tmem_st4(tmem_warp + 4u * (uint32_t)it, s0, s1, s2, s3);
                     // tile maximum per head over the warp's 16 keys (lanes sharing lane & 3)
                     float t0 = fmaxf(s0, s2), t1 = fmaxf(s1, s3);
 #pragma unroll
@@ -436,6 +433,7 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                 }
                 tail->fin_m[h] = mm;
                 tail->fin_l[h] = ll;
+                if (ACCUM != 0) tail->fin_c[h] = (h < p.g) ? mm + log2f(ll) : INFINITY;
             }
             consumer_bar_sync();   // [E2]
             if (*(volatile int*)&tail->abort_seen) break;   // all four warps leave together
@@ -490,9 +488,10 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                 fence_acq_rel_cluster();
                 consumer_bar_sync();
                 do_final = d.split == 0;
-                if (!do_final) {
-                    if (tid == 0) mbar_arrive_cluster(cluster_map_shared(smem_u32(&tail->cl_bar), 0));
-                } else {
+                if (!do_final && tid == 0) mbar_arrive_cluster(cluster_map_shared(smem_u32(&tail->cl_bar), 0));
+                // The first CTA waits for the others' partial results; on a window step the others wait for the first
+                // CTA to hand them the unit's normaliser (they hold the logits of their own keys).
+                if (do_final || ACCUM != 0) {
                     if (tid == 0) {
                         bool ok = false;
                         for (uint32_t i = 0; i < kWaitSpins && !ok; ++i) {
@@ -509,6 +508,8 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                     consumer_bar_sync();
                     if (!tail->is_last) break;   // all four warps: the cluster did not deliver
                     fence_acq_rel_cluster();
+                }
+                if (do_final) {
                     // (1) per head the global max, the pieces' weights and the global sum, (2) per dim the weighted sum
                     // of the pieces' accumulators
                     float* s_stat = reinterpret_cast<float*>(tail->scratch);   // [splits <= 8][16]: M[8] (then the weights), L[8]
@@ -528,8 +529,16 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                         }
                         tail->fin_m[h] = mm;
                         tail->fin_l[h] = ll;
+                        if (ACCUM != 0) {
+                            const float c = (h < p.g) ? mm + log2f(ll) : INFINITY;
+                            tail->fin_c[h] = c;
+                            for (int r = 1; r < p.splits; ++r) st_cluster_f32(cluster_map_shared(smem_u32(&tail->fin_c[h]), (uint32_t)r), c);
+                            fence_acq_rel_cluster();
+                        }
                     }
                     consumer_bar_sync();
+                    if (ACCUM != 0 && tid == 0)
+                        for (int r = 1; r < p.splits; ++r) mbar_arrive_cluster(cluster_map_shared(smem_u32(&tail->cl_bar), (uint32_t)r));
 #pragma unroll
                     for (int h = 0; h < 8; ++h) o[h] = 0.f;
 #pragma unroll 4
@@ -558,48 +567,31 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
                     __nv_bfloat16* orow = p.out + ((size_t)(d.layer_local * p.batch + d.seq) * p.h_q + (size_t)d.head * p.g + h) * kHeadDim;
                     *reinterpret_cast<uint4*>(orow + c * 8) = *reinterpret_cast<const uint4*>(tail->scratch + h * 256 + c * 16);
                 }
-                if (ACCUM != 0) {
-                    // Sacc[t] += max over the group of the final weights = exp2(max_h (z_h[t] - M_h - log2 L_h)).
-                    if (p.splits == 1) {
-                        const float c0 = (h0 < p.g) ? tail->fin_m[h0] + log2f(tail->fin_l[h0]) : INFINITY;
-                        const float c1 = (h0 + 1 < p.g) ? tail->fin_m[h0 + 1] + log2f(tail->fin_l[h0 + 1]) : INFINITY;
-                        // four tiles per TMEM access; columns past the last tile are allocated but never written by this
-                        // item and are ignored (key >= n); each key of the unit is owned by exactly one thread
-                        for (int it4 = 0; it4 < d.tiles_total; it4 += 4) {
-                            float z[16];
-                            tmem_ld16(tmem_warp + 4u * (uint32_t)it4, z);
+            }
+            if (ACCUM != 0) {
+                // Sacc[t] += max over the group of the final weights = exp2(max_h (z_h[t] - M_h - log2 L_h)), for the keys
+                // of this item's tiles: their logits are in this CTA's TMEM, and each key is owned by exactly one thread.
+                const float c0 = tail->fin_c[h0], c1 = tail->fin_c[h0 + 1];
+                float* gsum = p.sacc + (size_t)d.unit * p.C;
+                // four tiles per TMEM access; columns of tiles that are not this item's hold other data and are skipped
+                for (int it4 = d.t_begin & ~3; it4 < d.t_end; it4 += 4) {
+                    float z[16];
+                    tmem_ld16(tmem_warp + 4u * (uint32_t)it4, z);
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                float va = fmaxf(z[4 * u] - c0, z[4 * u + 1] - c1), vb = fmaxf(z[4 * u + 2] - c0, z[4 * u + 3] - c1);
-                                va = fmaxf(va, __shfl_xor_sync(0xffffffffu, va, 1));
-                                vb = fmaxf(vb, __shfl_xor_sync(0xffffffffu, vb, 1));
-                                va = fmaxf(va, __shfl_xor_sync(0xffffffffu, va, 2));
-                                vb = fmaxf(vb, __shfl_xor_sync(0xffffffffu, vb, 2));
-                                const int key = (it4 + u) * kTileKeys + warp * 16 + (lane >> 2) + ((lane & 1) ? 8 : 0);
-                                if ((lane & 2) == 0 && key < n) s_sum[key] += fast_exp2((lane & 1) ? vb : va);
-                            }
-                        }
-                        consumer_bar_sync();   // every key's sum is final (its prefetch landed before [E1])
-                        float* gsum = p.sacc + (size_t)d.unit * p.C;
-                        for (int t = tid; t < n; t += kConsumerThreads) gsum[t] = s_sum[t];
-                    } else {
-                        float c[8];
-#pragma unroll
-                        for (int h = 0; h < 8; ++h) c[h] = (h < p.g) ? tail->fin_m[h] + log2f(tail->fin_l[h]) : INFINITY;
-                        float* sacc = p.sacc + (size_t)d.unit * p.C;
-                        const float* g_log = p.logits + (size_t)d.unit_local * p.C * 8;
-#pragma unroll 4   // independent loads: a few L2 round trips for the unit's logits instead of one per iteration
-                        for (int t = tid; t < n; t += kConsumerThreads) {
-                            const float4 x0 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8));
-                            const float4 x1 = __ldcg(reinterpret_cast<const float4*>(g_log + (size_t)t * 8 + 4));
-                            float v = x0.x - c[0];
-                            v = fmaxf(v, x0.y - c[1]); v = fmaxf(v, x0.z - c[2]); v = fmaxf(v, x0.w - c[3]);
-                            v = fmaxf(v, x1.x - c[4]); v = fmaxf(v, x1.y - c[5]); v = fmaxf(v, x1.z - c[6]);
-                            v = fmaxf(v, x1.w - c[7]);
-                            atomicAdd(sacc + t, fast_exp2(v));
-                        }
+                    for (int u = 0; u < 4; ++u) {
+                        if (it4 + u < d.t_begin || it4 + u >= d.t_end) continue;   // the same for the whole warp
+                        float va = fmaxf(z[4 * u] - c0, z[4 * u + 1] - c1), vb = fmaxf(z[4 * u + 2] - c0, z[4 * u + 3] - c1);
+                        va = fmaxf(va, __shfl_xor_sync(0xffffffffu, va, 1));
+                        vb = fmaxf(vb, __shfl_xor_sync(0xffffffffu, vb, 1));
+                        va = fmaxf(va, __shfl_xor_sync(0xffffffffu, va, 2));
+                        vb = fmaxf(vb, __shfl_xor_sync(0xffffffffu, vb, 2));
+                        const int key = (it4 + u) * kTileKeys + warp * 16 + (lane >> 2) + ((lane & 1) ? 8 : 0);
+                        if ((lane & 2) == 0 && key < n) s_sum[key] += fast_exp2((lane & 1) ? vb : va);
                     }
                 }
+                consumer_bar_sync();   // every key's sum is final (its prefetch landed before [E1])
+                const int k_hi = min(d.t_end * kTileKeys, n);
+                for (int t = d.t_begin * kTileKeys + tid; t < k_hi; t += kConsumerThreads) gsum[t] = s_sum[t];
             }
 
             // The last item of a (layer, sequence) publishes the new length.

@@ -17,7 +17,6 @@ namespace gkv {
 struct WorkspaceLayout {
     uint64_t status;      // int32[64]   latched device status + diagnostics
     uint64_t seq_done;    // int32[L*batch]         CTA completion counters per (layer, sequence)
-    uint64_t logits;      // split-K window steps: per unit C x 8 fp32 scaled logits
     uint64_t kept;        // int32[units_per_layer * b]   kept lists of the staged eviction path
     uint64_t fscratch;    // fp32[units_per_layer * C]    merged scores of the staged eviction path
     uint64_t prompt_sums; // fp32[units_per_layer * max_prompt]  window sums of a prompt being compressed
@@ -39,7 +38,6 @@ struct DecodeLaunch {
     float* sacc;
     int32_t* len;        // plane 0 of the len buffer
     int32_t* seq_done;
-    float* logits;
     int32_t* status;
     int32_t* work_next;  // two zeroed words: the next item's number minus the grid size, and the CTAs that are done
     int layer0, n_layers, batch, h_q, h_kv, g, C;

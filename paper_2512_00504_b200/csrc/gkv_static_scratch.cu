@@ -139,7 +139,6 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     p.sacc = nullptr;
     p.len = d_len;
     p.seq_done = reinterpret_cast<int32_t*>(scratch + kOffSeqDone);
-    p.logits = nullptr;
     p.status = reinterpret_cast<int32_t*>(scratch + kOffStatus);
     p.work_next = p.status + 32;
     p.layer0 = 0; p.n_layers = 1; p.batch = batch; p.h_q = n_q_heads; p.h_kv = n_kv_heads;
