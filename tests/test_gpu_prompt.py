@@ -193,6 +193,50 @@ def test_prompt_compression_with_redundancy_term(pool):
     assert differs > 0            # the term changed at least one head's selection: the case exercises it
 
 
+def test_decode_over_many_sequences_of_different_length():
+    """600 units whose sequences hold between 1 and b tokens (prompts short enough to be kept whole), decoded by a
+    persistent grid of 444 CTAs that take items of very different size from the work counter: plain steps, then
+    the window steps up to the scheduled compression, which evicts from the sequences that have grown past b only."""
+    B, h_q, h_kv, b, buffer, w, s = 75, 16, 8, 200, 24, 8, 24
+    rng = np.random.default_rng(synth.BASE_SEED + 130)
+    lens = rng.integers(1, b + 1, size=B).tolist()
+    lens[0], lens[1], lens[2] = 1, b, 64                            # the extremes and an exact tile
+    cfg = gkv.make_config(n_layers=1, batch=B, h_q=h_q, h_kv=h_kv, b=b, buffer=buffer, w=w, s=s, fuse_window_scores=True,
+                          max_prompt=b)
+    cache = gkv.GKVCache(cfg, DEV)
+    C = cache.C
+    gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 131)
+    rnd = lambda *sh: torch.randn(*sh, generator=gen, device=DEV).to(torch.bfloat16)
+    kp, vp = rnd(B, h_kv, b, 128), rnd(B, h_kv, b, 128)
+    cache.compress_prompt(0, kp, vp, None, lens)
+    assert cache.len[0, 0].cpu().numpy().tolist() == lens
+    Kh, Vh = synth.bits(cache.k[0]), synth.bits(cache.v[0])
+    sel = sorted({0, 1, 2, int(np.argmin(lens)), int(np.argmax(lens)), B // 2, B - 1})
+    sacc = {n: np.zeros((h_kv, C), np.float64) for n in sel}
+    out = torch.empty((B, h_q, 128), dtype=torch.bfloat16, device=DEV)
+    cur = list(lens)
+    for t in range(s):
+        q, kn, vn = rnd(B, h_q, 128), rnd(B, h_kv, 128), rnd(B, h_kv, 128)
+        cache.decode_attn(0, q, kn, vn, out)
+        got = out.float().cpu().numpy()
+        qb, kb, vb = synth.bits(q), synth.bits(kn), synth.bits(vn)
+        for n in range(B):
+            Kh[n, :, cur[n]], Vh[n, :, cur[n]] = kb[n], vb[n]
+            cur[n] += 1
+        for n in sel:
+            ref = oracle.decode_attention(qb[n], Kh[n], Vh[n], cur[n], Sacc=sacc[n] if t >= s - w else None)
+            assert np.abs(got[n] - ref).max() < DECODE_ATOL, (t, n, cur[n])
+    cache.poll()
+    assert cache.len[0, 0].cpu().numpy().tolist() == cur
+    assert (synth.bits(cache.k[0]) == Kh).all() and (synth.bits(cache.v[0]) == Vh).all()
+    got_sums = cache.sacc[0].cpu().numpy()
+    for n in sel:
+        np.testing.assert_allclose(got_sums[n], sacc[n], rtol=SCORE_RTOL, atol=SCORE_ATOL)
+    cache.evict(0)
+    cache.poll()
+    assert cache.len[0, 0].cpu().numpy().tolist() == [min(c, b) for c in cur]
+
+
 def test_prompt_call_errors():
     cfg = gkv.make_config(n_layers=1, batch=2, h_q=8, h_kv=2, b=64, buffer=16, w=8, s=16)
     cache = gkv.GKVCache(cfg, DEV)
