@@ -186,8 +186,8 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
  * inside a server whose memory pool it does not own, or a latency-critical loop where cudaMalloc is
  * off limits because it synchronises the device and may fail late. The caller passes only inputs and
  * outputs (device pointers): q [batch][n_q_heads][128], k_new / v_new [batch][n_kv_heads][128],
- * k_cache / v_cache [batch][n_kv_heads][capacity][128] (16-byte aligned), out [batch][n_q_heads][128],
- * all bf16. Semantics are those of gkv_decode_attn without window-score accumulation: k_new, v_new are
+ * k_cache / v_cache [batch][n_kv_heads][capacity][128], out [batch][n_q_heads][128], all bf16 and
+ * 16-byte aligned. Semantics are those of gkv_decode_attn without window-score accumulation: k_new, v_new are
  * written to row `len` of every head's cache and out is the attention over rows 0..len; the caller
  * keeps track of `len` itself (it is passed by value, nothing is read back).
  * The length words, completion and work counters and the status word live in an array of 8.25 KiB
@@ -201,7 +201,7 @@ gkv_status gkv_evict_host(gkv_ctx* ctx, int32_t layer, const void* q_window_host
  * make that first call outside any stream capture. The call itself performs no cudaMalloc / cudaFree.
  * A bounded wait that expires inside the kernel cannot be polled through this entry point; `out` is
  * then undefined.
- * Errors: INVALID_ARG (NULL, non-positive sizes, misaligned cache), UNSUPPORTED (g > 8, capacity > 4096),
+ * Errors: INVALID_ARG (NULL, non-positive sizes, a pointer not 16-byte aligned), UNSUPPORTED (g > 8, capacity > 4096),
  * CAPACITY (len >= capacity), SCRATCH_LIMIT, CUDA. */
 gkv_status gkv_decode_attn_static(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                   void* v_cache, void* out, int32_t batch, int32_t n_q_heads,
