@@ -261,6 +261,18 @@ int64_t gkv_launch_count(const gkv_ctx* ctx);
  * declare the state anew with gkv_set_state before going on. */
 gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream);
 
+/* How gkv_decode_attn would launch its kernel (no paper counterpart: a view of the host-side planning, for
+ * capacity planning and for tests that need no GPU). n_layers_in_launch = 1 (one layer per call) or
+ * cfg->n_layers (layer = -1); window_step != 0 for a step that accumulates window scores; sm_count = SMs of the
+ * device (<= 0: 148). grid = CTAs launched (persistent: never more than are resident at once), splits = pieces a
+ * unit's keys are split into (> 1: the pieces of a unit form one thread-block cluster of that size), stages = depth
+ * of the K/V tile ring, ctas_per_sm = resident CTAs per SM, smem_bytes = dynamic shared memory per CTA,
+ * tmem_cols = tensor-memory columns per CTA on window steps. Pure host arithmetic.
+ * Errors: as gkv_query_sizes; INVALID_ARG for a layer count other than 1 or cfg->n_layers. */
+typedef struct { int32_t grid, splits, stages, ctas_per_sm, smem_bytes, tmem_cols; } gkv_decode_plan_t;
+gkv_status gkv_decode_launch_plan(const gkv_config* cfg, int32_t n_layers_in_launch, int32_t window_step,
+                                  int32_t sm_count, gkv_decode_plan_t* out);
+
 /* Memory model of the paper's appendix "Memory Analysis": bytes of the full KV cache at
  * seq_len tokens, of the compressed cache ((b + s) rows instead of seq_len), and of the score
  * cache F (b - w entries per head), for `elem_bytes`-wide elements, over all layers and the

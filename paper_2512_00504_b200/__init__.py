@@ -51,6 +51,10 @@ class gkv_buffers(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("k", "v", "f", "sacc", "pos", "len", "workspace", "staging")]
 
 
+class gkv_decode_plan_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("grid", "splits", "stages", "ctas_per_sm", "smem_bytes", "tmem_cols")]
+
+
 class gkv_memory_model_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint64) for n in ("full_kv", "compressed_kv", "score_cache")]
 
@@ -102,13 +106,14 @@ def lib() -> ctypes.CDLL:
         L.gkv_launch_count.restype = i64
         L.gkv_poll_device_status.argtypes = [vp, vp]
         L.gkv_memory_model.argtypes = [P(gkv_config), i64, i32, P(gkv_memory_model_t)]
+        L.gkv_decode_launch_plan.argtypes = [P(gkv_config), i32, i32, i32, P(gkv_decode_plan_t)]
         L.gkv_strerror.argtypes = [ctypes.c_int]
         L.gkv_strerror.restype = ctypes.c_char_p
         L.gkv_destroy.argtypes = [vp]
         L.gkv_destroy.restype = None
         for name in ("gkv_query_sizes", "gkv_init", "gkv_set_state", "gkv_decode_attn", "gkv_evict", "gkv_evict_stage",
                      "gkv_decode_attn_host", "gkv_evict_host", "gkv_get_state", "gkv_get_redundancy", "gkv_set_eviction_log", "gkv_compress_prompt", "gkv_poll_device_status",
-                     "gkv_memory_model"):
+                     "gkv_memory_model", "gkv_decode_launch_plan"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -153,6 +158,13 @@ def gkv_strerror(status: int) -> str:
 def gkv_query_sizes(cfg: gkv_config) -> gkv_sizes:
     out = gkv_sizes()
     _check(lib().gkv_query_sizes(ctypes.byref(cfg), ctypes.byref(out)), "gkv_query_sizes")
+    return out
+
+
+def gkv_decode_launch_plan(cfg: gkv_config, n_layers_in_launch: int, window_step: bool = False, sm_count: int = 148) -> gkv_decode_plan_t:
+    out = gkv_decode_plan_t()
+    _check(lib().gkv_decode_launch_plan(ctypes.byref(cfg), int(n_layers_in_launch), int(bool(window_step)), int(sm_count),
+                                        ctypes.byref(out)), "gkv_decode_launch_plan")
     return out
 
 

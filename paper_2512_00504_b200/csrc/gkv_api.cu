@@ -695,6 +695,25 @@ gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream) {
     return GKV_OK;
 }
 
+gkv_status gkv_decode_launch_plan(const gkv_config* cfg, int32_t n_layers_in_launch, int32_t window_step,
+                                  int32_t sm_count, gkv_decode_plan_t* out) {
+    if (!out) return GKV_ERR_INVALID_ARG;
+    const gkv_status st = check_config(cfg);
+    if (st != GKV_OK) return st;
+    if (n_layers_in_launch != 1 && n_layers_in_launch != cfg->n_layers) return GKV_ERR_INVALID_ARG;
+    DecodeLaunch d = {};
+    d.n_layers = n_layers_in_launch; d.batch = cfg->batch; d.h_kv = cfg->n_kv_heads; d.C = cfg->budget + cfg->buffer;
+    d.accum = window_step ? 1 : 0;
+    d.sm_count = sm_count;
+    decode_plan(&d, 0);
+    int ctas = 0;
+    size_t smem = 0;
+    decode_plan_resources(d, &ctas, &smem);
+    out->grid = d.grid; out->splits = d.splits; out->stages = d.stages; out->ctas_per_sm = ctas;
+    out->smem_bytes = (int32_t)smem; out->tmem_cols = d.accum ? d.tmem_cols : 0;
+    return GKV_OK;
+}
+
 gkv_status gkv_memory_model(const gkv_config* cfg, int64_t seq_len, int32_t elem_bytes, gkv_memory_model_t* out) {
     if (!cfg || !out || seq_len <= 0 || elem_bytes <= 0) return GKV_ERR_INVALID_ARG;
     if (cfg->n_layers <= 0 || cfg->batch <= 0 || cfg->n_kv_heads <= 0 || cfg->head_dim <= 0 || cfg->budget <= 0 ||

@@ -709,6 +709,11 @@ void decode_plan(DecodeLaunch* p, int max_pieces) {
     p->grid = (int)((p->splits > 1 || items < resident) ? items : resident);
 }
 
+void decode_plan_resources(const DecodeLaunch& p, int* ctas_per_sm, size_t* smem_bytes) {
+    *ctas_per_sm = decode_ctas_per_sm(p.C, p.accum, p.stages, p.splits);
+    *smem_bytes = decode_smem_bytes(p.C, p.accum, p.stages, p.splits);
+}
+
 cudaError_t decode_kernel_setup() {
     cudaError_t e = cudaFuncSetAttribute(gkv_decode_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;

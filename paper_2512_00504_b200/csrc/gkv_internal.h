@@ -140,6 +140,7 @@ namespace gkv {
 
 int decode_pick_splits(int units_in_launch, int C, int sm_count);
 void decode_plan(DecodeLaunch* p, int max_pieces);
+void decode_plan_resources(const DecodeLaunch& p, int* ctas_per_sm, size_t* smem_bytes);   // of a planned launch
 cudaError_t launch_decode(const DecodeLaunch& p, const DecodeMaps& maps, cudaStream_t s);
 cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s);
 cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s);

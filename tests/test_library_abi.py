@@ -97,6 +97,50 @@ def test_workspace_grows_with_the_prompt_limit():
     assert w64p - w64 >= upl * 65536 * 4                       # pooled scores (+ the cache-sized selection scratch)
 
 
+def test_decode_launch_plan_of_the_benchmark_shapes():
+    """Host-side planning of the decode launch. The 7B-shaped configuration fills a persistent grid of three CTAs per
+    SM with whole units; one layer of it at a time has too few units for that and splits each unit's keys over a
+    thread-block cluster."""
+    cfg2 = gkv.make_config(n_layers=28, batch=32, h_q=28, h_kv=4, b=1024, buffer=128, w=32, s=128)
+    for window in (False, True):
+        p = gkv.gkv_decode_launch_plan(cfg2, 28, window)
+        assert (p.grid, p.splits, p.stages, p.ctas_per_sm) == (3 * 148, 1, 2, 3)
+        assert p.tmem_cols == (128 if window else 0)             # 4 columns per 64-key tile of 1152 rows, power of two
+        assert 3 * (p.smem_bytes + 1024) <= 227 * 1024
+    one = gkv.gkv_decode_launch_plan(cfg2, 1, False)              # 128 units: two pieces each, 256 CTAs in one wave
+    assert (one.grid, one.splits) == (256, 2)
+    cfg1 = gkv.make_config(n_layers=1, batch=1, h_q=28, h_kv=4, b=512, buffer=128, w=16, s=128)
+    tiny = gkv.gkv_decode_launch_plan(cfg1, 1, False)             # 4 units of 10 tiles: clusters of at most 8
+    assert 1 < tiny.splits <= 8 and tiny.grid == 4 * tiny.splits
+    with pytest.raises(gkv.GKVError) as e:
+        gkv.gkv_decode_launch_plan(cfg2, 5, False)
+    assert e.value.status == gkv.GKV_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("sm_count", [148, 132, 64])
+def test_decode_launch_plan_invariants(sm_count):
+    """Over a grid of shapes: the grid never exceeds what is resident at once (no CTA waits for another to finish
+    before it can start, which the in-kernel work counter and the clusters rely on), clusters stay within the portable
+    size, shared and tensor memory of the resident CTAs fit one SM, and no piece of a split unit is left without
+    a tile at full length."""
+    for b, buffer in ((64, 16), (512, 128), (1024, 128), (2048, 256), (3968, 128)):
+        for batch, h_kv, layers in ((1, 2, 1), (8, 8, 1), (32, 4, 28), (256, 8, 1), (128, 8, 64)):
+            cfg = gkv.make_config(n_layers=layers, batch=batch, h_q=4 * h_kv, h_kv=h_kv, b=b, buffer=buffer, w=16, s=buffer)
+            for nl in {1, layers}:
+                for window in (False, True):
+                    p = gkv.gkv_decode_launch_plan(cfg, nl, window, sm_count)
+                    units, tiles = nl * batch * h_kv, -(-(b + buffer) // 64)
+                    assert 1 <= p.splits <= 8 and 2 <= p.stages <= 6 and 1 <= p.ctas_per_sm <= 3
+                    assert p.ctas_per_sm * (p.smem_bytes + 1024) <= 227 * 1024
+                    assert p.tmem_cols * p.ctas_per_sm <= 512 and (not window or p.tmem_cols >= 4 * tiles)
+                    assert p.grid <= max(units * p.splits, 1) and p.grid <= p.ctas_per_sm * sm_count or p.splits > 1
+                    if p.splits > 1:
+                        assert p.grid == units * p.splits <= 2 * sm_count + 8       # one wave, about two CTAs per SM
+                        assert (p.splits - 1) * -(-tiles // p.splits) < tiles         # the last piece has a tile
+                    else:
+                        assert p.grid == min(units, p.ctas_per_sm * sm_count)
+
+
 def test_memory_model_reproduces_the_papers_appendix():
     """Appendix "Memory Analysis": 28 layers, d = 128, 2 KV heads, bf16, 16k tokens -> ~0.44 GB per
     sequence and 56 GB at batch 128; with s = 128 and b = 512 / 1024 / 2048 the compressed cache
