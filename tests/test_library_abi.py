@@ -138,7 +138,9 @@ def test_decode_launch_plan_invariants(sm_count):
                         assert p.grid == units * p.splits <= 2 * sm_count + 8       # one wave, about two CTAs per SM
                         assert (p.splits - 1) * -(-tiles // p.splits) < tiles         # the last piece has a tile
                     else:
-                        assert p.grid == min(units, p.ctas_per_sm * sm_count)
+                        resident = p.ctas_per_sm * sm_count
+                        rounds = -(-units // resident)
+                        assert -(-units // rounds) <= p.grid <= min(units, resident)   # full grid, or equal rounds
 
 
 def test_memory_model_reproduces_the_papers_appendix():
