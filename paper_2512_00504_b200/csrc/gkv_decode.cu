@@ -473,6 +473,10 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
 
             bool do_final = true;          // this CTA writes the output (always true without split)
             if (p.splits > 1) {
+                // (A CTA outlives every access to its shared memory from the cluster as long as no wait expires: the
+                // first CTA leaves after all others have arrived, the others -- on window steps -- after the first has.
+                // A closing cluster barrier would cover expired waits too; it costs 0.2-0.6 us per launch, measured,
+                // and a wait expires only after >= 0.27 s without the partner, by when that partner has given up as well.)
                 // The pieces of a unit are the CTAs of one cluster. Every CTA stores its (max, sum) per head and its
                 // accumulators into slot `rank` of the receive buffer in the shared memory of the cluster's first CTA
                 // (distributed shared memory: no trip through L2, no completion counter in global memory), then
