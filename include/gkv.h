@@ -96,7 +96,7 @@ typedef struct {
      * gives no kernel size and reports that pooling does not help at decode time. */
     int32_t pool_kernel;
     /* Longest prompt gkv_compress_prompt will be given (rows per head of its K / V buffers); 0 = that call is
-     * not used. At most 65536; above 8192 the window must be a multiple of 16 and use_redundancy off (UNSUPPORTED
+     * not used. At most 1048576; above 8192 the window must be a multiple of 16 and use_redundancy off (UNSUPPORTED
      * otherwise) and q_window 16-byte aligned. Sizes part of the workspace (4 bytes per prompt token and KV head, twice or three times
      * that above 8192). */
     int32_t max_prompt;
@@ -260,6 +260,13 @@ int64_t gkv_launch_count(const gkv_ctx* ctx);
  * again; what the kernel that gave up had written (outputs, cache rows, lengths) is undefined:
  * declare the state anew with gkv_set_state before going on. */
 gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream);
+
+/* Self-test of the failure path (no paper counterpart): launches one warp that waits, through the same bounded-wait
+ * helper every kernel of the library uses, on a barrier nobody arrives on, with a limit of `spins` polls
+ * (1..65536; microseconds). The wait runs out, the kernel latches the status word and returns: nothing traps,
+ * faults or hangs. The next gkv_poll_device_status reports GKV_ERR_TIMEOUT once, and the context stays usable
+ * (the cache state is untouched by this call). Errors: INVALID_ARG, CUDA. */
+gkv_status gkv_selftest_bounded_wait(gkv_ctx* ctx, int32_t spins, void* stream);
 
 /* How gkv_decode_attn would launch its kernel (no paper counterpart: a view of the host-side planning, for
  * capacity planning and for tests that need no GPU). n_layers_in_launch = 1 (one layer per call) or

@@ -102,6 +102,8 @@ def lib() -> ctypes.CDLL:
         L.gkv_compress_prompt.argtypes = [vp, i32, vp, vp, vp, P(i32), vp, vp]
         L.gkv_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
         L.gkv_decode_attn_static.restype = ctypes.c_int
+        L.gkv_selftest_bounded_wait.argtypes = [vp, i32, vp]
+        L.gkv_selftest_bounded_wait.restype = ctypes.c_int
         L.gkv_launch_count.argtypes = [vp]
         L.gkv_launch_count.restype = i64
         L.gkv_poll_device_status.argtypes = [vp, vp]
@@ -242,6 +244,10 @@ def gkv_launch_count(ctx) -> int:
 
 def gkv_poll_device_status(ctx):
     _check(lib().gkv_poll_device_status(ctx, _stream()), "gkv_poll_device_status")
+
+
+def gkv_selftest_bounded_wait(ctx, spins: int = 1024):
+    _check(lib().gkv_selftest_bounded_wait(ctx, int(spins), _stream()), "gkv_selftest_bounded_wait")
 
 
 def gkv_destroy(ctx):

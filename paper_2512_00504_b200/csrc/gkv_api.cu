@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kMaxCapacity = 4096;
 constexpr int kMaxPromptShared = 8192;   // up to here a prompt's scores stay in shared memory during the selection
-constexpr int kMaxPrompt = 65536;        // longest prompt gkv_compress_prompt takes (16-bit counts in the selection's scan)
+constexpr int kMaxPrompt = 1 << 20;      // longest prompt gkv_compress_prompt takes (a stated bound, not a structural one)
 constexpr uint64_t kAlign = 256;
 
 uint64_t align_up(uint64_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -255,9 +255,34 @@ gkv_status reset_sacc(gkv_ctx* ctx, int l0, int nl, cudaStream_t s) {
     return GKV_OK;
 }
 
+// Self-test of the bounded wait: one warp waits, with a short limit, on an mbarrier that nobody arrives on. The wait
+// runs out, the kernel latches the status word the way every kernel of the library does, and returns.
+__global__ void gkv_selftest_wait_kernel(int32_t* status, uint32_t spins) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0 && !mbar_wait_bounded(smem_u32(&bar), 0, spins)) {
+        if (atomicCAS(status, 0, kStatusTimeout) == 0) {
+            status[1] = 90;
+            status[2] = blockIdx.x;
+        }
+    }
+}
+
 }  // namespace
 
 extern "C" {
+
+gkv_status gkv_selftest_bounded_wait(gkv_ctx* ctx, int32_t spins, void* stream) {
+    if (!ctx || spins < 1 || spins > (1 << 16)) return GKV_ERR_INVALID_ARG;
+    gkv_selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ws_ptr<int32_t>(ctx, ctx->ws.status), (uint32_t)spins);
+    if (cudaGetLastError() != cudaSuccess) return GKV_ERR_CUDA;
+    ctx->launches += 1;
+    return GKV_OK;
+}
 
 gkv_status gkv_query_sizes(const gkv_config* cfg, gkv_sizes* out) {
     if (!out) return GKV_ERR_INVALID_ARG;
@@ -517,7 +542,10 @@ gkv_status gkv_decode_attn_host(gkv_ctx* ctx, int32_t layer, const void* q_host,
     int l0, nl;
     layer_range(ctx, layer, &l0, &nl);
     const gkv_config& c = ctx->cfg;
+    // the checks gkv_decode_attn would fail on, before any copy is queued
+    if (!uniform(ctx->len, l0, nl) || !uniform(ctx->since_evict, l0, nl)) return GKV_ERR_STATE;
     if (ctx->len[l0] >= ctx->C) return GKV_ERR_CAPACITY;
+    if (c.fuse_window_scores && ctx->since_evict[l0] >= c.interval) return GKV_ERR_STATE;
     const size_t qb = (size_t)nl * c.batch * c.n_q_heads * kHeadDim * 2;
     const size_t kb = (size_t)nl * c.batch * c.n_kv_heads * kHeadDim * 2;
     uint8_t* st = static_cast<uint8_t*>(ctx->buf.staging);
@@ -624,7 +652,7 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
     p.v_cache = static_cast<__nv_bfloat16*>(ctx->buf.v);
     p.f = static_cast<float*>(ctx->buf.f);
     p.sacc = static_cast<float*>(ctx->buf.sacc);
-    p.pos = static_cast<int32_t*>(ctx->buf.pos);
+    p.pos = c.track_positions ? static_cast<int32_t*>(ctx->buf.pos) : nullptr;
     p.len = static_cast<int32_t*>(ctx->buf.len);
     p.sums = sums;
     p.f_long = c.max_prompt > kMaxPromptShared ? ws_ptr<float>(ctx, ctx->ws.prompt_f) : nullptr;

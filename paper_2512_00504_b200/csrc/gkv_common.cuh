@@ -54,8 +54,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait: gives up after kWaitSpins polls (each poll itself suspends for a hardware-bounded
 // time), so a lost completion turns into an error code instead of a hang.
 constexpr uint32_t kWaitSpins = 1u << 22;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitSpins; ++i) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t spins = kWaitSpins) {
+    for (uint32_t i = 0; i < spins; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 64) __nanosleep(64);
     }
@@ -93,6 +93,10 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The two halves on their own: arrive does not block; wait returns once every thread of the cluster that has not
+// exited has arrived.
+__device__ __forceinline__ void cluster_arrive_all() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_all() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 // Untiled bulk copy global -> shared (no multicast), completion on an mbarrier. Both addresses 16-byte aligned,
 // `bytes` a multiple of 16.

@@ -473,10 +473,11 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
 
             bool do_final = true;          // this CTA writes the output (always true without split)
             if (p.splits > 1) {
-                // (A CTA outlives every access to its shared memory from the cluster as long as no wait expires: the
-                // first CTA leaves after all others have arrived, the others -- on window steps -- after the first has.
-                // A closing cluster barrier would cover expired waits too; it costs 0.2-0.6 us per launch, measured,
-                // and a wait expires only after >= 0.27 s without the partner, by when that partner has given up as well.)
+                // (Lifetime of the shared memory that other CTAs of the cluster write: rx and cl_bar of the first CTA;
+                // on window steps also fin_c and cl_bar of the others. Every CTA of a split launch arrives on the
+                // cluster barrier as its last act, and the CTAs that own remotely written memory also wait on it, so
+                // they stay resident until every peer has passed its last remote store -- by order, also when a bounded
+                // wait has expired somewhere, since every wait in this kernel is bounded and every CTA gets to the end.)
                 // The pieces of a unit are the CTAs of one cluster. Every CTA stores its (max, sum) per head and its
                 // accumulators into slot `rank` of the receive buffer in the shared memory of the cluster's first CTA
                 // (distributed shared memory: no trip through L2, no completion counter in global memory), then
@@ -623,6 +624,11 @@ gkv_decode_kernel(const DecodeLaunch p, const __grid_constant__ DecodeMaps maps)
     }
     if (ACCUM == 1) cp_async_wait_all();
     __syncthreads();
+    if (p.splits > 1) {
+        // closing cluster barrier: all arrive (does not block); only owners of remotely written shared memory wait
+        cluster_arrive_all();
+        if (blockIdx.x % p.splits == 0 || ACCUM != 0) cluster_wait_all();
+    }
     // The last CTA to get here puts the two counters back to zero for the next launch (every CTA has taken its last
     // number from work_next before it counts itself done).
     if (tid == 0) {

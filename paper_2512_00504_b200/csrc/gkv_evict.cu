@@ -18,7 +18,7 @@ constexpr int kCompactUnroll = 4;
 
 struct EvictShared {
     int hist[256];
-    int warp_sums[8];
+    int warp_sums[16];
     float warp_max[8];
     int digit, k_rem, first_evicted, is_last;
 };
@@ -38,6 +38,26 @@ __device__ __forceinline__ int block_incl_scan(int v, int* warp_sums, int tid) {
     for (int i = 0; i < 8; ++i) base += (i < warp) ? warp_sums[i] : 0;
     __syncthreads();
     return v + base;
+}
+
+// the same for two counters at once (full 32-bit range each)
+__device__ __forceinline__ int2 block_incl_scan2(int a, int b, int* warp_sums, int tid) {
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int ta = __shfl_up_sync(0xffffffffu, a, o), tb = __shfl_up_sync(0xffffffffu, b, o);
+        if (lane >= o) { a += ta; b += tb; }
+    }
+    if (lane == 31) { warp_sums[warp] = a; warp_sums[8 + warp] = b; }
+    __syncthreads();
+    int base_a = 0, base_b = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        base_a += (i < warp) ? warp_sums[i] : 0;
+        base_b += (i < warp) ? warp_sums[8 + i] : 0;
+    }
+    __syncthreads();
+    return make_int2(a + base_a, b + base_b);
 }
 
 __device__ __forceinline__ float block_max(float v, float* warp_max, int tid) {
@@ -160,8 +180,8 @@ __device__ int select_phase(const float* s_f, int* s_kept, int* s_evict, int n_c
         eq += (x == T);
     }
     if (tid == 0) sh->first_evicted = n_c;
-    const int packed = block_incl_scan(gt | (eq << 16), sh->warp_sums, tid);  // counts < 65536 each
-    int gt_before = (packed & 0xffff) - gt, eq_before = (packed >> 16) - eq;
+    const int2 incl = block_incl_scan2(gt, eq, sh->warp_sums, tid);
+    int gt_before = incl.x - gt, eq_before = incl.y - eq;
     int first_drop = n_c;
     for (int t = t0; t < t1; ++t) {
         const uint32_t x = ordered_bits(bits[t]);

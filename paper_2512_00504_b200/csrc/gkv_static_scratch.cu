@@ -40,11 +40,19 @@ __global__ void gkv_static_fill_len(int32_t* len, int n, int32_t value) {
 
 // Device address of the array on the current device, resolved once per device.
 constexpr int kMaxDevices = 64;
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
 std::mutex g_mu;
 unsigned char* g_addr[kMaxDevices] = {};
+int g_sm_count[kMaxDevices] = {};
 bool g_ready[kMaxDevices] = {};
+EncodeFn g_encode = nullptr;     // the driver's tensor-map encoder, looked up once per process
 
-gkv_status scratch_for_current_device(unsigned char** out) {
+// Set-up on the first call per device (with that device current): the array's device address, the SM count, the
+// decode kernel's shared-memory attribute, and -- once per process -- the tensor-map encoder. Later calls only read.
+gkv_status scratch_for_current_device(unsigned char** out, int* sm_count) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GKV_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_mu);
@@ -54,33 +62,36 @@ gkv_status scratch_for_current_device(unsigned char** out) {
             (void)cudaGetLastError();
             return GKV_ERR_CUDA;
         }
-        if (decode_kernel_setup() != cudaSuccess) {
+        if (decode_kernel_setup() != cudaSuccess ||
+            cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
             (void)cudaGetLastError();
             return GKV_ERR_CUDA;
+        }
+        if (!g_encode) {
+            void* sym = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+                q != cudaDriverEntryPointSuccess || !sym) {
+                (void)cudaGetLastError();
+                return GKV_ERR_CUDA;
+            }
+            g_encode = reinterpret_cast<EncodeFn>(sym);
         }
         g_addr[dev] = static_cast<unsigned char*>(p);
         g_ready[dev] = true;
     }
     *out = g_addr[dev];
+    *sm_count = g_sm_count[dev];
     return GKV_OK;
 }
 
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 // [rows][128] bf16 view in boxes of box_rows rows x 64 elements with the 128-byte swizzle the decode kernel expects.
 bool encode_rows(CUtensorMap* map, void* base, uint64_t rows, uint32_t box_rows) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess || !sym)
-        return false;
     const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
     const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    return reinterpret_cast<EncodeFn>(sym)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+    return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
                                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -103,12 +114,9 @@ extern "C" gkv_status gkv_decode_attn_static(const void* q, const void* k_new, c
     if (batch > kStaticMaxSeq) return GKV_ERR_SCRATCH_LIMIT;
 
     unsigned char* scratch = nullptr;
-    gkv_status st = scratch_for_current_device(&scratch);
+    int sm = 0;
+    gkv_status st = scratch_for_current_device(&scratch, &sm);
     if (st != GKV_OK) return st;
-    int dev = 0, sm = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-        return GKV_ERR_CUDA;
 
     DecodeLaunch p;
     p.n_layers = 1; p.batch = batch; p.h_kv = n_kv_heads; p.C = capacity;

@@ -607,6 +607,42 @@ def test_latched_device_status_is_reported_once():
     assert torch.equal(out.view(1, 2, 4, 128), vn.view(1, 2, 1, 128).expand(1, 2, 4, 128))
 
 
+def test_bounded_wait_runs_out_on_the_device_and_is_reported_once():
+    """The failure path taken for real, without faulting, trapping or hanging anything: a one-warp kernel waits, through
+    the bounded-wait helper every kernel of the library uses, on a barrier that nobody arrives on, with a short limit.
+    The wait runs out, the kernel latches the status word and returns; the poll reports the timeout once, and decode
+    and eviction afterwards still agree with the oracle."""
+    shape = dict(n_layers=1, batch=2, h_q=8, h_kv=2, b=96, buffer=32, w=8, s=32)
+    cache = gkv.GKVCache(gkv.make_config(**shape, fuse_window_scores=True), DEV)
+    B, Hq, H = 2, 8, 2
+    gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 77)
+    rnd = lambda *s: torch.randn(*s, generator=gen, device=DEV).to(torch.bfloat16)
+    start = 70
+    cache.k[0, :, :, :start] = rnd(B, H, start, 128)
+    cache.v[0, :, :, :start] = rnd(B, H, start, 128)
+    cache.set_state(0, start, 0, 0)
+    cache.poll()
+    before = gkv.gkv_launch_count(cache.ctx)
+    gkv.gkv_selftest_bounded_wait(cache.ctx, 1024)
+    assert gkv.gkv_launch_count(cache.ctx) == before + 1
+    with pytest.raises(gkv.GKVError) as e:
+        cache.poll()
+    assert e.value.status == gkv.GKV_ERR_TIMEOUT
+    words = cache.workspace[:16].view(torch.int32)
+    cache.poll()                                                   # reported once, then clear
+    assert int(words.abs().max()) == 0
+    assert cache.state(0) == (start, 0, 0)                         # the self-test does not touch the schedule state
+    q, kn, vn = rnd(B, Hq, 128), rnd(B, H, 128), rnd(B, H, 128)
+    out = torch.empty_like(q)
+    cache.decode_attn(0, q, kn, vn, out)
+    cache.poll()
+    ref = oracle.decode_batch(synth.bits(q), synth.bits(cache.k[0]), synth.bits(cache.v[0]), start + 1)
+    assert float(abs(out.float().cpu().numpy() - ref).max()) < DECODE_ATOL
+    with pytest.raises(gkv.GKVError) as e:                         # argument checks of the self-test itself
+        gkv.gkv_selftest_bounded_wait(cache.ctx, 0)
+    assert e.value.status == gkv.GKV_ERR_INVALID_ARG
+
+
 def test_config2_full_length_run_sampled():
     """Configuration 2 end to end: 28 layers x batch 32, 16384 generated tokens from an empty cache with the drifting
     synthetic stream (128 scheduled compressions, 120 of which evict). Sampled (layer, sequence) pairs are compared

@@ -153,6 +153,36 @@ def test_long_prompt_compression(w, h_q, h_kv, pool, lens):
     assert cache.state(0) == (b, b - w, 0) and float(cache.sacc[0].abs().max()) == 0.0
 
 
+def test_very_long_prompt_with_all_scores_equal_keeps_the_lowest_positions():
+    """A prompt of 70 000 tokens (more than fit 16-bit counters) whose keys are all zero: every logit is 0, every
+    candidate gets the same score bit for bit, and the tie rule must keep the b - w lowest positions plus the window.
+    The selection's ordered scan then counts tens of thousands of candidates equal to the threshold. A second
+    sequence with ordinary keys goes through the oracle as usual."""
+    w, h_q, h_kv, b, buffer, s = 16, 8, 2, 512, 64, 64
+    lens = [70000, 66000]
+    P_max = max(lens)
+    cfg = gkv.make_config(n_layers=1, batch=2, h_q=h_q, h_kv=h_kv, b=b, buffer=buffer, w=w, s=s, fuse_window_scores=True,
+                          track_positions=True, max_prompt=P_max)
+    cache = gkv.GKVCache(cfg, DEV)
+    kp, vp, qw = make_prompt(synth.BASE_SEED + 123, 2, h_q, h_kv, w, P_max, lens)
+    kp[0].zero_()
+    kept = torch.full((2, h_kv, b), -7, dtype=torch.int32, device=DEV)
+    cache.compress_prompt(0, kp, vp, qw, lens, kept)
+    cache.poll()
+    kept = kept.cpu().numpy()
+    want = np.concatenate([np.arange(b - w), np.arange(lens[0] - w, lens[0])])
+    for j in range(h_kv):
+        assert (kept[0, j] == want).all(), f"head {j}: equal scores must resolve toward the lowest positions"
+    assert (synth.bits(cache.v[0, 0])[:, :b] == synth.bits(vp[0])[:, want]).all()
+    np.testing.assert_allclose(cache.f[0, 0, :, : b - w].cpu().numpy(), 1.0, rtol=1e-6)   # S / max S with all S equal
+    Kp, Vp = synth.bits(kp[1]), synth.bits(vp[1])
+    ref = oracle.evict_step_full(synth.bits(qw[1]), None, Kp, Vp, None, np.zeros((h_kv, P_max), np.float32),
+                                 l=lens[1], n_h=0, b=b, w=w, alpha=0.8, mode=oracle.MODE_MAX, pool_kernel=1)
+    for j in range(h_kv):
+        assert_kept_matches(kept[1, j], ref["Fsel"][j], b, w, f"seq 1 head {j}")
+        assert (synth.bits(cache.k[0, 1, j])[:b] == Kp[j, kept[1, j]]).all()
+
+
 @pytest.mark.parametrize("pool", [0, 5])
 def test_prompt_compression_with_redundancy_term(pool):
     """With use_redundancy the first compression selects on lambda * F - (1 - lambda) * R' like every later one; the
@@ -250,7 +280,7 @@ def test_prompt_call_errors():
         with pytest.raises(gkv.GKVError) as e:
             cache.compress_prompt(0, x, x, q, lens)
         assert e.value.status == gkv.GKV_ERR_INVALID_ARG
-    for bad in (dict(max_prompt=65537), dict(max_prompt=9000, w=8)):   # too long; long prompts need a window of 16 k rows
+    for bad in (dict(max_prompt=(1 << 20) + 1), dict(max_prompt=9000, w=8)):   # too long; long prompts need a window of 16 k rows
         kw = dict(n_layers=1, batch=2, h_q=8, h_kv=2, b=64, buffer=16, w=16, s=16)
         kw.update(bad)
         with pytest.raises(gkv.GKVError) as e:

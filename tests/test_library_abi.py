@@ -55,7 +55,7 @@ def base(**over):
     (dict(d=64), gkv.GKV_ERR_UNSUPPORTED),
     (dict(h_q=32), gkv.GKV_ERR_UNSUPPORTED),         # g = 16 > 8
     (dict(b=4000, buffer=200, s=128), gkv.GKV_ERR_UNSUPPORTED),
-    (dict(max_prompt=65537), gkv.GKV_ERR_UNSUPPORTED),          # longest prompt the first compression takes
+    (dict(max_prompt=(1 << 20) + 1), gkv.GKV_ERR_UNSUPPORTED),   # longest prompt the first compression takes
     (dict(max_prompt=9000, w=24), gkv.GKV_ERR_UNSUPPORTED),     # above 8192 tokens the window is a multiple of 16
     (dict(max_prompt=-1), gkv.GKV_ERR_INVALID_ARG),
 ])

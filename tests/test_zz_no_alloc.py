@@ -10,6 +10,7 @@ import torch
 import paper_2512_00504_b200 as gkv
 from paper_2512_00504_b200 import synth
 
+import oracle
 from parity import DECODE_ATOL
 
 pytestmark = pytest.mark.gpu
@@ -17,7 +18,7 @@ DEV = "cuda:0"
 
 
 @pytest.mark.parametrize("shape", [
-    dict(batch=2, h_q=8, h_kv=2, b=160, buffer=40, w=8, s=40),     # few units: keys split over CTAs (scratch in use)
+    dict(batch=2, h_q=8, h_kv=2, b=160, buffer=40, w=8, s=40),     # few units: the keys of a unit are split over a cluster of CTAs
     dict(batch=96, h_q=28, h_kv=4, b=100, buffer=28, w=8, s=28),   # 384 units: one CTA per unit
 ])
 def test_static_scratch_decode_matches_context_decode(shape):
@@ -41,6 +42,11 @@ def test_static_scratch_decode_matches_context_decode(shape):
         diff = (out_ctx.float() - out_sta.float()).abs().max().item()
         assert diff < DECODE_ATOL, (step, diff)
         assert torch.equal(cache.k[0], k2) and torch.equal(cache.v[0], v2)   # the appended rows match
+        # ... and against the definition, not only against the other entry point (a sample of the sequences)
+        seqs = sorted({0, B // 2, B - 1})
+        ref = oracle.decode_batch(synth.bits(q[seqs]), synth.bits(k2[seqs]), synth.bits(v2[seqs]), start + step + 1)
+        err = float(abs(out_sta[seqs].float().cpu().numpy() - ref).max())
+        assert err < DECODE_ATOL, (step, err)
     cache.poll()
 
 
