@@ -151,6 +151,8 @@ EvictLaunch make_evict(gkv_ctx* ctx, int l0, int nl, int32_t* kept_out) {
     p.kept_ws = ws_ptr<int32_t>(ctx, ctx->ws.kept);
     p.f_ws = ws_ptr<float>(ctx, ctx->ws.fscratch);
     p.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
+    p.work = p.status + 34;       // (the decode kernel's counters are words 32 and 33)
+    p.sm_count = ctx->sm_count;
     p.layer0 = l0; p.n_layers = nl; p.L_total = c.n_layers; p.batch = c.batch; p.h_kv = c.n_kv_heads;
     p.C = ctx->C; p.b = c.budget; p.w = c.window; p.alpha = c.alpha; p.mode = c.mode;
     p.evict_log = ctx->evict_log;

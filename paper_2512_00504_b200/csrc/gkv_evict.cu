@@ -2,12 +2,21 @@
 // history into the global score (Section 5, Eq. 3-5), select the top-(b-w) candidates per KV head
 // (ties toward the lower position), and compact K, V, F and pos in place.
 //
-// One CTA owns one unit (layer, sequence, KV head). All per-row score state of a unit (at most
-// C <= 4096 rows) lives in shared memory. The selection is a 4-pass radix select on the fp32 bit
-// patterns (scores are >= 0, so they order as unsigned integers) followed by one ordered scan that
-// assigns destinations. The compaction moves rows in ascending order, a group of rows fully loaded
-// into registers before any of them is stored: a row's destination never lies above its source,
-// so earlier groups can only overwrite rows that are already consumed.
+// A unit is one (layer, sequence, KV head). All per-row score state of a unit (at most C <= 4096
+// rows) lives in shared memory. The selection is a radix select on the fp32 bit patterns (mapped so
+// that they order as unsigned integers) followed by one ordered scan that assigns destinations.
+//
+// The fused kernel is persistent and warp-specialised: eight "selection" warps take units from a
+// device-wide counter and produce each unit's kept list; a ninth "copy" warp moves the rows of the
+// unit before, so the selection of one unit (latency-bound: a few dependent passes over a few
+// thousand scores) runs while the copy engine streams the rows of another. The copy warp gathers
+// the rows of 32 consecutive destination rows into a shared-memory stage with bulk copies
+// (cp.async.bulk global -> shared, consecutive source rows merged into one copy) and writes the
+// stage to its contiguous destination with one bulk copy per tensor; no row passes through
+// registers and no CTA-wide barrier sits in the copy loop. In place is safe because kept[r] >= r
+// and kept is ascending: a group's destination ends below the sources of every later group, and
+// the rows a group overwrites are sources of that group or of earlier ones, whose loads have
+// completed before the group is stored.
 #include "gkv_common.cuh"
 #include "gkv_internal.h"
 
@@ -15,6 +24,10 @@ namespace gkv {
 
 constexpr int kEvictThreads = 256;
 constexpr int kCompactUnroll = 4;
+
+// Barrier among the 256 threads that run the score phases (all threads of the staged and prompt kernels; the
+// selection warps of the fused kernel, whose copy warp does not take part).
+__device__ __forceinline__ void sel_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 struct EvictShared {
     int hist[256];
@@ -32,11 +45,11 @@ __device__ __forceinline__ int block_incl_scan(int v, int* warp_sums, int tid) {
         if (lane >= o) v += t;
     }
     if (lane == 31) warp_sums[warp] = v;
-    __syncthreads();
+    sel_sync();
     int base = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) base += (i < warp) ? warp_sums[i] : 0;
-    __syncthreads();
+    sel_sync();
     return v + base;
 }
 
@@ -49,14 +62,14 @@ __device__ __forceinline__ int2 block_incl_scan2(int a, int b, int* warp_sums, i
         if (lane >= o) { a += ta; b += tb; }
     }
     if (lane == 31) { warp_sums[warp] = a; warp_sums[8 + warp] = b; }
-    __syncthreads();
+    sel_sync();
     int base_a = 0, base_b = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         base_a += (i < warp) ? warp_sums[i] : 0;
         base_b += (i < warp) ? warp_sums[8 + i] : 0;
     }
-    __syncthreads();
+    sel_sync();
     return make_int2(a + base_a, b + base_b);
 }
 
@@ -64,18 +77,18 @@ __device__ __forceinline__ float block_max(float v, float* warp_max, int tid) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
     if ((tid & 31) == 0) warp_max[tid >> 5] = v;
-    __syncthreads();
+    sel_sync();
     float r = warp_max[0];
 #pragma unroll
     for (int i = 1; i < 8; ++i) r = fmaxf(r, warp_max[i]);
-    __syncthreads();
+    sel_sync();
     return r;
 }
 
 // Section 5: S_hat = S / max S over the n_c candidates; F = merge(alpha * F_prev, S_hat) on the
 // n_h rows with history, F = S_hat elsewhere. `s_f` receives F for t < n_c.
 // `sums` holds w * S (the 1/w of Eq. 2 cancels in the normalisation).
-__device__ void merge_phase(const float* __restrict__ sums, const float* __restrict__ f_prev, float* s_f,
+__device__ void merge_phase(const float* sums, const float* f_prev, float* s_f,
                             int n_c, int n_h, float alpha, int mode, EvictShared* sh, int tid) {
     float mx = 0.f;
     for (int t = tid; t < n_c; t += kEvictThreads) {
@@ -95,7 +108,7 @@ __device__ void merge_phase(const float* __restrict__ sums, const float* __restr
         }
         s_f[t] = f;
     }
-    __syncthreads();
+    sel_sync();
 }
 
 // Appendix on combining the global score with other methods, SnapKV: sequence-wise max-pooling of the score
@@ -107,7 +120,7 @@ __device__ void pool_phase(const float* s_f, float* s_sel, int n_c, int kernel, 
         for (int u = max(t - half, 0); u <= min(t + half, n_c - 1); ++u) m = fmaxf(m, s_f[u]);
         s_sel[t] = m;
     }
-    __syncthreads();
+    sel_sync();
 }
 
 // Same appendix, redundancy term: R = softmax(cbar), R' = R / max R = exp(cbar - max cbar) (maximum over all
@@ -119,7 +132,7 @@ __device__ void combine_phase(const float* __restrict__ cbar, const float* s_in,
     mx = block_max(mx, sh->warp_max, tid);
     for (int t = tid; t < n_c; t += kEvictThreads)
         s_sel[t] = lambda * s_in[t] - (1.f - lambda) * fast_exp2((cbar[t] - mx) * 1.4426950408889634f);
-    __syncthreads();
+    sel_sync();
 }
 
 // F in s_f -> the scores the selection runs on in s_sel (s_sel == s_f when no optional term is on):
@@ -141,32 +154,49 @@ __device__ __forceinline__ uint32_t ordered_bits(uint32_t x) {
 // Top-n_keep of s_f[0..n_c) with ties toward the lower index; kept rows ascending into s_kept,
 // followed by the w window rows n_c .. n_c+w-1. Returns (CTA-uniform) the first row that moves.
 // s_evict (may be NULL) receives the n_c - n_keep evicted rows in ascending order.
-__device__ int select_phase(const float* s_f, int* s_kept, int* s_evict, int n_c, int n_keep, int w, EvictShared* sh,
+template <typename KT>   // element type of the kept list: int, or uint16_t where rows are known to be < 65536
+__device__ int select_phase(const float* s_f, KT* s_kept, int* s_evict, int n_c, int n_keep, int w, EvictShared* sh,
                             int tid) {
     const uint32_t* bits = reinterpret_cast<const uint32_t*>(s_f);
+    const int lane = tid & 31;
     uint32_t prefix = 0;
     int k = n_keep;
+    sh->hist[tid] = 0;
+    sel_sync();
+    // Radix select, 8 bits a pass from the top: the histogram of the candidates that match the prefix found so far,
+    // a scan from the top digit down, and the digit that holds the k-th largest joins the prefix. Scores crowd into a
+    // few top digits (same sign and exponent), so equal digits within a warp are counted once (match) and added with
+    // one atomic. A pass whose digit holds exactly the k candidates still wanted ends the search early: all of them
+    // are kept, whatever their lower bits.
 #pragma unroll 1
     for (int shift = 24; shift >= 0; shift -= 8) {
-        sh->hist[tid] = 0;
-        __syncthreads();
         const uint32_t mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
-        for (int t = tid; t < n_c; t += kEvictThreads) {
-            const uint32_t x = ordered_bits(bits[t]);
-            if ((x & mask) == prefix) atomicAdd(&sh->hist[(x >> shift) & 255], 1);
+        for (int t0 = 0; t0 < n_c; t0 += kEvictThreads) {
+            const int t = t0 + tid;
+            const uint32_t x = (t < n_c) ? ordered_bits(bits[t]) : 0u;
+            const bool in = t < n_c && (x & mask) == prefix;
+            const uint32_t d = in ? ((x >> shift) & 255u) : 256u;
+            const uint32_t peers = __match_any_sync(0xffffffffu, d);
+            if (in && (peers & ((1u << lane) - 1u)) == 0u) atomicAdd(&sh->hist[d], __popc(peers));
         }
-        __syncthreads();
-        // thread tid looks at digit 255 - tid; `ge` = number of matching elements with digit >= mine
+        sel_sync();
+        // thread tid looks at digit 255 - tid (and clears it for the next pass); `ge` = matching elements with digit >= mine
         const int mine = sh->hist[255 - tid];
+        sh->hist[255 - tid] = 0;
         const int ge = block_incl_scan(mine, sh->warp_sums, tid);
         const int gt = ge - mine;
         if (ge >= k && gt < k) {  // exactly one digit holds the k-th largest
             sh->digit = 255 - tid;
             sh->k_rem = k - gt;
+            sh->is_last = (mine == k - gt);
         }
-        __syncthreads();
+        sel_sync();
         prefix |= static_cast<uint32_t>(sh->digit) << shift;
         k = sh->k_rem;
+        if (sh->is_last) {      // (CTA-uniform) every candidate of this digit is kept: threshold = the digit's lowest pattern
+            k = n_c;
+            break;
+        }
     }
     // prefix = ordered bit pattern T of the n_keep-th largest score; take everything above it and the
     // first k rows equal to it
@@ -188,10 +218,10 @@ __device__ int select_phase(const float* s_f, int* s_kept, int* s_evict, int n_c
         const int kept_before = gt_before + min(eq_before, k);   // kept rows below t
         bool dropped = false;
         if (x > T) {
-            s_kept[kept_before] = t;
+            s_kept[kept_before] = (KT)t;
             ++gt_before;
         } else if (x == T) {
-            if (eq_before < k) s_kept[kept_before] = t;
+            if (eq_before < k) s_kept[kept_before] = (KT)t;
             else dropped = true;
             ++eq_before;
         } else {
@@ -203,8 +233,8 @@ __device__ int select_phase(const float* s_f, int* s_kept, int* s_evict, int n_c
         }
     }
     if (first_drop < n_c) atomicMin(&sh->first_evicted, first_drop);
-    for (int r = tid; r < w; r += kEvictThreads) s_kept[n_keep + r] = n_c + r;
-    __syncthreads();
+    for (int r = tid; r < w; r += kEvictThreads) s_kept[n_keep + r] = (KT)(n_c + r);
+    sel_sync();
     return sh->first_evicted;
 }
 
@@ -312,7 +342,8 @@ __device__ __forceinline__ UnitIndex unit_of(const EvictLaunch& p, int unit_loca
 }
 
 // Record the per-row state after selection: compact F and pos, clear the window sums, export kept.
-__device__ void write_score_state(const EvictLaunch& p, const UnitIndex& u, const float* s_f, const int* s_kept,
+template <typename KT>
+__device__ void write_score_state(const EvictLaunch& p, const UnitIndex& u, const float* s_f, const KT* s_kept,
                                   int* s_pos, const int* s_evict, int n, int tid) {
     const int n_keep = p.b - p.w;
     float* f = p.f + (size_t)u.unit * p.C;
@@ -320,7 +351,7 @@ __device__ void write_score_state(const EvictLaunch& p, const UnitIndex& u, cons
     if (p.pos) {
         int32_t* pos = p.pos + (size_t)u.unit * p.C;
         for (int t = tid; t < n; t += kEvictThreads) s_pos[t] = pos[t];
-        __syncthreads();
+        sel_sync();
         for (int r = tid; r < p.b; r += kEvictThreads) pos[r] = s_pos[s_kept[r]];
     }
     if (p.evict_log) {   // what left the cache: original positions when they are tracked, else pre-compaction rows
@@ -350,51 +381,280 @@ __device__ void publish_state(const EvictLaunch& p, const UnitIndex& u, int ctas
     }
 }
 
-// s_sel (the scores the selection runs on) is s_f itself unless the redundancy term is on.
+// s_sel (the scores the selection runs on) is s_f itself unless an optional term is on. `kept_bufs` kept lists
+// of b entries follow the scores (two in the fused kernel: one being produced, one being copied from).
 __device__ __forceinline__ void carve(uint8_t* smem, const EvictLaunch& p, float** s_f, int** s_kept, int** s_pos,
-                                      EvictShared** sh, float** s_sel, int** s_evict) {
+                                      EvictShared** sh, float** s_sel, int** s_evict, int kept_bufs = 1) {
     *sh = reinterpret_cast<EvictShared*>(smem);
     *s_f = reinterpret_cast<float*>(smem + sizeof(EvictShared));
     *s_kept = reinterpret_cast<int*>(*s_f + p.C);
-    *s_pos = *s_kept + p.b;
+    *s_pos = *s_kept + kept_bufs * p.b;
     const bool terms = p.cbar != nullptr || p.pool_kernel > 1;
     *s_sel = terms ? reinterpret_cast<float*>(*s_pos + (p.pos ? p.C : 0)) : *s_f;
     *s_evict = p.evict_log ? *s_pos + (p.pos ? p.C : 0) + (terms ? p.C : 0) : nullptr;
 }
-static size_t evict_state_bytes(const EvictLaunch& p) {
-    return sizeof(EvictShared) + sizeof(float) * p.C + sizeof(int) * p.b + (p.pos ? sizeof(int) * p.C : 0) +
+static size_t evict_state_bytes(const EvictLaunch& p, int kept_bufs = 1) {
+    return sizeof(EvictShared) + sizeof(float) * p.C + sizeof(int) * p.b * kept_bufs + (p.pos ? sizeof(int) * p.C : 0) +
            ((p.cbar || p.pool_kernel > 1) ? sizeof(float) * p.C : 0) + (p.evict_log ? sizeof(int) * (p.C - p.b) : 0);
 }
 static size_t evict_smem_bytes(const EvictLaunch& p) { return evict_state_bytes(p); }
-// the fused kernel adds the copy ring, 128-byte aligned behind the score state
-static size_t evict_ring_offset(const EvictLaunch& p) { return (evict_state_bytes(p) + 127) & ~size_t(127); }
 
 // ---------------------------------------------------------------------------------------------
-// Whole step in one launch: merge -> select -> score-state update -> K/V compaction.
-__global__ void __launch_bounds__(kEvictThreads) gkv_evict_fused_kernel(const EvictLaunch p, int ring_offset) {
-    extern __shared__ __align__(128) uint8_t evict_smem[];
-    float* s_f; int* s_kept; int* s_pos; EvictShared* sh; float* s_sel; int* s_evict;
-    carve(evict_smem, p, &s_f, &s_kept, &s_pos, &sh, &s_sel, &s_evict);
-    const int tid = threadIdx.x;
-    const UnitIndex u = unit_of(p, blockIdx.x);
-    const int n = p.len[u.lseq_global];
-    const int n_h = p.len[(size_t)p.L_total * p.batch + u.lseq_global];
-    if (n <= p.b) {  // nothing to evict: only the window sums restart
-        float* sacc = p.sacc + (size_t)u.unit * p.C;
-        for (int t = tid; t < p.C; t += kEvictThreads) sacc[t] = 0.f;
-        if (p.evict_log)
-            for (int e = tid; e < p.C - p.b; e += kEvictThreads) p.evict_log[(size_t)u.unit * (p.C - p.b) + e] = -1;
-        return;
+// Whole step in one launch: merge -> select -> score-state update on the selection warps, K/V compaction on the
+// copy warp, one unit behind.
+constexpr int kFusedThreads = kEvictThreads + 32;
+constexpr int kFusedMaxStages = 8;
+
+struct __align__(16) FusedPipe {
+    uint64_t kept_full[2];    // selection -> copy: the kept list in buffer i is complete (tid 0 arrives)
+    uint64_t kept_empty[2];   // copy -> selection: every load that reads buffer i has been issued
+    uint64_t taken[2];        // copy -> selection: the copy warp has started on the list in buffer i
+    uint64_t ring_full[kFusedMaxStages];   // the rows of a stage have landed
+    long unit[2];             // the unit whose kept list is in buffer i, or -1: no more
+    int r_first[2];           // first destination row that moves
+    uint32_t dst_row[kFusedMaxStages];     // per stage: first destination row (in rows of the whole K / V tensor), rows held
+    int n_rows[kFusedMaxStages];
+    int cur_item, abort_flag, is_last, go;
+};
+
+// Shared memory of the fused kernel (byte offsets): the selection warps' score arrays, two kept lists of b 16-bit
+// rows (one being produced, one being copied from; C <= 4096), the hand-over structure, the copy ring.
+struct FusedLayout {
+    int f, fp, sel, pos, evict, kept, pipe, ring;
+};
+__host__ __device__ inline FusedLayout fused_layout(int C, int b, bool terms, bool has_pos, bool has_log) {
+    FusedLayout l;
+    int off = (int)sizeof(EvictShared);
+    l.f = off;      off += 4 * C;                       // F (the sums arrive here first)
+    l.fp = off;     off += 4 * C;                       // F_prev
+    l.sel = terms ? off : l.f;   off += terms ? 4 * C : 0;
+    l.pos = off;    off += has_pos ? 4 * C : 0;
+    l.evict = off;  off += has_log ? 4 * (C - b) : 0;
+    l.kept = off;   off += 2 * 2 * b;
+    l.pipe = (off + 15) & ~15;
+    l.ring = (l.pipe + (int)sizeof(FusedPipe) + 127) & ~127;
+    return l;
+}
+
+__device__ __forceinline__ bool evict_wait(uint32_t bar, uint32_t parity, const int* abort_flag) {
+    for (uint32_t i = 0; i < kWaitSpins; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*(volatile const int*)abort_flag) return false;
+        if (i > 64) __nanosleep(64);
     }
-    const int n_c = n - p.w;
-    merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
-    selection_scores(p, u.unit, s_f, s_sel, n, n_c, sh, tid);
-    const int r_first = select_phase(s_sel, s_kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
-    write_score_state(p, u, s_f, s_kept, s_pos, s_evict, n, tid);
-    __nv_bfloat16* kb = p.k_cache + (size_t)u.unit * p.C * kHeadDim;
-    __nv_bfloat16* vb = p.v_cache + (size_t)u.unit * p.C * kHeadDim;
-    compact_phase_async(kb, vb, kb, vb, s_kept, p.b, r_first, evict_smem + ring_offset, tid);
-    publish_state(p, u, p.h_kv, sh, tid);
+    return false;
+}
+__device__ __forceinline__ void evict_abort(FusedPipe* pipe, int32_t* status, int where) {
+    if (atomicExch(&pipe->abort_flag, 1) == 0 && atomicCAS(status, 0, kStatusTimeout) == 0) {
+        status[1] = where;
+        status[2] = blockIdx.x;
+    }
+}
+
+__global__ void __launch_bounds__(kFusedThreads, 5) gkv_evict_fused_kernel(const EvictLaunch p, int stages) {
+    extern __shared__ __align__(128) uint8_t evict_smem[];
+    const FusedLayout lay = fused_layout(p.C, p.b, has_selection_terms(p), p.pos != nullptr, p.evict_log != nullptr);
+    EvictShared* sh = reinterpret_cast<EvictShared*>(evict_smem);
+    float* s_f = reinterpret_cast<float*>(evict_smem + lay.f);
+    float* s_fp = reinterpret_cast<float*>(evict_smem + lay.fp);
+    float* s_sel = reinterpret_cast<float*>(evict_smem + lay.sel);
+    int* s_pos = reinterpret_cast<int*>(evict_smem + lay.pos);
+    int* s_evict = p.evict_log ? reinterpret_cast<int*>(evict_smem + lay.evict) : nullptr;
+    uint16_t* s_kept = reinterpret_cast<uint16_t*>(evict_smem + lay.kept);
+    FusedPipe* pipe = reinterpret_cast<FusedPipe*>(evict_smem + lay.pipe);
+    uint8_t* ring = evict_smem + lay.ring;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int total = p.n_layers * p.batch * p.h_kv;
+
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&pipe->kept_full[i]), 1);
+            mbar_init(smem_u32(&pipe->kept_empty[i]), 1);
+            mbar_init(smem_u32(&pipe->taken[i]), 1);
+        }
+        for (int s = 0; s < stages; ++s) mbar_init(smem_u32(&pipe->ring_full[s]), 1);
+        pipe->abort_flag = 0;
+        pipe->is_last = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    if (warp < kEvictThreads / 32) {
+        // ------------------------------------------------------------------ selection warps
+        int handed = 0;      // units handed to the copy warp so far
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+            // Units are handed out first come, first served: this CTA's index first, then numbers from a device-wide
+            // counter. The barrier also ends the previous unit's use of the score arrays.
+            // A CTA asks for its next unit only once its copy warp has started on the unit before: it then holds one
+            // unit in the copy and one in the selection, not three, and the units go to the CTAs that get through
+            // them fastest.
+            if (tid == 0) {
+                int item = -1;
+                if (handed == 0 || evict_wait(smem_u32(&pipe->taken[(handed - 1) & 1]), ((handed - 1) >> 1) & 1, &pipe->abort_flag))
+                    item = (k == 0) ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(p.work, 1);
+                else
+                    evict_abort(pipe, p.status, 40);
+                pipe->cur_item = item < total ? item : -1;
+            }
+            sel_sync();
+            const int item = *(volatile int*)&pipe->cur_item;
+            if (item < 0) break;
+            const UnitIndex u = unit_of(p, item);
+            // The unit's window sums and recorded scores start their way into shared memory at once (all C entries:
+            // the length is not known yet), so the length, the sums and the scores cost one memory round trip, not three.
+            {
+                const float* gs = p.sacc + (size_t)u.unit * p.C;
+                const float* gf = p.f + (size_t)u.unit * p.C;
+                for (int t = tid; t < p.C; t += kEvictThreads) {
+                    cp_async_4(smem_u32(s_f + t), gs + t);
+                    cp_async_4(smem_u32(s_fp + t), gf + t);
+                }
+                cp_async_commit();
+            }
+            const int n = p.len[u.lseq_global];
+            const int n_h = p.len[(size_t)p.L_total * p.batch + u.lseq_global];
+            cp_async_wait_all();
+            sel_sync();
+            if (n <= p.b) {  // nothing to evict: only the window sums restart
+                float* sacc = p.sacc + (size_t)u.unit * p.C;
+                for (int t = tid; t < p.C; t += kEvictThreads) sacc[t] = 0.f;
+                if (p.evict_log)
+                    for (int e = tid; e < p.C - p.b; e += kEvictThreads) p.evict_log[(size_t)u.unit * (p.C - p.b) + e] = -1;
+                continue;
+            }
+            const int buf = handed & 1;
+            uint16_t* kept = s_kept + buf * p.b;
+            const int n_c = n - p.w;
+            merge_phase(s_f, s_fp, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
+            selection_scores(p, u.unit, s_f, s_sel, n, n_c, sh, tid);
+            // the copy warp has issued every load that reads this buffer's previous list (two units ago)
+            if (handed >= 2) {   // one thread waits, the barrier hands its verdict (and the ordering) to the others
+                if (tid == 0) pipe->go = evict_wait(smem_u32(&pipe->kept_empty[buf]), ((handed >> 1) - 1) & 1, &pipe->abort_flag);
+                sel_sync();
+                if (!*(volatile int*)&pipe->go) { evict_abort(pipe, p.status, 41); break; }
+            }
+            const int r_first = select_phase(s_sel, kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
+            if (tid == 0) {
+                pipe->unit[buf] = u.unit;
+                pipe->r_first[buf] = r_first;
+                mbar_arrive(smem_u32(&pipe->kept_full[buf]));
+            }
+            ++handed;
+            write_score_state(p, u, s_f, kept, s_pos, s_evict, n, tid);
+        }
+        // the end of the list: a buffer that carries -1
+        if (tid == 0 && !*(volatile int*)&pipe->abort_flag) {
+            const int buf = handed & 1;
+            if (handed < 2 || evict_wait(smem_u32(&pipe->kept_empty[buf]), ((handed >> 1) - 1) & 1, &pipe->abort_flag)) {
+                pipe->unit[buf] = -1;
+                mbar_arrive(smem_u32(&pipe->kept_full[buf]));
+            } else {
+                evict_abort(pipe, p.status, 42);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ copy warp
+        const int D = stages - 2;                      // groups of loads in flight
+        const uint32_t ring_addr = smem_u32(ring);
+        uint32_t G = 0, stored = 0;                    // ring groups loaded / stored so far, across units
+        bool ok = true;
+        // store ring group `stored`: its rows have landed (and with them every row loaded before)
+        auto store_next = [&]() {
+            const int st = stored % stages;
+            if (!evict_wait(smem_u32(&pipe->ring_full[st]), (stored / stages) & 1, &pipe->abort_flag)) {
+                evict_abort(pipe, p.status, 44);
+                ok = false;
+                return;
+            }
+            if (lane == 0) {
+                const uint32_t src = ring_addr + (uint32_t)st * kCopyStageBytes;
+                const uint32_t bytes = (uint32_t)pipe->n_rows[st] * kRowBytes;
+                const size_t dst = (size_t)pipe->dst_row[st] * kHeadDim;
+                bulk_store(p.k_cache + dst, src, bytes);
+                bulk_store(p.v_cache + dst, src + kCopyRows * kRowBytes, bytes);
+                bulk_commit();
+            }
+            ++stored;
+        };
+        for (int k = 0; ok; ++k) {
+            const int buf = k & 1;
+            // while the next list is not there yet, the groups already loaded go out
+            while (ok && stored < G && !mbar_try_wait(smem_u32(&pipe->kept_full[buf]), (k >> 1) & 1)) store_next();
+            if (!ok) break;
+            if (!evict_wait(smem_u32(&pipe->kept_full[buf]), (k >> 1) & 1, &pipe->abort_flag)) {
+                evict_abort(pipe, p.status, 43);
+                break;
+            }
+            const long unit = *(volatile long*)&pipe->unit[buf];
+            if (unit < 0) break;
+            const int r_first = *(volatile int*)&pipe->r_first[buf];
+            if (lane == 0) mbar_arrive(smem_u32(&pipe->taken[buf]));
+            const uint16_t* kept = s_kept + buf * p.b;
+            const uint4* k4 = reinterpret_cast<const uint4*>(p.k_cache + (size_t)unit * p.C * kHeadDim);
+            const uint4* v4 = reinterpret_cast<const uint4*>(p.v_cache + (size_t)unit * p.C * kHeadDim);
+            for (int r0 = r_first; r0 < p.b && ok; r0 += kCopyRows, ++G) {
+                const int st = G % stages;
+                // the stage was last read by the store of ring group G - stages; stores issued so far: groups < `stored`
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
+                const int rows = min(kCopyRows, p.b - r0);
+                const uint32_t bar = smem_u32(&pipe->ring_full[st]);
+                if (lane == 0) {
+                    pipe->dst_row[st] = (uint32_t)(unit * p.C + r0);
+                    pipe->n_rows[st] = rows;
+                    mbar_arrive_expect_tx(bar, (uint32_t)rows * 2 * kRowBytes);
+                }
+                __syncwarp();
+                // lane i owns destination row r0 + i; runs of consecutive source rows travel as one copy
+                const bool valid = lane < rows;
+                const int src = valid ? (int)kept[r0 + lane] : -2;
+                const int prev = __shfl_up_sync(0xffffffffu, src, 1);
+                const bool start = valid && (lane == 0 || src != prev + 1);
+                const uint32_t starts = __ballot_sync(0xffffffffu, start);
+                if (start) {
+                    const uint32_t rest = (lane == 31) ? 0u : (starts >> (lane + 1));
+                    const int run = rest ? __ffs(rest) : rows - lane;
+                    const uint32_t dst = ring_addr + (uint32_t)st * kCopyStageBytes + (uint32_t)lane * kRowBytes;
+                    bulk_load(dst, k4 + (size_t)src * 16, (uint32_t)run * kRowBytes, bar);
+                    bulk_load(dst + kCopyRows * kRowBytes, v4 + (size_t)src * 16, (uint32_t)run * kRowBytes, bar);
+                }
+                if (G >= (uint32_t)D + stored) store_next();   // keeps D groups of loads in flight
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&pipe->kept_empty[buf]));
+        }
+        while (ok && stored < G) store_next();
+        if (!ok || *(volatile int*)&pipe->abort_flag) {
+            // loads still in flight get a bounded time to land before the CTA exits
+            for (uint32_t g = stored; g < G; ++g) mbar_wait_bounded(smem_u32(&pipe->ring_full[g % stages]), (g / stages) & 1);
+        }
+        if (lane == 0) bulk_wait<0>();                 // all rows written
+    }
+
+    __syncthreads();
+    // The last CTA to finish puts the two counters back to zero and publishes the new state of every sequence of the
+    // launch that was compressed: len = b, n_hist = b - w. (No CTA may do that for its own sequence earlier: the other
+    // KV heads of the sequence read the old length when they start.)
+    if (tid == 0) {
+        __threadfence();
+        pipe->is_last = atomicAdd(p.work + 1, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (pipe->is_last) {
+        const int n_seq = p.n_layers * p.batch;
+        for (int ls = tid; ls < n_seq; ls += kFusedThreads) {
+            const int lseq = p.layer0 * p.batch + ls;
+            if (p.len[lseq] > p.b) {
+                p.len[lseq] = p.b;
+                p.len[(size_t)p.L_total * p.batch + lseq] = p.b - p.w;
+            }
+        }
+        if (tid == 0) {
+            p.work[0] = 0;
+            p.work[1] = 0;
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -545,12 +805,42 @@ static cudaError_t ensure_smem(const void* fn, size_t bytes) {
     return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
+// Launch shape of the fused kernel. Ring depth: the one that keeps the most groups of loads in flight per SM
+// (resident CTAs x (stages - 2)); among equals the one with more CTAs, whose selection phases then hide each other.
+// Grid: persistent, at most the resident CTAs; with three rounds of units or fewer the rounds are filled equally
+// (512 units on 296 slots run as 256 CTAs x 2 units: a unit cannot be split, and a CTA holding two units next to
+// CTAs holding one sets the end of the launch).
+void evict_plan(const EvictLaunch& p, int* stages, int* grid, size_t* smem) {
+    const FusedLayout lay = fused_layout(p.C, p.b, p.cbar != nullptr || p.pool_kernel > 1, p.pos != nullptr, p.evict_log != nullptr);
+    auto ctas_with = [&](int st) {
+        const int by_smem = (int)((227 * 1024) / ((size_t)lay.ring + (size_t)st * kCopyStageBytes + 1024));
+        return by_smem > 5 ? 5 : by_smem;
+    };
+    int st = 3, best = -1;
+    for (int c = 3; c <= kFusedMaxStages; ++c) {
+        const int score = ctas_with(c) * (c - 2) * 8 + ctas_with(c);
+        if (ctas_with(c) >= 1 && score > best) { best = score; st = c; }
+    }
+    const int sm = p.sm_count > 0 ? p.sm_count : 148;
+    const long total = (long)p.n_layers * p.batch * p.h_kv;
+    const long resident = (long)max(1, ctas_with(st)) * sm;
+    long g = total < resident ? total : resident;
+    if (total > resident) {
+        const long rounds = (total + resident - 1) / resident;
+        if (rounds <= 3) g = (total + rounds - 1) / rounds;
+    }
+    *stages = st;
+    *grid = (int)g;
+    *smem = (size_t)lay.ring + (size_t)st * kCopyStageBytes;
+}
+
 cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s) {
-    const size_t ring = evict_ring_offset(p);
-    const size_t smem = ring + kCopyRingBytes;
+    int stages, grid;
+    size_t smem;
+    evict_plan(p, &stages, &grid, &smem);
     cudaError_t e = ensure_smem((const void*)gkv_evict_fused_kernel, smem);
     if (e != cudaSuccess) return e;
-    gkv_evict_fused_kernel<<<p.n_layers * p.batch * p.h_kv, kEvictThreads, smem, s>>>(p, (int)ring);
+    gkv_evict_fused_kernel<<<grid, kFusedThreads, smem, s>>>(p, stages);
     return cudaGetLastError();
 }
 cudaError_t launch_prompt_compress(const PromptLaunch& p, cudaStream_t s) {

@@ -69,6 +69,8 @@ struct EvictLaunch {
     int32_t* kept_ws;    // staged path scratch
     float* f_ws;         // staged path scratch
     int32_t* status;
+    int32_t* work;       // two zeroed words of the fused kernel: the next unit's number minus the grid size, CTAs done
+    int sm_count;        // SMs of the device (sizes the fused kernel's persistent grid)
     int layer0, n_layers, L_total, batch, h_kv, C, b, w;
     float alpha;
     int mode;
