@@ -209,7 +209,7 @@ gkv_status launch_score_for(gkv_ctx* ctx, int l0, int nl, const void* q_window, 
     sp.len = static_cast<const int32_t*>(ctx->buf.len);
     sp.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
     sp.layer0 = l0; sp.n_layers = nl; sp.batch = c.batch; sp.h_q = c.n_q_heads; sp.h_kv = c.n_kv_heads;
-    sp.g = ctx->g; sp.C = ctx->C; sp.w = c.window;
+    sp.g = ctx->g; sp.C = ctx->C; sp.w = c.window; sp.sm_count = ctx->sm_count;
     sp.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
     return dispatch_score(ctx, sp, ctx->tm_k, s);
 }
@@ -622,7 +622,7 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
         sp.len = d_len;
         sp.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
         sp.layer0 = 0; sp.n_layers = 1; sp.batch = c.batch; sp.h_q = c.n_q_heads; sp.h_kv = c.n_kv_heads;
-        sp.g = ctx->g; sp.C = c.max_prompt; sp.w = c.window;
+        sp.g = ctx->g; sp.C = c.max_prompt; sp.w = c.window; sp.sm_count = ctx->sm_count;
         sp.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
         const gkv_status st = dispatch_score(ctx, sp, tm_kp, s);
         if (st != GKV_OK) {

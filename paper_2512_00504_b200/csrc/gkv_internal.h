@@ -119,6 +119,7 @@ struct ScoreLaunch {
     const int32_t* len;
     int32_t* status;
     int layer0, n_layers, batch, h_q, h_kv, g, C, w;
+    int sm_count;                // SMs of the device (sizes the tensor-core kernel's persistent grid)
     float scale_log2;
 };
 
