@@ -47,6 +47,7 @@ def lib() -> ctypes.CDLL:
         _lib.gkvo_evict_step.restype = ctypes.c_int
         _lib.gkvo_evict_step_redundancy.restype = ctypes.c_int
         _lib.gkvo_evict_step_full.restype = ctypes.c_int
+        _lib.gkvo_evict_step_streaming.restype = ctypes.c_int
     return _lib
 
 
@@ -217,6 +218,28 @@ def evict_step_full(Q_win, S_in, K, V, pos, F_prev, *, l, n_h, b, w, alpha, mode
         int(lam is not None), ctypes.c_double(1.0 if lam is None else lam), ctypes.c_double(tau), int(recent),
         ctypes.c_double(eps), _p(out["F"], np.float64), _p(out["Fsel"], np.float64), _p(out["kept"], np.int32),
         _p(out["K"], np.uint16), _p(out["V"], np.uint16), _p(out["pos"], np.int32), _p(out["F_state"], np.float64)))
+    return out
+
+
+def streaming_select(h_kv, l, b, n_sink):
+    """Sink-plus-recent policy: the first n_sink rows and the most recent b - n_sink, ascending. [h_kv][b]."""
+    assert l > b and 0 <= n_sink <= b
+    kept = np.empty((h_kv, b), np.int32)
+    lib().gkvo_streaming_select(h_kv, l, b, n_sink, _p(kept, np.int32))
+    return kept
+
+
+def evict_step_streaming(K, V, pos, *, l, b, w, n_sink):
+    """One compression step under the sink-plus-recent policy. K, V [h_kv][C][d] uint16; pos [h_kv][C] int32 or None."""
+    h_kv, C, d = K.shape
+    if l <= b:
+        return {"len": l, "evicted": False}
+    out = {"kept": np.empty((h_kv, b), np.int32), "K": np.zeros_like(K), "V": np.zeros_like(V),
+           "pos": None if pos is None else np.zeros_like(pos), "F_state": np.zeros((h_kv, C), np.float64)}
+    out["len"] = int(lib().gkvo_evict_step_streaming(_p(K, np.uint16), _p(V, np.uint16), _p(pos, np.int32), h_kv, d, C, l, b, w,
+                                                     n_sink, _p(out["kept"], np.int32), _p(out["K"], np.uint16),
+                                                     _p(out["V"], np.uint16), _p(out["pos"], np.int32), _p(out["F_state"], np.float64)))
+    out["evicted"] = True
     return out
 
 

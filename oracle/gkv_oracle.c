@@ -16,7 +16,8 @@
  *   Appendix on combining the global score with other methods: the redundancy score (normalised
  *       keys, thresholded cosine similarity, column sums, softmax, max-normalisation) and
  *       F' = lambda F - (1 - lambda) R' (gkvo_redundancy, gkvo_combine; its threshold, recent-token
- *       count and epsilon are not in the paper and are parameters).
+ *       count and epsilon are not in the paper and are parameters); the StreamingLLM baseline of Section 6.1 as a
+ *       score-free selection (gkvo_streaming_select).
  * Inputs are the exact bits the GPU consumes: bf16 as uint16 (widened exactly to double) and
  * fp32 score state (widened exactly to double). All arithmetic is double. No blocking, fusion or
  * reordering beyond what the text states.
@@ -414,6 +415,34 @@ int gkvo_evict_step_redundancy(const uint16_t* Q_win, const float* S_in, const u
     if (Fsel_out) memcpy(Fsel_out, Fsel, sizeof(double) * (size_t)h_kv * n_c);
     if (kept_out) memcpy(kept_out, kept, sizeof(int32_t) * (size_t)h_kv * b);
     free(F); free(cbar); free(R); free(Rn); free(Fsel); free(kept);
+    return b;
+}
+
+/* StreamingLLM policy (the sink-plus-recent baseline the paper compares with: related work on decoding-time eviction,
+ * baselines of the experimental setup, Section 6.1), as a degenerate selection on the same framework: no score; the
+ * first n_sink rows of the cache (the attention sinks) and the most recent b - n_sink rows are kept, in ascending
+ * position. kept [h_kv][b] (every head the same list). Requires l > b and 0 <= n_sink <= b. */
+void gkvo_streaming_select(int h_kv, int l, int b, int n_sink, int32_t* kept) {
+    for (int j = 0; j < h_kv; ++j) {
+        int r = 0;
+        for (int t = 0; t < l; ++t)
+            if (t < n_sink || t >= l - (b - n_sink)) kept[(size_t)j * b + r++] = t;
+    }
+}
+
+/* One compression step under that policy: the kept rows are gathered like in gkvo_evict_step; no score exists, so the
+ * recorded score state of the kept rows is 0. Returns the new length (b), or l when l <= b (nothing evicted). */
+int gkvo_evict_step_streaming(const uint16_t* K, const uint16_t* V, const int32_t* pos, int h_kv, int d, int C, int l,
+                              int b, int w, int n_sink, int32_t* kept_out, uint16_t* K_out, uint16_t* V_out,
+                              int32_t* pos_out, double* F_state) {
+    if (l <= b) return l;
+    const int n_c = l - w;
+    int32_t* kept = (int32_t*)malloc(sizeof(int32_t) * (size_t)h_kv * b);
+    double* F = (double*)calloc((size_t)h_kv * n_c, sizeof(double));
+    gkvo_streaming_select(h_kv, l, b, n_sink, kept);
+    if (K_out && V_out && F_state) gkvo_compact(K, V, pos, F, kept, h_kv, C, d, n_c, b, w, K_out, V_out, pos_out, F_state);
+    if (kept_out) memcpy(kept_out, kept, sizeof(int32_t) * (size_t)h_kv * b);
+    free(kept); free(F);
     return b;
 }
 
