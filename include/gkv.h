@@ -67,6 +67,7 @@ typedef enum {
 
 /* Form of the global score (Section 5). LOCAL disables the history: F = normalised S. */
 typedef enum { GKV_MODE_MAX = 0, GKV_MODE_MEAN = 1, GKV_MODE_SUM = 2, GKV_MODE_LOCAL = 3 } gkv_mode;
+typedef enum { GKV_POLICY_SCORE = 0, GKV_POLICY_STREAMING = 1 } gkv_policy;
 
 typedef struct {
     int32_t n_layers, batch, n_q_heads, n_kv_heads, head_dim; /* head_dim must be 128           */
@@ -100,6 +101,13 @@ typedef struct {
      * otherwise) and q_window 16-byte aligned. Sizes part of the workspace (4 bytes per prompt token and KV head, twice or three times
      * that above 8192). */
     int32_t max_prompt;
+    /* Selection policy. GKV_POLICY_SCORE (0): the paper's method, top-(b-w) by the global score. GKV_POLICY_STREAMING:
+     * the sink-plus-recent policy of StreamingLLM, one of the baselines of the paper's experimental setup, as a
+     * score-free selection on the same compaction path: every compression keeps the first n_sink rows of the cache
+     * (the attention sinks; 0 <= n_sink <= b - w) and the most recent b - n_sink rows. No window scores or q_window
+     * are needed (they are ignored), the recorded scores are 0, the redundancy term and pooling must be off. */
+    int32_t policy;
+    int32_t n_sink;
 } gkv_config;
 
 typedef struct { uint64_t k, v, f, sacc, pos, len, workspace, staging; } gkv_sizes; /* bytes      */

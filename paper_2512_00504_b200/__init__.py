@@ -25,6 +25,7 @@ GKV_OK, GKV_ERR_INVALID_ARG, GKV_ERR_STATE, GKV_ERR_CAPACITY, GKV_ERR_CUDA, GKV_
     GKV_ERR_SCRATCH_LIMIT = range(8)
 GKV_MODE_MAX, GKV_MODE_MEAN, GKV_MODE_SUM, GKV_MODE_LOCAL = range(4)
 GKV_STAGE_SCORE, GKV_STAGE_MERGE, GKV_STAGE_SELECT, GKV_STAGE_COMPACT, GKV_STAGE_REDUNDANCY = range(5)
+GKV_POLICY_SCORE, GKV_POLICY_STREAMING = range(2)
 
 
 class GKVError(RuntimeError):
@@ -40,7 +41,8 @@ class gkv_config(ctypes.Structure):
                 ("track_positions", ctypes.c_int32), ("use_redundancy", ctypes.c_int32),
                 ("redundancy_lambda", ctypes.c_float), ("redundancy_threshold", ctypes.c_float),
                 ("redundancy_recent", ctypes.c_int32), ("redundancy_eps", ctypes.c_float),
-                ("pool_kernel", ctypes.c_int32), ("max_prompt", ctypes.c_int32)]
+                ("pool_kernel", ctypes.c_int32), ("max_prompt", ctypes.c_int32), ("policy", ctypes.c_int32),
+                ("n_sink", ctypes.c_int32)]
 
 
 class gkv_sizes(ctypes.Structure):
@@ -143,13 +145,14 @@ def _stream():
 
 def make_config(*, n_layers, batch, h_q, h_kv, d=128, b, buffer, w, s, alpha=0.8, mode=GKV_MODE_MAX,
                 fuse_window_scores=True, track_positions=False, redundancy_lambda=None, redundancy_threshold=0.5,
-                redundancy_recent=None, redundancy_eps=1e-6, pool_kernel=0, max_prompt=0, **_ignored) -> gkv_config:
+                redundancy_recent=None, redundancy_eps=1e-6, pool_kernel=0, max_prompt=0, policy=GKV_POLICY_SCORE, n_sink=0,
+                **_ignored) -> gkv_config:
     """redundancy_lambda=None leaves the redundancy term off; redundancy_recent defaults to the window."""
     use = redundancy_lambda is not None
     return gkv_config(n_layers, batch, h_q, h_kv, d, b, buffer, w, s, alpha, mode,
                       int(fuse_window_scores), int(track_positions), int(use), float(redundancy_lambda if use else 1.0),
                       float(redundancy_threshold), int(w if redundancy_recent is None else redundancy_recent),
-                      float(redundancy_eps), int(pool_kernel), int(max_prompt))
+                      float(redundancy_eps), int(pool_kernel), int(max_prompt), int(policy), int(n_sink))
 
 
 # ------------------------------------------------------------------ C-ABI calls, same names

@@ -44,6 +44,10 @@ gkv_status check_config(const gkv_config* c) {
         if (!(c->redundancy_threshold > 0.f) || !(c->redundancy_eps >= 0.f) || c->redundancy_recent < 0)
             return GKV_ERR_INVALID_ARG;
     }
+    if (c->policy != GKV_POLICY_SCORE && c->policy != GKV_POLICY_STREAMING) return GKV_ERR_INVALID_ARG;
+    if (c->policy == GKV_POLICY_STREAMING &&
+        (c->n_sink < 0 || c->n_sink > c->budget - c->window || c->use_redundancy || c->pool_kernel > 1))
+        return GKV_ERR_INVALID_ARG;
     if (c->head_dim != kHeadDim) return GKV_ERR_UNSUPPORTED;
     if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return GKV_ERR_UNSUPPORTED;
     if (c->budget + c->buffer > kMaxCapacity) return GKV_ERR_UNSUPPORTED;
@@ -160,6 +164,7 @@ EvictLaunch make_evict(gkv_ctx* ctx, int l0, int nl, int32_t* kept_out) {
     p.fsel_ws = ws_ptr<float>(ctx, ctx->ws.fsel);
     p.lambda = c.redundancy_lambda;
     p.pool_kernel = c.pool_kernel;
+    p.policy = c.policy; p.n_sink = c.n_sink;
     return p;
 }
 
@@ -224,7 +229,7 @@ gkv_status evict_precheck(gkv_ctx* ctx, int32_t layer, bool need_window_sums, in
     const int len = ctx->len[*l0];
     *noop = len <= ctx->cfg.budget;
     if (*noop) return GKV_OK;
-    if (need_window_sums) {
+    if (need_window_sums && ctx->cfg.policy != GKV_POLICY_STREAMING) {
         const bool fused_ready = ctx->cfg.fuse_window_scores && ctx->since_evict[*l0] == ctx->cfg.interval;
         if (!fused_ready && !ctx->sacc_valid[*l0]) return GKV_ERR_STATE;
     }
@@ -441,7 +446,7 @@ gkv_status gkv_evict(gkv_ctx* ctx, int32_t layer, const void* q_window, int32_t*
         after_evict(ctx, l0, nl, true);
         return GKV_OK;
     }
-    if (q_window) {
+    if (q_window && ctx->cfg.policy != GKV_POLICY_STREAMING) {
         st = launch_score_for(ctx, l0, nl, q_window, s);
         if (st != GKV_OK) return st;
     }
@@ -498,7 +503,7 @@ gkv_status gkv_evict_stage(gkv_ctx* ctx, int32_t layer, int32_t stage, const voi
     if (stage == GKV_STAGE_MERGE) {
         if (next != 0 && next != GKV_STAGE_MERGE) return GKV_ERR_STATE;
         const bool fused_ready = ctx->cfg.fuse_window_scores && ctx->since_evict[l0] == ctx->cfg.interval;
-        if (!fused_ready && !ctx->sacc_valid[l0]) return GKV_ERR_STATE;
+        if (!fused_ready && !ctx->sacc_valid[l0] && ctx->cfg.policy != GKV_POLICY_STREAMING) return GKV_ERR_STATE;
         if (ctx->cfg.use_redundancy && !ctx->cbar_valid[l0]) return GKV_ERR_STATE;   // REDUNDANCY stage first
         e = launch_evict_merge(p, s);
         if (e == cudaSuccess) next = GKV_STAGE_SELECT;
@@ -603,7 +608,8 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
         const int rows = n > c.budget ? c.budget : n;
         if (rows > longest) longest = rows;
     }
-    if (any_long && !q_window) return GKV_ERR_INVALID_ARG;
+    const bool scored = c.policy != GKV_POLICY_STREAMING;
+    if (any_long && scored && !q_window) return GKV_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int32_t* d_len = ws_ptr<int32_t>(ctx, ctx->ws.prompt_len);
     // a copy from pageable host memory has staged its source when the call returns
@@ -612,7 +618,7 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
         return GKV_ERR_CUDA;
     }
     float* sums = ws_ptr<float>(ctx, ctx->ws.prompt_sums);
-    if (any_long) {
+    if (any_long && scored) {
         CUtensorMap tm_kp;
         const uint64_t rows = (uint64_t)c.batch * c.n_kv_heads * c.max_prompt;
         if (encode_map(&tm_kp, const_cast<void*>(k_prompt), rows) != GKV_OK) return GKV_ERR_CUDA;
@@ -666,6 +672,7 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
     p.status = ws_ptr<int32_t>(ctx, ctx->ws.status);
     p.layer = layer; p.L_total = c.n_layers; p.batch = c.batch; p.h_kv = c.n_kv_heads; p.C = ctx->C;
     p.P_max = c.max_prompt; p.b = c.budget; p.w = c.window; p.pool_kernel = c.pool_kernel;
+    p.policy = c.policy; p.n_sink = c.n_sink;
     if (launch_prompt_compress(p, s) != cudaSuccess) {
         (void)cudaGetLastError();
         return GKV_ERR_CUDA;

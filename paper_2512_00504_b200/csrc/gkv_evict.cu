@@ -238,6 +238,20 @@ __device__ int select_phase(const float* s_f, KT* s_kept, int* s_evict, int n_c,
     return sh->first_evicted;
 }
 
+// Sink-plus-recent policy (StreamingLLM, a baseline of the paper's experimental setup) as a selection without a
+// score: rows 0 .. n_sink - 1 stay, rows n_sink .. n_sink + (n - b) - 1 leave, the rest moves up. Writes the same
+// outputs as select_phase, clears s_f (no score is recorded) and returns the first row that moves.
+template <typename KT>
+__device__ int streaming_phase(float* s_f, KT* s_kept, int* s_evict, int n, int n_c, int b, int n_sink, int tid) {
+    const int shift = n - b;
+    for (int t = tid; t < n_c; t += kEvictThreads) s_f[t] = 0.f;
+    for (int r = tid; r < b; r += kEvictThreads) s_kept[r] = (KT)(r < n_sink ? r : r + shift);
+    if (s_evict)
+        for (int e = tid; e < shift; e += kEvictThreads) s_evict[e] = n_sink + e;
+    sel_sync();
+    return n_sink;
+}
+
 // Move the rows kept[r] -> r for r in [r_first, b) of one unit's K and V, restricted to the
 // 16-byte chunks [chunk0, chunk0 + cpr) of every row (cpr divides 16).
 __device__ void compact_phase(__nv_bfloat16* kbase, __nv_bfloat16* vbase, const int* kept, int b, int r_first,
@@ -526,15 +540,19 @@ __global__ void __launch_bounds__(kFusedThreads, 5) gkv_evict_fused_kernel(const
             const int buf = handed & 1;
             uint16_t* kept = s_kept + buf * p.b;
             const int n_c = n - p.w;
-            merge_phase(s_f, s_fp, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
-            selection_scores(p, u.unit, s_f, s_sel, n, n_c, sh, tid);
+            const bool scored = p.policy != GKV_POLICY_STREAMING;
+            if (scored) {
+                merge_phase(s_f, s_fp, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
+                selection_scores(p, u.unit, s_f, s_sel, n, n_c, sh, tid);
+            }
             // the copy warp has issued every load that reads this buffer's previous list (two units ago)
             if (handed >= 2) {   // one thread waits, the barrier hands its verdict (and the ordering) to the others
                 if (tid == 0) pipe->go = evict_wait(smem_u32(&pipe->kept_empty[buf]), ((handed >> 1) - 1) & 1, &pipe->abort_flag);
                 sel_sync();
                 if (!*(volatile int*)&pipe->go) { evict_abort(pipe, p.status, 41); break; }
             }
-            const int r_first = select_phase(s_sel, kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
+            const int r_first = scored ? select_phase(s_sel, kept, s_evict, n_c, p.b - p.w, p.w, sh, tid)
+                                       : streaming_phase(s_f, kept, s_evict, n, n_c, p.b, p.n_sink, tid);
             if (tid == 0) {
                 pipe->unit[buf] = u.unit;
                 pipe->r_first[buf] = r_first;
@@ -685,7 +703,9 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_prompt_compress_kernel(cons
     const bool compress = n > p.b;
     const int rows = compress ? p.b : n;                   // rows of the cache after this call
     const int n_keep = p.b - p.w;
-    if (compress) {
+    if (compress && p.policy == GKV_POLICY_STREAMING) {
+        streaming_phase(s_f, s_kept, (int*)nullptr, n, n - p.w, p.b, p.n_sink, tid);
+    } else if (compress) {
         const int n_c = n - p.w;
         merge_phase(p.sums + (size_t)unit_local * p.P_max, nullptr, s_f, n_c, 0, 0.f, GKV_MODE_LOCAL, sh, tid);
         if (p.pool_kernel > 1) pool_phase(s_f, s_sel, n_c, p.pool_kernel, tid);
@@ -734,7 +754,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_merge_kernel(const Ev
     const UnitIndex u = unit_of(p, blockIdx.x);
     const int n = p.len[u.lseq_global];
     const int n_h = p.len[(size_t)p.L_total * p.batch + u.lseq_global];
-    if (n <= p.b) return;
+    if (n <= p.b || p.policy == GKV_POLICY_STREAMING) return;   // (the policy without a score has nothing to merge)
     const int n_c = n - p.w;
     merge_phase(p.sacc + (size_t)u.unit * p.C, p.f + (size_t)u.unit * p.C, s_f, n_c, n_h, p.alpha, p.mode, sh, tid);
     float* out = p.f_ws + (size_t)u.unit_local * p.C;
@@ -759,14 +779,18 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const E
         return;
     }
     const int n_c = n - p.w;
-    const float* in = p.f_ws + (size_t)u.unit_local * p.C;
-    for (int t = tid; t < n_c; t += kEvictThreads) s_f[t] = in[t];
-    if (has_selection_terms(p)) {
-        const float* in2 = p.fsel_ws + (size_t)u.unit_local * p.C;
-        for (int t = tid; t < n_c; t += kEvictThreads) s_sel[t] = in2[t];
+    if (p.policy == GKV_POLICY_STREAMING) {
+        streaming_phase(s_f, s_kept, s_evict, n, n_c, p.b, p.n_sink, tid);
+    } else {
+        const float* in = p.f_ws + (size_t)u.unit_local * p.C;
+        for (int t = tid; t < n_c; t += kEvictThreads) s_f[t] = in[t];
+        if (has_selection_terms(p)) {
+            const float* in2 = p.fsel_ws + (size_t)u.unit_local * p.C;
+            for (int t = tid; t < n_c; t += kEvictThreads) s_sel[t] = in2[t];
+        }
+        __syncthreads();
+        select_phase(s_sel, s_kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
     }
-    __syncthreads();
-    select_phase(s_sel, s_kept, s_evict, n_c, p.b - p.w, p.w, sh, tid);
     write_score_state(p, u, s_f, s_kept, s_pos, s_evict, n, tid);
     int32_t* kw = p.kept_ws + (size_t)u.unit_local * p.b;
     for (int r = tid; r < p.b; r += kEvictThreads) kw[r] = s_kept[r];

@@ -80,6 +80,7 @@ struct EvictLaunch {
     float* fsel_ws;      // staged path scratch
     float lambda;
     int pool_kernel;     // > 1: sequence-wise max-pooling of the score before the selection
+    int policy, n_sink;  // GKV_POLICY_STREAMING: the kept list is the first n_sink rows and the most recent b - n_sink
 };
 
 struct PromptLaunch {
@@ -101,6 +102,7 @@ struct PromptLaunch {
     int32_t* kept_out;           // may be NULL: [batch*h_kv][b], -1 padded
     int32_t* status;
     int layer, L_total, batch, h_kv, C, P_max, b, w, pool_kernel;
+    int policy, n_sink;
 };
 
 struct RedundancyLaunch {

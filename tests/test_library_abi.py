@@ -58,6 +58,9 @@ def base(**over):
     (dict(max_prompt=(1 << 20) + 1), gkv.GKV_ERR_UNSUPPORTED),   # longest prompt the first compression takes
     (dict(max_prompt=9000, w=24), gkv.GKV_ERR_UNSUPPORTED),     # above 8192 tokens the window is a multiple of 16
     (dict(max_prompt=-1), gkv.GKV_ERR_INVALID_ARG),
+    (dict(policy=1, n_sink=497), gkv.GKV_ERR_INVALID_ARG),       # more sinks than b - w
+    (dict(policy=1, n_sink=4, pool_kernel=5), gkv.GKV_ERR_INVALID_ARG),   # the score-free policy has nothing to pool
+    (dict(policy=2), gkv.GKV_ERR_INVALID_ARG),
 ])
 def test_config_validation(over, status):
     with pytest.raises(gkv.GKVError) as e:
