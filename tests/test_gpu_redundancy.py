@@ -71,6 +71,8 @@ def run(shape, seed, lam, tau, recent, l=None, n_h=None, staged=False, dup=True)
             assert (np.abs(cbar[n, j, : case.l][dirty] - ref["cbar"][j][dirty]) <=
                     ref["band"][j][dirty] * (tau + BAND) + 1e-3).all(), what + ": borderline cbar"
             flips += int(dirty.sum())
+            assert int(dirty.sum()) <= max(8, case.l // 50), what + ": too many columns with a borderline similarity"
+
             assert (cbar[n, j, case.l - recent: case.l] == 0).all() and (cbar[n, j, case.l:] == 0).all()
             # selection: same set as the oracle's ranking of Fsel up to rows within tolerance of the threshold score;
             # the exp of the redundancy term carries cbar's relative error times |cbar - max|
@@ -80,8 +82,15 @@ def run(shape, seed, lam, tau, recent, l=None, n_h=None, staged=False, dup=True)
             order = np.lexsort((np.arange(case.l - w), -fsel))
             thr = fsel[order[n_keep - 1]]
             band = SCORE_RTOL * (abs(thr) + (1.0 - lam)) + SCORE_ATOL
+            # A column with n borderline similarities may be off by n threshold-sized terms in cbar, i.e. by the factor
+            # exp(n (tau + BAND)) in R' = exp(cbar - max cbar) (and every column by the same factor if the maximum's own
+            # column has such entries): that, and nothing more, is added to the band of such a row.
+            cb = ref["cbar"][j]
+            rn = np.exp(cb - cb.max())
+            n_max = int(ref["band"][j][int(np.argmax(cb))])
             for t in set(order[:n_keep].tolist()) ^ set(k[:n_keep].tolist()):
-                assert abs(fsel[t] - thr) <= band or not clean[t], f"{what}: row {t} differs outside the band"
+                slack = (1.0 - lam) * rn[t] * (np.exp((int(ref["band"][j][t]) + n_max) * (tau + BAND)) - 1.0)
+                assert abs(fsel[t] - thr) <= band + slack, f"{what}: row {t} differs outside the band"
             # compaction by the GPU's own kept list; the recorded score is F, not the combined score
             assert (K_after[n, j, :b] == snap["K"][n, j, k]).all() and (V_after[n, j, :b] == snap["V"][n, j, k]).all()
             assert (pos_after[n, j, :b] == snap["pos"][n, j, k]).all()
@@ -95,6 +104,7 @@ def run(shape, seed, lam, tau, recent, l=None, n_h=None, staged=False, dup=True)
     (dict(batch=1, h_q=28, h_kv=4, b=300, buffer=100, w=32, s=100), 0.9, 0.35, 8, 391),    # ragged: 2 blocks, last one 135 keys
     (dict(batch=3, h_q=4, h_kv=4, b=100, buffer=28, w=8, s=28), 0.3, 0.6, 0, None),        # one 128-key block, no protected tokens
     (dict(batch=1, h_q=16, h_kv=2, b=1100, buffer=130, w=64, s=130), 0.7, 0.45, 64, None),  # 1230 keys: 5 blocks, 10 tiles
+    (dict(batch=1, h_q=8, h_kv=2, b=2048, buffer=128, w=64, s=128), 0.7, 0.5, 64, None),    # 2176 keys, the sweep's largest cache
 ])
 def test_redundancy_eviction_matches_oracle(shape, lam, tau, recent, l):
     run(shape, synth.BASE_SEED + 40 + shape["w"], lam, tau, recent, l=l)
