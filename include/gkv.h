@@ -62,7 +62,9 @@ typedef enum {
     GKV_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed                            */
     GKV_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (latched status word)       */
     GKV_ERR_UNSUPPORTED = 6, /* valid but not built (head_dim != 128, g > 8, ...)              */
-    GKV_ERR_SCRATCH_LIMIT = 7 /* problem larger than the library's built-in scratch array      */
+    GKV_ERR_SCRATCH_LIMIT = 7, /* problem larger than the library's built-in scratch array     */
+    GKV_ERR_INTERNAL = 8     /* checked build only (-DGKV_CHECK_BOUNDS): a kernel computed a row index out of
+                                range; the access was skipped and the status word latched          */
 } gkv_status;
 
 /* Form of the global score (Section 5). LOCAL disables the history: F = normalised S. */
@@ -263,7 +265,8 @@ gkv_status gkv_get_state(const gkv_ctx* ctx, int32_t layer, int32_t* len, int32_
 int64_t gkv_launch_count(const gkv_ctx* ctx);
 
 /* Synchronises `stream` and returns GKV_ERR_TIMEOUT if any kernel latched an expired bounded
- * wait since the last poll, GKV_ERR_CUDA on a CUDA error, else OK. On TIMEOUT the latch and the
+ * wait since the last poll (GKV_ERR_INTERNAL if a library built with -DGKV_CHECK_BOUNDS caught a row index out of
+ * range), GKV_ERR_CUDA on a CUDA error, else OK. On TIMEOUT the latch and the
  * kernels' completion and work counters in the workspace are cleared, so the context can be used
  * again; what the kernel that gave up had written (outputs, cache rows, lengths) is undefined:
  * declare the state anew with gkv_set_state before going on. */

@@ -17,12 +17,15 @@ from pathlib import Path
 
 _PKG = Path(__file__).resolve().parent
 _ROOT = _PKG.parent
-LIB_PATH = _PKG / "libgkv.so"
+# GKV_LIB_VARIANT=check selects the library built with -DGKV_CHECK_BOUNDS (every row index that selection and compaction
+# compute is tested before use; see build_library(check_bounds=True)); the default is the production build.
+_CHECKED = os.environ.get("GKV_LIB_VARIANT", "") == "check"
+LIB_PATH = _PKG / ("libgkv_check.so" if _CHECKED else "libgkv.so")
 _SOURCES = ["gkv_api.cu", "gkv_decode.cu", "gkv_evict.cu", "gkv_score.cu", "gkv_score_tc.cu", "gkv_redundancy.cu",
             "gkv_static_scratch.cu"]
 
 GKV_OK, GKV_ERR_INVALID_ARG, GKV_ERR_STATE, GKV_ERR_CAPACITY, GKV_ERR_CUDA, GKV_ERR_TIMEOUT, GKV_ERR_UNSUPPORTED, \
-    GKV_ERR_SCRATCH_LIMIT = range(8)
+    GKV_ERR_SCRATCH_LIMIT, GKV_ERR_INTERNAL = range(9)
 GKV_MODE_MAX, GKV_MODE_MEAN, GKV_MODE_SUM, GKV_MODE_LOCAL = range(4)
 GKV_STAGE_SCORE, GKV_STAGE_MERGE, GKV_STAGE_SELECT, GKV_STAGE_COMPACT, GKV_STAGE_REDUNDANCY = range(5)
 GKV_POLICY_SCORE, GKV_POLICY_STREAMING = range(2)
@@ -61,20 +64,25 @@ class gkv_memory_model_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint64) for n in ("full_kv", "compressed_kv", "score_cache")]
 
 
-def build_library(force: bool = False, verbose: bool = False) -> Path:
-    """Compile csrc/*.cu into libgkv.so for sm_100a with nvcc (cross-compiles without a GPU)."""
+def build_library(force: bool = False, verbose: bool = False, check_bounds: bool | None = None) -> Path:
+    """Compile csrc/*.cu into libgkv.so for sm_100a with nvcc (cross-compiles without a GPU). check_bounds builds
+    libgkv_check.so with -DGKV_CHECK_BOUNDS instead (default: whichever variant this process loads)."""
+    check = _CHECKED if check_bounds is None else check_bounds
+    out = _PKG / ("libgkv_check.so" if check else "libgkv.so")
     srcs = [_PKG / "csrc" / s for s in _SOURCES if (_PKG / "csrc" / s).exists()]
     deps = srcs + list((_PKG / "csrc").glob("*.h")) + list((_PKG / "csrc").glob("*.cuh")) + [_ROOT / "include" / "gkv.h"]
-    if not force and LIB_PATH.exists() and all(LIB_PATH.stat().st_mtime >= d.stat().st_mtime for d in deps):
-        return LIB_PATH
-    tmp = LIB_PATH.with_suffix(f".so.tmp{os.getpid()}")
+    if not force and out.exists() and all(out.stat().st_mtime >= d.stat().st_mtime for d in deps):
+        return out
+    tmp = out.with_suffix(f".so.tmp{os.getpid()}")
     cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
            "-Xcompiler", "-fPIC", "-I", str(_ROOT / "include"), "-o", str(tmp)] + [str(s) for s in srcs]
+    if check:
+        cmd.insert(1, "-DGKV_CHECK_BOUNDS")
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, out)
+    return out
 
 
 _lib = None

@@ -727,7 +727,7 @@ gkv_status gkv_poll_device_status(gkv_ctx* ctx, void* stream) {
         // A kernel that gave up may have left its completion and work counters part-way (they are returned to zero
         // by the last CTA of a launch that runs to its end): clear them together with the latch.
         if (cudaMemsetAsync(d, 0, ctx->ws.kept - ctx->ws.status, s) != cudaSuccess) return GKV_ERR_CUDA;
-        return GKV_ERR_TIMEOUT;
+        return h[0] == kStatusBounds ? GKV_ERR_INTERNAL : GKV_ERR_TIMEOUT;
     }
     return GKV_OK;
 }
@@ -775,6 +775,7 @@ const char* gkv_strerror(gkv_status status) {
         case GKV_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case GKV_ERR_UNSUPPORTED: return "configuration not supported by this library";
         case GKV_ERR_SCRATCH_LIMIT: return "problem exceeds the library's built-in scratch array";
+        case GKV_ERR_INTERNAL: return "checked build: a kernel computed a row index out of range (access skipped)";
         default: return "unknown status";
     }
 }

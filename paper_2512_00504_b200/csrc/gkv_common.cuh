@@ -19,6 +19,23 @@ constexpr int kMaxGroup = 8;          // query heads per KV head handled by one 
 
 // Device status word (workspace): 0 = fine; set to a code when a bounded wait gives up.
 constexpr int kStatusTimeout = 1;
+constexpr int kStatusBounds = 2;      // checked build only: an index was out of range (the access was skipped)
+
+// Checked build (-DGKV_CHECK_BOUNDS): every row index that selection and compaction compute is tested before it is
+// used; a bad one is not used (the access is skipped) and latches kStatusBounds with the place in status[1] -- no
+// trap, no assert. In the normal build the macro is the constant true and costs nothing.
+#ifdef GKV_CHECK_BOUNDS
+__device__ __forceinline__ bool gkv_bounds_fail(int32_t* status, int where) {
+    if (status && atomicCAS(status, 0, kStatusBounds) == 0) {
+        status[1] = where;
+        status[2] = blockIdx.x;
+    }
+    return false;
+}
+#define GKV_BOUNDS_OK(cond, status, where) ((cond) ? true : gkv::gkv_bounds_fail((status), (where)))
+#else
+#define GKV_BOUNDS_OK(cond, status, where) (true)
+#endif
 
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -34,6 +34,7 @@ struct EvictShared {
     int warp_sums[16];
     float warp_max[8];
     int digit, k_rem, first_evicted, is_last;
+    int32_t* status;   // the launch's status word (checked build: where a bad index is reported)
 };
 
 // inclusive prefix sum over the 256 threads of the CTA
@@ -218,18 +219,22 @@ __device__ int select_phase(const float* s_f, KT* s_kept, int* s_evict, int n_c,
         const int kept_before = gt_before + min(eq_before, k);   // kept rows below t
         bool dropped = false;
         if (x > T) {
-            s_kept[kept_before] = (KT)t;
+            if (GKV_BOUNDS_OK(kept_before >= 0 && kept_before < n_keep, sh->status, 61)) s_kept[kept_before] = (KT)t;
             ++gt_before;
         } else if (x == T) {
-            if (eq_before < k) s_kept[kept_before] = (KT)t;
-            else dropped = true;
+            if (eq_before < k) {
+                if (GKV_BOUNDS_OK(kept_before >= 0 && kept_before < n_keep, sh->status, 62)) s_kept[kept_before] = (KT)t;
+            } else {
+                dropped = true;
+            }
             ++eq_before;
         } else {
             dropped = true;
         }
         if (dropped) {
             first_drop = min(first_drop, t);
-            if (s_evict) s_evict[t - kept_before] = t;
+            if (s_evict && GKV_BOUNDS_OK(t - kept_before >= 0 && t - kept_before < n_c - n_keep, sh->status, 63))
+                s_evict[t - kept_before] = t;
         }
     }
     if (first_drop < n_c) atomicMin(&sh->first_evicted, first_drop);
@@ -254,8 +259,10 @@ __device__ int streaming_phase(float* s_f, KT* s_kept, int* s_evict, int n, int 
 
 // Move the rows kept[r] -> r for r in [r_first, b) of one unit's K and V, restricted to the
 // 16-byte chunks [chunk0, chunk0 + cpr) of every row (cpr divides 16).
+// (`n_rows` = rows of the unit that hold tokens and `status` are used by the checked build only.)
 __device__ void compact_phase(__nv_bfloat16* kbase, __nv_bfloat16* vbase, const int* kept, int b, int r_first,
-                              int chunk0, int cpr, int tid) {
+                              int chunk0, int cpr, int tid, int n_rows, int32_t* status) {
+    (void)n_rows; (void)status;
     const int rows_per_pass = kEvictThreads / cpr;
     const int my_r = tid / cpr;
     const int my_c = chunk0 + (tid - my_r * cpr);
@@ -268,6 +275,7 @@ __device__ void compact_phase(__nv_bfloat16* kbase, __nv_bfloat16* vbase, const 
         for (int u = 0; u < kCompactUnroll; ++u) {
             const int r = r0 + u * rows_per_pass + my_r;
             src[u] = (r < b) ? kept[r] : -1;
+            if (src[u] >= 0 && !GKV_BOUNDS_OK(src[u] >= r && src[u] < n_rows, status, 64)) src[u] = -1;
             if (src[u] >= 0) {
                 kx[u] = k4[(size_t)src[u] * 16 + my_c];
                 vx[u] = v4[(size_t)src[u] * 16 + my_c];
@@ -298,7 +306,9 @@ constexpr int kCopyRingBytes = kCopyStages * kCopyStageBytes;
 
 // Source and destination may be the same buffers (compaction in place) or different ones (gather of a prompt).
 __device__ void compact_phase_async(const __nv_bfloat16* ksrc, const __nv_bfloat16* vsrc, __nv_bfloat16* kbase,
-                                    __nv_bfloat16* vbase, const int* kept, int b, int r_first, uint8_t* ring, int tid) {
+                                    __nv_bfloat16* vbase, const int* kept, int b, int r_first, uint8_t* ring, int tid,
+                                    int n_rows, int32_t* status) {
+    (void)n_rows; (void)status;
     constexpr int D = kCopyStages - 2;                        // groups of loads in flight
     const int n_groups = (b - r_first + kCopyRows - 1) / kCopyRows;
     const uint32_t ring_addr = smem_u32(ring);
@@ -317,7 +327,7 @@ __device__ void compact_phase_async(const __nv_bfloat16* ksrc, const __nv_bfloat
                 const int e = u * kEvictThreads + tid;
                 const int is_v = e >> 9, row = (e >> 4) & (kCopyRows - 1), chunk = e & 15;
                 const int r = r0 + row;
-                if (r < b) {
+                if (r < b && GKV_BOUNDS_OK(kept[r] >= r && kept[r] < n_rows, status, 65)) {
                     const uint4* src = (is_v ? v4 : k4) + (size_t)kept[r] * 16 + chunk;
                     cp_async_16(stage + (uint32_t)(is_v * kCopyRows * kRowBytes + row * kRowBytes + chunk * 16), src);
                 }
@@ -361,7 +371,8 @@ __device__ void write_score_state(const EvictLaunch& p, const UnitIndex& u, cons
                                   int* s_pos, const int* s_evict, int n, int tid) {
     const int n_keep = p.b - p.w;
     float* f = p.f + (size_t)u.unit * p.C;
-    for (int r = tid; r < p.C; r += kEvictThreads) f[r] = (r < n_keep) ? s_f[s_kept[r]] : 0.f;
+    for (int r = tid; r < p.C; r += kEvictThreads)
+        f[r] = (r < n_keep && GKV_BOUNDS_OK((int)s_kept[r] >= r && (int)s_kept[r] < n - p.w, p.status, 66)) ? s_f[s_kept[r]] : 0.f;
     if (p.pos) {
         int32_t* pos = p.pos + (size_t)u.unit * p.C;
         for (int t = tid; t < n; t += kEvictThreads) s_pos[t] = pos[t];
@@ -426,8 +437,9 @@ struct __align__(16) FusedPipe {
     uint64_t ring_full[kFusedMaxStages];   // the rows of a stage have landed
     long unit[2];             // the unit whose kept list is in buffer i, or -1: no more
     int r_first[2];           // first destination row that moves
+    int n_rows[2];            // rows of that unit that hold tokens (checked build)
     uint32_t dst_row[kFusedMaxStages];     // per stage: first destination row (in rows of the whole K / V tensor), rows held
-    int n_rows[kFusedMaxStages];
+    int st_rows[kFusedMaxStages];
     int cur_item, abort_flag, is_last, go;
 };
 
@@ -489,6 +501,7 @@ __global__ void __launch_bounds__(kFusedThreads, 5) gkv_evict_fused_kernel(const
         for (int s = 0; s < stages; ++s) mbar_init(smem_u32(&pipe->ring_full[s]), 1);
         pipe->abort_flag = 0;
         pipe->is_last = 0;
+        sh->status = p.status;
         fence_mbar_init();
     }
     __syncthreads();
@@ -556,6 +569,7 @@ __global__ void __launch_bounds__(kFusedThreads, 5) gkv_evict_fused_kernel(const
             if (tid == 0) {
                 pipe->unit[buf] = u.unit;
                 pipe->r_first[buf] = r_first;
+                pipe->n_rows[buf] = n;
                 mbar_arrive(smem_u32(&pipe->kept_full[buf]));
             }
             ++handed;
@@ -587,7 +601,7 @@ __global__ void __launch_bounds__(kFusedThreads, 5) gkv_evict_fused_kernel(const
             }
             if (lane == 0) {
                 const uint32_t src = ring_addr + (uint32_t)st * kCopyStageBytes;
-                const uint32_t bytes = (uint32_t)pipe->n_rows[st] * kRowBytes;
+                const uint32_t bytes = (uint32_t)pipe->st_rows[st] * kRowBytes;
                 const size_t dst = (size_t)pipe->dst_row[st] * kHeadDim;
                 bulk_store(p.k_cache + dst, src, bytes);
                 bulk_store(p.v_cache + dst, src + kCopyRows * kRowBytes, bytes);
@@ -620,7 +634,7 @@ __global__ void __launch_bounds__(kFusedThreads, 5) gkv_evict_fused_kernel(const
                 const uint32_t bar = smem_u32(&pipe->ring_full[st]);
                 if (lane == 0) {
                     pipe->dst_row[st] = (uint32_t)(unit * p.C + r0);
-                    pipe->n_rows[st] = rows;
+                    pipe->st_rows[st] = rows;
                     mbar_arrive_expect_tx(bar, (uint32_t)rows * 2 * kRowBytes);
                 }
                 __syncwarp();
@@ -632,10 +646,18 @@ __global__ void __launch_bounds__(kFusedThreads, 5) gkv_evict_fused_kernel(const
                 const uint32_t starts = __ballot_sync(0xffffffffu, start);
                 if (start) {
                     const uint32_t rest = (lane == 31) ? 0u : (starts >> (lane + 1));
-                    const int run = rest ? __ffs(rest) : rows - lane;
+                    int run = rest ? __ffs(rest) : rows - lane;
+                    // (checked build: a run must start at or above its destination and end inside the unit's tokens;
+                    // a bad one is not copied, its bytes are taken off the stage's expected count)
+                    if (!GKV_BOUNDS_OK(src >= r0 + lane && src + run <= pipe->n_rows[buf] && r0 + lane + run <= p.b, p.status, 67)) {
+                        asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"((uint32_t)run * 2 * kRowBytes) : "memory");
+                        run = 0;
+                    }
+                    if (run > 0) {
                     const uint32_t dst = ring_addr + (uint32_t)st * kCopyStageBytes + (uint32_t)lane * kRowBytes;
                     bulk_load(dst, k4 + (size_t)src * 16, (uint32_t)run * kRowBytes, bar);
                     bulk_load(dst + kCopyRows * kRowBytes, v4 + (size_t)src * 16, (uint32_t)run * kRowBytes, bar);
+                    }
                 }
                 if (G >= (uint32_t)D + stored) store_next();   // keeps D groups of loads in flight
             }
@@ -687,6 +709,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_prompt_compress_kernel(cons
     extern __shared__ __align__(128) uint8_t evict_smem[];
     EvictShared* sh = reinterpret_cast<EvictShared*>(evict_smem);
     const int tid = threadIdx.x;
+    if (tid == 0) sh->status = p.status;     // (read after the barriers of the phases below)
     const int unit_local = blockIdx.x;
     // The unit's scores [P_max] (and the pooled ones) live in shared memory, or, for prompts too long for it, in the
     // workspace: the phases below only need a pointer, and a CTA-wide barrier orders global accesses as well.
@@ -732,7 +755,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_prompt_compress_kernel(cons
     }
     compact_phase_async(p.k_src + (size_t)unit_local * p.P_max * kHeadDim, p.v_src + (size_t)unit_local * p.P_max * kHeadDim,
                         p.k_cache + (size_t)unit * p.C * kHeadDim, p.v_cache + (size_t)unit * p.C * kHeadDim, s_kept, rows, 0,
-                        evict_smem + ring_offset, tid);
+                        evict_smem + ring_offset, tid, n, p.status);
     __syncthreads();
     if (tid == 0) {   // the last CTA of the sequence publishes its length and the rows that carry history
         const int prev = atomicAdd(&p.seq_done[lseq_global], 1);
@@ -779,6 +802,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_select_kernel(const E
         return;
     }
     const int n_c = n - p.w;
+    if (tid == 0) sh->status = p.status;
     if (p.policy == GKV_POLICY_STREAMING) {
         streaming_phase(s_f, s_kept, s_evict, n, n_c, p.b, p.n_sink, tid);
     } else {
@@ -819,7 +843,7 @@ __global__ void __launch_bounds__(kEvictThreads) gkv_evict_compact_kernel(const 
     __syncthreads();
     const int cpr = 16 / slices;
     compact_phase(p.k_cache + (size_t)u.unit * p.C * kHeadDim, p.v_cache + (size_t)u.unit * p.C * kHeadDim, s_kept,
-                  p.b, sh->first_evicted, slice * cpr, cpr, tid);
+                  p.b, sh->first_evicted, slice * cpr, cpr, tid, n, p.status);
     publish_state(p, u, p.h_kv * slices, sh, tid);
 }
 
