@@ -99,7 +99,7 @@ typedef struct {
      * gives no kernel size and reports that pooling does not help at decode time. */
     int32_t pool_kernel;
     /* Longest prompt gkv_compress_prompt will be given (rows per head of its K / V buffers); 0 = that call is
-     * not used. At most 1048576; above 8192 the window must be a multiple of 16 and use_redundancy off (UNSUPPORTED
+     * not used. At most 1048576; above 8192 the window must be a multiple of 16 (UNSUPPORTED
      * otherwise) and q_window 16-byte aligned. Sizes part of the workspace (4 bytes per prompt token and KV head, twice or three times
      * that above 8192). */
     int32_t max_prompt;

@@ -36,8 +36,6 @@ gkv_status check_config(const gkv_config* c) {
         score_tc_rows_per_cta(c->n_q_heads / c->n_kv_heads, c->window) == 0)
         return GKV_ERR_UNSUPPORTED;
     if ((uint64_t)c->batch * c->n_kv_heads * (uint64_t)c->max_prompt >= (1ull << 31)) return GKV_ERR_UNSUPPORTED;
-    // the redundancy kernel keeps a unit's inverse key norms in shared memory
-    if (c->use_redundancy && c->max_prompt > kMaxPromptShared) return GKV_ERR_UNSUPPORTED;
     if (c->pool_kernel < 0 || (c->pool_kernel > 1 && (c->pool_kernel & 1) == 0)) return GKV_ERR_INVALID_ARG;
     if (c->use_redundancy) {
         if (!(c->redundancy_lambda >= 0.f && c->redundancy_lambda <= 1.f)) return GKV_ERR_INVALID_ARG;
@@ -69,7 +67,7 @@ void layout_workspace(const gkv_config* c, int sm_count, WorkspaceLayout* w) {
     const uint64_t red = c->use_redundancy ? 1 : 0;   // the redundancy term's scratch exists only when it is on
     w->prompt_sums = off; off = align_up(off + upl * (uint64_t)c->max_prompt * sizeof(float));
     w->prompt_len = off;  off = align_up(off + (c->max_prompt > 0 ? B : 0) * sizeof(int32_t));
-    const uint64_t long_arrays = c->max_prompt > kMaxPromptShared ? (c->pool_kernel > 1 ? 2 : 1) : 0;
+    const uint64_t long_arrays = c->max_prompt > kMaxPromptShared ? ((c->pool_kernel > 1 || c->use_redundancy) ? 2 : 1) : 0;
     w->prompt_f = off;    off = align_up(off + long_arrays * upl * (uint64_t)c->max_prompt * sizeof(float));
     const uint64_t sel = (c->use_redundancy || c->pool_kernel > 1) ? 1 : 0;
     w->fsel = off;     off = align_up(off + sel * upl * C * sizeof(float));

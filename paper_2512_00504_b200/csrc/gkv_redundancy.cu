@@ -90,6 +90,9 @@ __device__ __forceinline__ float ge_mask(float a, float b) {
 }
 __device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kRdEpiThreads) : "memory"); }
 
+// LONG: the unit's inverse norms do not fit shared memory (prompts of more than 8192 tokens being compressed): they are
+// read from the workspace (L2) with plain loads, 32 per chunk of columns, the same addresses for every lane.
+template <bool LONG>
 __global__ void __launch_bounds__(kRdThreads, 1)
 gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUtensorMap tm_k, int blocks_per_unit,
                          int stages) {
@@ -98,7 +101,7 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
     constexpr int a_half = kRdABytes / 2;
     uint8_t* a_smem = smem;
     uint8_t* k_smem = smem + kRdABytes;
-    const int c_pad = (p.C + 127) & ~127;
+    const int c_pad = LONG ? 0 : (p.C + 127) & ~127;
     float* s_inv = reinterpret_cast<float*>(k_smem + stages * kRdStageBytes);   // [c_pad] inverse norms of the unit, 0 beyond n
     float* s_part = s_inv + c_pad;                                              // [groups][128] partial row sums
     RedundancyTail* tail = reinterpret_cast<RedundancyTail*>(s_part + kRdGroups * 128);
@@ -135,10 +138,8 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
         tmem_relinquish_alloc_permit();
         tmem_fence_before_sync();
     }
-    {
-        const float* ginv = p.inv_norm + (size_t)unit * p.C;
-        for (int t = tid; t < c_pad; t += kRdThreads) s_inv[t] = (t < n) ? ginv[t] : 0.f;
-    }
+    const float* ginv = p.inv_norm + (size_t)unit * p.C;
+    for (int t = tid; t < c_pad; t += kRdThreads) s_inv[t] = (t < n) ? ginv[t] : 0.f;
     __syncthreads();
     tmem_fence_after_sync();
     const uint32_t tmem_base = *(volatile uint32_t*)&tail->tmem_base;
@@ -222,7 +223,7 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
         const int nch = (MT == 2) ? 4 : 2;
         const uint32_t t_p = t_lane + (uint32_t)((MT == 2) ? sub * 128 : col0);
         const int row = a0 + rl;                       // the key this thread sums for
-        const float inv_r = (row < n) ? s_inv[row] : 0.f;
+        const float inv_r = (row < n) ? (LONG ? ginv[row] : s_inv[row]) : 0.f;
         const float thr = (row < n) ? __fdiv_rn(p.tau, inv_r) : INFINITY;   // Cm >= tau  <=>  G * inv_col >= tau / inv_row
         float sum = 0.f;
         bool ok = true;
@@ -234,7 +235,17 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
             for (int ch = 0; ch < nch; ++ch) {
                 float gacc[32];
                 tmem_ld<32>(t_p + (uint32_t)(buf * kRdAccCols + ch * 32), gacc);
-                const float4* iv = reinterpret_cast<const float4*>(s_inv + i * kRdTileKeys + col0 + ch * 32);
+                const int colbase = i * kRdTileKeys + col0 + ch * 32;
+                float4 ivl[8];
+                const float4* iv = LONG ? ivl : reinterpret_cast<const float4*>(s_inv + colbase);
+                if (LONG) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int c = colbase + 4 * j;
+                        ivl[j] = make_float4(c < n ? __ldg(ginv + c) : 0.f, c + 1 < n ? __ldg(ginv + c + 1) : 0.f,
+                                             c + 2 < n ? __ldg(ginv + c + 2) : 0.f, c + 3 < n ? __ldg(ginv + c + 3) : 0.f);
+                    }
+                }
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
                 if (i + 1 < T) {
                     // per element one compare (1.0 / 0.0) and half a packed multiply and half a packed multiply-add: a
@@ -292,13 +303,16 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
     }
 }
 
+constexpr int kRdMaxShared = 8192;   // keys whose inverse norms are kept in shared memory
 static size_t redundancy_smem_bytes(int C, int stages) {
     return 1024 + (size_t)kRdABytes + (size_t)stages * kRdStageBytes +
-           sizeof(float) * (((C + 127) & ~127) + kRdGroups * 128) + sizeof(RedundancyTail);
+           sizeof(float) * ((C > kRdMaxShared ? 0 : ((C + 127) & ~127)) + kRdGroups * 128) + sizeof(RedundancyTail);
 }
 
 cudaError_t redundancy_kernel_setup() {
-    return cudaFuncSetAttribute(gkv_redundancy_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(gkv_redundancy_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(gkv_redundancy_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }
 
 cudaError_t launch_keynorm(const RedundancyLaunch& p, cudaStream_t s) {
@@ -312,8 +326,12 @@ cudaError_t launch_redundancy(const RedundancyLaunch& p, const CUtensorMap& tm_k
     const int blocks_per_unit = (p.C + kRdBlockRows - 1) / kRdBlockRows;
     int stages = 2;
     while (stages < kRdMaxStages && redundancy_smem_bytes(p.C, stages + 1) <= 227 * 1024) ++stages;
-    gkv_redundancy_tc_kernel<<<units * blocks_per_unit, kRdThreads, redundancy_smem_bytes(p.C, stages), s>>>(
-        p, tm_k, blocks_per_unit, stages);
+    if (p.C > kRdMaxShared)
+        gkv_redundancy_tc_kernel<true><<<units * blocks_per_unit, kRdThreads, redundancy_smem_bytes(p.C, stages), s>>>(
+            p, tm_k, blocks_per_unit, stages);
+    else
+        gkv_redundancy_tc_kernel<false><<<units * blocks_per_unit, kRdThreads, redundancy_smem_bytes(p.C, stages), s>>>(
+            p, tm_k, blocks_per_unit, stages);
     return cudaGetLastError();
 }
 

@@ -183,14 +183,17 @@ def test_very_long_prompt_with_all_scores_equal_keeps_the_lowest_positions():
         assert (synth.bits(cache.k[0, 1, j])[:b] == Kp[j, kept[1, j]]).all()
 
 
-@pytest.mark.parametrize("pool", [0, 5])
-def test_prompt_compression_with_redundancy_term(pool):
+@pytest.mark.parametrize("pool,P_max,lens,h_q,h_kv", [
+    (0, 1500, [1500, 200, 777], 8, 2),
+    (5, 1500, [1500, 200, 777], 8, 2),
+    (0, 8400, [8400, 300], 4, 1),        # more than 8192 tokens: scores and inverse key norms live in the workspace
+])
+def test_prompt_compression_with_redundancy_term(pool, P_max, lens, h_q, h_kv):
     """With use_redundancy the first compression selects on lambda * F - (1 - lambda) * R' like every later one; the
     redundancy level comes from the prompt's own keys (cosine similarities above the threshold, the most recent
     columns zeroed). The heavy hitters of the synthetic prompt share a direction, so they are mutually redundant."""
-    w, h_q, h_kv, b, buffer, s, P_max = 16, 8, 2, 256, 32, 32, 1500
+    w, b, buffer, s = 16, 256, 32, 32
     lam, tau, recent = 0.7, 0.3, 16
-    lens = [1500, 200, 777]
     B = len(lens)
     cfg = gkv.make_config(n_layers=1, batch=B, h_q=h_q, h_kv=h_kv, b=b, buffer=buffer, w=w, s=s, fuse_window_scores=True,
                           track_positions=True, max_prompt=P_max, pool_kernel=pool, redundancy_lambda=lam,
