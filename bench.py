@@ -369,11 +369,14 @@ def run_ours(args) -> dict:
 
 # ------------------------------------------------------------------------------------------
 def time_evict_cell(sh: dict, dev: str, *, reps: int, stages: bool, red_kwargs: dict, peaks: dict, n_planted: int,
-                    seed: int, oracle_seconds: float = 0.0) -> dict:
+                    seed: int, oracle_seconds: float = 0.0, group: int = 1) -> dict:
     """One eviction step of one layer at shape `sh` with the cache at l = b + buffer rows and n_h = b - w rows of
     history: the step as it runs (`fused`: one launch reading the window sums; `recompute`: scoring launch from the
     window queries + the fused launch), the scoring launch alone and, with `stages`, every stage as its own launch.
-    L2 is flushed (a 512 MB memset) before every timed launch; medians of `reps` after 3 warm-up rounds."""
+    L2 is flushed (a 512 MB memset) before every timed region; medians of `reps` after 3 warm-up rounds.
+    group > 1: the cache holds `group` layers of the shape and a timed region is the `group` per-layer launches of the
+    step back to back, the way a model compresses layer by layer (every layer's rows are cold: the flush precedes the
+    group); the reported time is the region's divided by `group`. The stages are always timed on one layer."""
     import torch
     import paper_2512_00504_b200 as gkv
     from paper_2512_00504_b200 import synth
@@ -382,27 +385,30 @@ def time_evict_cell(sh: dict, dev: str, *, reps: int, stages: bool, red_kwargs: 
     g, C = sh["h_q"] // H, b + sh["buffer"]
     l, n_h, units = C, b - w, batch * H
     red = bool(red_kwargs)
-    cfg = gkv.make_config(**sh, alpha=0.8, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True, **red_kwargs)
+    cfg = gkv.make_config(**dict(sh, n_layers=group), alpha=0.8, mode=gkv.GKV_MODE_MAX, fuse_window_scores=True, **red_kwargs)
     cache = gkv.GKVCache(cfg, dev)
     case = synth.eviction_case(seed, batch=batch, h_q=sh["h_q"], h_kv=H, b=b, buffer=sh["buffer"], w=w,
                                n_planted=n_planted, device=dev)
-    cache.k[0].copy_(case.k); cache.v[0].copy_(case.v); cache.f[0].copy_(case.f_prev)
+    for layer in range(group):
+        cache.k[layer].copy_(case.k); cache.v[layer].copy_(case.v); cache.f[layer].copy_(case.f_prev)
     q_win = case.q_win.unsqueeze(0).contiguous()
     sample = None
     if oracle_seconds > 0:          # the oracle's inputs: the first sequences of the cell, the GPU's own bits
         n_s = min(batch, 16)
         sample = (synth.bits(case.q_win[:n_s]), synth.bits(case.k[:n_s]), synth.bits(case.v[:n_s]), case.f_prev[:n_s].cpu().numpy())
     del case
-    cache.set_state(0, l, n_h, sh["s"], False)
-    cache.evict_stage(0, gkv.GKV_STAGE_SCORE, q_win)          # the window sums of this state (w * S)
+    cache.set_state(-1, l, n_h, sh["s"], False)
+    for layer in range(group):
+        cache.evict_stage(layer, gkv.GKV_STAGE_SCORE, q_win)  # the window sums of this state (w * S)
     sums0, f0 = cache.sacc.clone(), cache.f.clone()
-    kept = torch.empty((1, batch, H, b), dtype=torch.int32, device=dev)
+    kept = torch.empty((group, batch, H, b), dtype=torch.int32, device=dev)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     ev = lambda: torch.cuda.Event(enable_timing=True)
+    layers = range(group)
 
     def restore():
         cache.sacc.copy_(sums0); cache.f.copy_(f0)
-        cache.set_state(0, l, n_h, sh["s"], True)
+        cache.set_state(-1, l, n_h, sh["s"], True)
         flush.zero_()
 
     def timed(fn):
@@ -410,14 +416,21 @@ def time_evict_cell(sh: dict, dev: str, *, reps: int, stages: bool, red_kwargs: 
         e0.record(); fn(); e1.record()
         return e0, e1
 
+    def each_layer(fn):
+        def run():
+            for layer in layers:
+                fn(layer)
+        return run
+
     names = ["score", "fused", "recompute"] + (["redundancy", "merge", "select", "compact"] if stages else [])
+    per_group = {"score", "fused", "recompute"}
     t = {k: [] for k in names}
     moved = 0.0
     l0 = gkv.gkv_launch_count(cache.ctx)
     for it in range(reps + 3):
         pairs = {}
         restore()
-        pairs["score"] = timed(lambda: cache.evict_stage(0, gkv.GKV_STAGE_SCORE, q_win))
+        pairs["score"] = timed(each_layer(lambda layer: cache.evict_stage(layer, gkv.GKV_STAGE_SCORE, q_win)))
         if stages:
             if red:
                 flush.zero_()
@@ -425,18 +438,18 @@ def time_evict_cell(sh: dict, dev: str, *, reps: int, stages: bool, red_kwargs: 
             flush.zero_()
             pairs["merge"] = timed(lambda: cache.evict_stage(0, gkv.GKV_STAGE_MERGE))
             flush.zero_()
-            pairs["select"] = timed(lambda: cache.evict_stage(0, gkv.GKV_STAGE_SELECT, None, kept))
+            pairs["select"] = timed(lambda: cache.evict_stage(0, gkv.GKV_STAGE_SELECT, None, kept[0]))
             flush.zero_()
             pairs["compact"] = timed(lambda: cache.evict_stage(0, gkv.GKV_STAGE_COMPACT))
         restore()
-        pairs["fused"] = timed(lambda: cache.evict(0, None, kept))
-        moved = float((kept != torch.arange(b, device=dev, dtype=torch.int32)).sum().item())
+        pairs["fused"] = timed(each_layer(lambda layer: cache.evict(layer, None, kept[layer])))
+        moved = float((kept[0] != torch.arange(b, device=dev, dtype=torch.int32)).sum().item())
         restore()
-        pairs["recompute"] = timed(lambda: cache.evict(0, q_win, kept))
+        pairs["recompute"] = timed(each_layer(lambda layer: cache.evict(layer, q_win, kept[layer])))
         torch.cuda.synchronize()
         if it >= 3:
             for k, (e0, e1) in pairs.items():
-                t[k].append(e0.elapsed_time(e1))
+                t[k].append(e0.elapsed_time(e1) / (group if k in per_group else 1))
     cache.poll()
     launches = gkv.gkv_launch_count(cache.ctx) - l0
     med = {k: sorted(v)[len(v) // 2] for k, v in t.items() if v}
@@ -458,7 +471,7 @@ def time_evict_cell(sh: dict, dev: str, *, reps: int, stages: bool, red_kwargs: 
             "recompute_frac": rec_bound / (med["recompute"] * 1e-3),
             "scored_kv_tokens_per_s": units * l / (med["recompute"] * 1e-3),
             "scored_kv_tokens_per_s_window_sums": units * l / (med["fused"] * 1e-3),
-            "gpu_launches": int(launches)}
+            "launches_per_timed_region": group, "gpu_launches": int(launches)}
     if red and "redundancy" in med:
         cell["redundancy_TFLOPs"] = 2.0 * units * l * l * 128 / (med["redundancy"] * 1e-3) / 1e12
     if sample is not None:
@@ -513,10 +526,11 @@ def other_configs(args, dev: str, peaks: dict) -> dict:
                 sh = dict(n_layers=1, batch=batch, h_q=c3["h_q"], h_kv=c3["h_kv"], d=128, b=b, buffer=c3["buffer"], w=w, s=c3["s"])
                 cells.append(time_evict_cell(sh, dev, reps=5, stages=False, red_kwargs={}, peaks=peaks,
                                              n_planted=math.ceil(0.01 * (b + c3["buffer"])), seed=synth.BASE_SEED + 3,
-                                             oracle_seconds=0.0 if args.no_cpu else 1.0))
+                                             oracle_seconds=0.0 if args.no_cpu else 1.0, group=args.sweep_group))
     out["cfg3"] = {"workload": "config 3: eviction-step sweep, 1 layer, 32 q / 8 kv heads, l = b + 128; cells with batch >= 64 "
                                "(python bench.py --workload cfg3 runs all 32 cells with the stages timed one by one)",
-                   "l2": "flushed (512 MB memset) before every timed launch",
+                   "l2": "flushed (512 MB memset) before every timed region; a region is the per-layer launches of "
+                         f"{args.sweep_group} layers of the cell's shape back to back (every layer's rows cold), time per launch = region / {args.sweep_group}",
                    "min_fused_frac": min(c["fused_frac"] for c in cells), "min_score_frac": min(c["score_frac"] for c in cells),
                    "cells": cells, "clocks": sampler.stop()}
     # configuration 4: the 32B-shaped stress case, 77 GB of K+V resident; 3 periods in steady state after 3 warm-up periods
@@ -562,7 +576,8 @@ def run_sweep(args) -> dict:
             for w in pick(args.sweep_w, c3["w_sweep"]):
                 sh = dict(n_layers=1, batch=batch, h_q=c3["h_q"], h_kv=c3["h_kv"], d=128, b=b, buffer=c3["buffer"], w=w, s=c3["s"])
                 cells.append(time_evict_cell(sh, dev, reps=reps, stages=True, red_kwargs=redundancy_kwargs(args), peaks=peaks,
-                                             n_planted=math.ceil(0.01 * (b + c3["buffer"])), seed=synth.BASE_SEED + 3))
+                                             n_planted=math.ceil(0.01 * (b + c3["buffer"])), seed=synth.BASE_SEED + 3,
+                                             group=args.sweep_group))
     clocks = sampler.stop()
     top = cells[-1]
     return {"metric": "scored KV tokens/s of one eviction step (score from the window queries + merge + top-(b-w) + compaction)",
@@ -571,7 +586,8 @@ def run_sweep(args) -> dict:
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"config 3 sweep, largest cell: 1 layer, batch {top['batch']}, 32 q / 8 kv heads, d 128, b={top['b']}, "
                                    f"buffer=128, w={top['w']}, l={top['b'] + 128}; step = one eviction step",
-                       "l2": "flushed (512 MB memset) before every timed launch"},
+                       "l2": "flushed (512 MB memset) before every timed region; fused / recompute / score regions are the per-layer "
+                             f"launches of {args.sweep_group} layers back to back, stages are single launches"},
             "clocks": clocks, "e2e": None, "gpu_launches": int(sum(c["gpu_launches"] for c in cells)),
             "roofline": {"kernel": "gkv_evict_fused_kernel", "bound": "hbm", "achieved": top["fused_GBps"], "peak": peak_gbs,
                          "unit": "GB/s", "frac": top["fused_frac"], "peak_source": peaks["source"], "traffic": None,
@@ -811,6 +827,8 @@ def main():
     ap.add_argument("--sweep-b", default="", help="cfg3: comma-separated budgets instead of the full sweep")
     ap.add_argument("--sweep-batch", default="", help="cfg3: comma-separated batch sizes instead of the full sweep")
     ap.add_argument("--sweep-w", default="", help="cfg3: comma-separated windows instead of the full sweep")
+    ap.add_argument("--sweep-group", type=int, default=4,
+                    help="cfg3: per-layer launches timed back to back between one pair of events (layers of the cell's shape)")
     ap.add_argument("--redundancy", type=float, default=None, metavar="LAMBDA",
                     help="select on LAMBDA * F - (1 - LAMBDA) * R' (redundancy term on; adds two launches per eviction)")
     ap.add_argument("--redundancy-threshold", type=float, default=0.5)
