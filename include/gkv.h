@@ -291,6 +291,14 @@ typedef struct { int32_t grid, splits, stages, ctas_per_sm, smem_bytes, tmem_col
 gkv_status gkv_decode_launch_plan(const gkv_config* cfg, int32_t n_layers_in_launch, int32_t window_step,
                                   int32_t sm_count, gkv_decode_plan_t* out);
 
+/* How gkv_evict would launch its fused kernel (no paper counterpart; host arithmetic, for capacity planning and tests
+ * without a GPU; the eviction log, which adds C - b words of shared memory, is taken as off): grid = CTAs launched
+ * (persistent: at most the resident ones; with three rounds of units or fewer the rounds are filled equally), stages =
+ * depth of the copy ring (32 rows of K and V per stage), ctas_per_sm, smem_bytes = dynamic shared memory per CTA.
+ * Errors: as gkv_query_sizes; INVALID_ARG for a layer count other than 1 or cfg->n_layers. */
+typedef struct { int32_t grid, stages, ctas_per_sm, smem_bytes; } gkv_evict_plan_t;
+gkv_status gkv_evict_launch_plan(const gkv_config* cfg, int32_t n_layers_in_launch, int32_t sm_count, gkv_evict_plan_t* out);
+
 /* Memory model of the paper's appendix "Memory Analysis": bytes of the full KV cache at
  * seq_len tokens, of the compressed cache ((b + s) rows instead of seq_len), and of the score
  * cache F (b - w entries per head), for `elem_bytes`-wide elements, over all layers and the

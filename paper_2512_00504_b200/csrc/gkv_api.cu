@@ -749,6 +749,26 @@ gkv_status gkv_decode_launch_plan(const gkv_config* cfg, int32_t n_layers_in_lau
     return GKV_OK;
 }
 
+gkv_status gkv_evict_launch_plan(const gkv_config* cfg, int32_t n_layers_in_launch, int32_t sm_count, gkv_evict_plan_t* out) {
+    if (!out) return GKV_ERR_INVALID_ARG;
+    const gkv_status st = check_config(cfg);
+    if (st != GKV_OK) return st;
+    if (n_layers_in_launch != 1 && n_layers_in_launch != cfg->n_layers) return GKV_ERR_INVALID_ARG;
+    EvictLaunch p = {};
+    p.n_layers = n_layers_in_launch; p.batch = cfg->batch; p.h_kv = cfg->n_kv_heads;
+    p.C = cfg->budget + cfg->buffer; p.b = cfg->budget; p.w = cfg->window;
+    p.sm_count = sm_count;
+    p.pool_kernel = cfg->pool_kernel;
+    // only whether these are set matters for the shared-memory layout
+    p.pos = cfg->track_positions ? reinterpret_cast<int32_t*>(1) : nullptr;
+    p.cbar = cfg->use_redundancy ? reinterpret_cast<const float*>(1) : nullptr;
+    int stages = 0, grid = 0, ctas = 0;
+    size_t smem = 0;
+    evict_plan(p, &stages, &grid, &smem, &ctas);
+    out->grid = grid; out->stages = stages; out->ctas_per_sm = ctas; out->smem_bytes = (int32_t)smem;
+    return GKV_OK;
+}
+
 gkv_status gkv_memory_model(const gkv_config* cfg, int64_t seq_len, int32_t elem_bytes, gkv_memory_model_t* out) {
     if (!cfg || !out || seq_len <= 0 || elem_bytes <= 0) return GKV_ERR_INVALID_ARG;
     if (cfg->n_layers <= 0 || cfg->batch <= 0 || cfg->n_kv_heads <= 0 || cfg->head_dim <= 0 || cfg->budget <= 0 ||

@@ -858,7 +858,7 @@ static cudaError_t ensure_smem(const void* fn, size_t bytes) {
 // Grid: persistent, at most the resident CTAs; with three rounds of units or fewer the rounds are filled equally
 // (512 units on 296 slots run as 256 CTAs x 2 units: a unit cannot be split, and a CTA holding two units next to
 // CTAs holding one sets the end of the launch).
-void evict_plan(const EvictLaunch& p, int* stages, int* grid, size_t* smem) {
+void evict_plan(const EvictLaunch& p, int* stages, int* grid, size_t* smem, int* ctas_per_sm) {
     const FusedLayout lay = fused_layout(p.C, p.b, p.cbar != nullptr || p.pool_kernel > 1, p.pos != nullptr, p.evict_log != nullptr);
     auto ctas_with = [&](int st) {
         const int by_smem = (int)((227 * 1024) / ((size_t)lay.ring + (size_t)st * kCopyStageBytes + 1024));
@@ -880,12 +880,13 @@ void evict_plan(const EvictLaunch& p, int* stages, int* grid, size_t* smem) {
     *stages = st;
     *grid = (int)g;
     *smem = (size_t)lay.ring + (size_t)st * kCopyStageBytes;
+    if (ctas_per_sm) *ctas_per_sm = max(1, ctas_with(st));
 }
 
 cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s) {
     int stages, grid;
     size_t smem;
-    evict_plan(p, &stages, &grid, &smem);
+    evict_plan(p, &stages, &grid, &smem, nullptr);
     cudaError_t e = ensure_smem((const void*)gkv_evict_fused_kernel, smem);
     if (e != cudaSuccess) return e;
     gkv_evict_fused_kernel<<<grid, kFusedThreads, smem, s>>>(p, stages);

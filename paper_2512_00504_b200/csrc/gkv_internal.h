@@ -148,6 +148,7 @@ void decode_plan(DecodeLaunch* p, int max_pieces);
 void decode_plan_resources(const DecodeLaunch& p, int* ctas_per_sm, size_t* smem_bytes);   // of a planned launch
 cudaError_t launch_decode(const DecodeLaunch& p, const DecodeMaps& maps, cudaStream_t s);
 cudaError_t launch_evict_fused(const EvictLaunch& p, cudaStream_t s);
+void evict_plan(const EvictLaunch& p, int* stages, int* grid, size_t* smem, int* ctas_per_sm);   // shape of that launch
 cudaError_t launch_evict_merge(const EvictLaunch& p, cudaStream_t s);
 cudaError_t launch_evict_select(const EvictLaunch& p, cudaStream_t s);
 cudaError_t launch_evict_compact(const EvictLaunch& p, int sm_count, cudaStream_t s);

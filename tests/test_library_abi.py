@@ -146,6 +146,30 @@ def test_decode_launch_plan_invariants(sm_count):
                         assert -(-units // rounds) <= p.grid <= min(units, resident)   # full grid, or equal rounds
 
 
+@pytest.mark.parametrize("sm_count", [148, 132, 64])
+def test_evict_launch_plan_invariants(sm_count):
+    """Host-side planning of the fused eviction launch: what the kernel relies on (a ring of at least three stages so
+    that a group of loads is in flight while another is stored; shared memory within the 227 KB of a CTA; a persistent
+    grid that is never larger than what is resident at once, nor than the units) and the equal-rounds rule."""
+    for kw in (dict(), dict(b=256, buffer=128), dict(b=2048, buffer=256, w=64, s=256, h_q=64, h_kv=8),
+               dict(b=3968, buffer=128, track_positions=True, pool_kernel=5), dict(b=1024, buffer=128, w=32, h_q=28, h_kv=4)):
+        for batch in (1, 8, 64, 256, 1024):
+            cfg = base(batch=batch, n_layers=1, **kw)
+            units = batch * cfg.n_kv_heads
+            p = gkv.gkv_evict_launch_plan(cfg, 1, sm_count)
+            assert 3 <= p.stages <= 8 and 1 <= p.ctas_per_sm <= 5
+            assert p.smem_bytes <= 227 * 1024 and (p.smem_bytes + 1024) * p.ctas_per_sm <= 227 * 1024 + 1024 * p.ctas_per_sm
+            resident = p.ctas_per_sm * sm_count
+            assert 1 <= p.grid <= min(units, resident)
+            rounds = -(-units // p.grid)
+            if units > resident and -(-units // resident) <= 3:
+                assert p.grid == -(-units // -(-units // resident))        # equally filled rounds
+                assert rounds == -(-units // resident)                     # ... and no more of them
+    # the cases the design notes name: 512 units of the 7B shape run as 256 CTAs x 2 units on 148 SMs
+    p = gkv.gkv_evict_launch_plan(gkv.make_config(n_layers=4, batch=32, h_q=28, h_kv=4, b=1024, buffer=128, w=32, s=128), 4, 148)
+    assert (p.grid, p.stages, p.ctas_per_sm) == (256, 6, 2)
+
+
 def test_memory_model_reproduces_the_papers_appendix():
     """Appendix "Memory Analysis": 28 layers, d = 128, 2 KV heads, bf16, 16k tokens -> ~0.44 GB per
     sequence and 56 GB at batch 128; with s = 128 and b = 512 / 1024 / 2048 the compressed cache
