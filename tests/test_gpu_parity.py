@@ -730,3 +730,76 @@ def test_config2_full_length_run_sampled():
     cache.poll()
     assert real == 120
     assert int(cache.len[0].min()) == int(cache.len[0].max()) == b and int(cache.len[1].min()) == b - w
+
+
+# ------------------------------------------------------------------------- seeded sweep of odd shapes
+def _random_eviction_setup(i):
+    """The i-th shape of a fixed pseudo-random sweep: head geometry, window, budget, buffer, cache length, history
+    length, merge form, decay and launch form drawn independently, so that combinations nobody wrote down by hand
+    (an odd window with g = 7, a one-row buffer, history shorter than the budget, ...) meet every kernel."""
+    rng = np.random.default_rng(synth.BASE_SEED + 1000 + i)
+    h_kv = int(rng.choice([1, 2, 4, 8]))
+    g = int(rng.choice([1, 2, 3, 4, 7, 8]))
+    w = int(rng.choice([1, 3, 8, 16, 24, 32, 48, 64]))
+    b = w + int(rng.integers(1, 700))
+    buffer = max(w, int(rng.integers(1, 260)))       # the library wants w <= interval <= buffer
+    s = int(rng.integers(w, buffer + 1))
+    C = b + buffer
+    l = int(rng.integers(b + 1, C + 1))
+    n_h = int(rng.integers(0, min(b - w, l - w) + 1)) if rng.random() < 0.5 else min(b - w, l - w)
+    shape = dict(batch=int(rng.integers(1, 4)), h_q=g * h_kv, h_kv=h_kv, b=b, buffer=buffer, w=w, s=s)
+    kw = dict(l=l, n_h=n_h, mode=int(rng.integers(0, 4)), alpha=float(rng.choice([0.0, 0.3, 0.8, 1.0])),
+              recompute=bool(rng.random() < 0.6), staged=bool(rng.random() < 0.3), track=bool(rng.random() < 0.7))
+    return shape, kw
+
+
+@pytest.mark.parametrize("i", range(24))
+def test_evict_random_shapes(i):
+    shape, kw = _random_eviction_setup(i)
+    run_single_eviction(shape, synth.BASE_SEED + 2000 + i, **kw)
+
+
+@pytest.mark.parametrize("i", range(12))
+def test_decode_random_shapes(i):
+    """Seeded sweep of decode shapes: a few plain steps, then the w window steps before a compression, at a random
+    cache length; every step's output and the accumulated window sums against the oracle."""
+    rng = np.random.default_rng(synth.BASE_SEED + 3000 + i)
+    h_kv = int(rng.choice([1, 2, 4, 8]))
+    g = int(rng.choice([1, 2, 3, 4, 7, 8]))
+    w = int(rng.choice([1, 3, 8, 16, 32]))
+    b = w + int(rng.integers(1, 900))
+    buffer = max(w, int(rng.integers(1, 200)))
+    s = int(rng.integers(w, buffer + 1))
+    extra = int(rng.integers(0, min(3, s - w) + 1))                 # plain steps before the window
+    B = int(rng.choice([1, 2, 5, 40]))
+    cfg = gkv.make_config(n_layers=1, batch=B, h_q=g * h_kv, h_kv=h_kv, b=b, buffer=buffer, w=w, s=s, fuse_window_scores=True)
+    cache = gkv.GKVCache(cfg, DEV)
+    C, Hq, H = cache.C, g * h_kv, h_kv
+    l_end = int(rng.integers(w + extra + 1, C + 1))
+    start = l_end - w - extra
+    gen = torch.Generator(device=DEV).manual_seed(synth.BASE_SEED + 3100 + i)
+    rnd = lambda *sh: torch.randn(*sh, generator=gen, device=DEV).to(torch.bfloat16)
+    cache.k[0, :, :, :start] = rnd(B, H, start, 128)
+    cache.v[0, :, :, :start] = rnd(B, H, start, 128)
+    cache.set_state(0, start, 0, s - w - extra)
+    K, V = synth.bits(cache.k[0]), synth.bits(cache.v[0])
+    sel = np.arange(B) if B <= 5 else np.array([0, B // 2, B - 1])
+    out = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device=DEV)
+    qs = []
+    for t in range(start, l_end):
+        q, kn, vn = rnd(B, Hq, 128), rnd(B, H, 128), rnd(B, H, 128)
+        cache.decode_attn(0, q, kn, vn, out)
+        K[:, :, t], V[:, :, t] = synth.bits(kn), synth.bits(vn)
+        ref = oracle.decode_batch(synth.bits(q)[sel], K[sel], V[sel], t + 1)
+        assert np.abs(out.float().cpu().numpy()[sel] - ref).max() < DECODE_ATOL, (i, t)
+        if t >= l_end - w:
+            qs.append(q)
+    cache.poll()
+    assert cache.state(0) == (l_end, 0, s)
+    assert (synth.bits(cache.k[0]) == K).all() and (synth.bits(cache.v[0]) == V).all()
+    q_win = torch.stack(qs, dim=2).contiguous()
+    sacc = cache.sacc[0].cpu().numpy()
+    for n in sel:
+        S = oracle.window_mean(oracle.group_max(oracle.window_attention(synth.bits(q_win[n]), K[n], l_end), H))
+        np.testing.assert_allclose(sacc[n][:, :l_end] / w, S, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+        assert not sacc[n][:, l_end:].any()
