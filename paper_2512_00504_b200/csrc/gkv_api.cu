@@ -193,7 +193,7 @@ gkv_status dispatch_score(gkv_ctx* ctx, const ScoreLaunch& sp, const CUtensorMap
     if (wk > 0 && (reinterpret_cast<uintptr_t>(sp.q_win) & 15) == 0) {
         CUtensorMap tm_q;
         const uint64_t q_rows = (uint64_t)sp.n_layers * c.batch * c.n_q_heads * c.window;
-        if (encode_map(&tm_q, const_cast<__nv_bfloat16*>(sp.q_win), q_rows, (uint32_t)wk) != GKV_OK) return GKV_ERR_CUDA;
+        if (encode_map(&tm_q, const_cast<__nv_bfloat16*>(sp.q_win), q_rows, (uint32_t)score_tc_q_box_rows(wk)) != GKV_OK) return GKV_ERR_CUDA;
         if (launch_score_tc(sp, tm_k, tm_q, wk, s) != cudaSuccess) return GKV_ERR_CUDA;
     } else if (sp.C > kMaxPromptShared) {
         return GKV_ERR_INVALID_ARG;   // a long prompt with misaligned window queries: the other kernel holds all sums on chip

@@ -155,6 +155,7 @@ cudaError_t launch_evict_compact(const EvictLaunch& p, int sm_count, cudaStream_
 cudaError_t launch_score(const ScoreLaunch& p, const CUtensorMap& tm_k, cudaStream_t s);
 cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s);
 int score_tc_rows_per_cta(int g, int w);
+int score_tc_q_box_rows(int wk);
 cudaError_t score_tc_kernel_setup();
 cudaError_t launch_prompt_compress(const PromptLaunch& p, cudaStream_t s);
 cudaError_t launch_keynorm(const RedundancyLaunch& p, cudaStream_t s);

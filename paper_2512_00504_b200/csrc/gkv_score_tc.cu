@@ -7,7 +7,7 @@
 // that every reduction is a loop inside one thread:
 //   pass 1   D[q row][key] = Q K^T   (M = 128 query rows, N = 128 keys per tile): the thread that
 //            owns a TMEM lane owns a query row and keeps its online (max, sum) over the keys;
-//   pass 2   D[key][q row] = K Q^T   (M = 128 keys, N = g * wk query rows): the thread that owns a
+//   pass 2   D[key][q row] = K Q^T   (M = 128 keys, N = up to 128 query rows): the thread that owns a
 //            lane owns a key, and the max over heads and the sum over window rows run over columns.
 // A work item is one unit (layer, sequence, KV head) and wk <= 64 window rows of all g heads
 // (g * wk <= 256 rows; wider windows take several items that add into the same sums).
@@ -16,12 +16,17 @@
 // on across item boundaries, so the next item's window queries and first key tiles are in flight,
 // and its first products issued, while the softmax warps finish the item before. Warp 0 streams K
 // tiles by TMA (a ring that continues across items; pass 2 walks the tiles backwards, so what it
-// reads is still in L2) and the window queries (two buffers), warp 1 issues tcgen05.mma into two
-// 256-column TMEM accumulators, warps 2-17 (four groups of four, one TMEM lane quarter per warp)
-// read the accumulators back with tcgen05.ld and do the softmax arithmetic.
+// reads is still in L2) and the window queries (two buffers). The products are cut into turns of
+// 128 x 128 (eight tcgen05.mma) that go round four 128-column TMEM accumulators; the turns of even
+// number are issued by one thread (warp 1) and read back by one set of eight softmax warps, those
+// of odd number by a second thread (warp 18) and the other set (warps 2-17: two sets of two groups
+// of four warps, one TMEM lane quarter per warp). One thread needs longer to issue a turn (two
+// waits, eight instructions, two commits) than the tensor core to execute it, and a set's
+// tcgen05.ld latency is exposed once per turn: with two independent issuer / reader pairs, each
+// with two accumulators of its own, one pair's waits and loads run under the other's work.
 //
-// Pass 1 is bound by the exponentials (one per logit; the special-function unit does 16 a clock and
-// SM, the tensor core 8192 flop): half of them are evaluated on the FMA pipe instead, as
+// Pass 1 is bound by the instructions of the exponentials (one per logit; the special-function unit
+// does 16 a clock and SM): half of them are evaluated on the FMA pipe instead, as
 // 2^x = 2^round(x) * P(x - round(x)) with a cubic P (relative error < 8e-5; pass 1 only feeds the
 // row sums, and the scores are compared at 1e-3). With at most 64 query rows the rows are loaded
 // twice (lanes 64-127 of the accumulator repeat lanes 0-63) and the two copies split the keys of a
@@ -35,12 +40,13 @@ namespace gkv {
 
 constexpr int kTcGroups = 4;                                 // softmax warp groups (4 warps each)
 constexpr int kTcSoftmaxThreads = kTcGroups * 128;
-constexpr int kTcThreads = 64 + kTcSoftmaxThreads;
+constexpr int kTcIssuerB = 2 + kTcSoftmaxThreads / 32;       // the warp after the softmax warps: second tcgen05.mma issuer
+constexpr int kTcThreads = 64 + kTcSoftmaxThreads + 32;
 constexpr int kTcTileKeys = 128;
 constexpr int kTcMaxStages = 6;                              // K ring depth is chosen per launch from the shared memory left
 constexpr int kTcKStageBytes = kTcTileKeys * kRowBytes;      // 32 KB: d-low half then d-high half
 constexpr int kTcMaxRows = 256;
-constexpr int kTcAccCols = 256;                              // TMEM columns of one accumulator
+constexpr int kTcAccCols = 128;                              // TMEM columns of one accumulator (four of them)
 constexpr uint32_t kTcTmemCols = 512;
 constexpr int kTcChunkKeys = 8192;                           // keys whose window sums are held in shared memory at a time
 
@@ -49,9 +55,9 @@ struct __align__(8) ScoreTcTail {
     uint64_t q_empty[2];
     uint64_t k_full[kTcMaxStages];
     uint64_t k_empty[kTcMaxStages];
-    uint64_t d_full[2];
-    uint64_t d_empty[2];
-    uint64_t drain;
+    uint64_t d_full[4];
+    uint64_t d_empty[4];
+    uint64_t drain[2];
     uint64_t chunk_bar;   // the softmax warps meet here when the window sums move on to the next chunk of keys
     uint32_t tmem_base;
     int abort_flag;
@@ -65,6 +71,12 @@ __device__ __forceinline__ void tc_abort(ScoreTcTail* tail, int32_t* status, int
         status[1] = where;
         status[2] = blockIdx.x;
     }
+}
+// Maximum of three (one instruction; NaN operands are dropped like in fmaxf).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
 }
 __device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kTcSoftmaxThreads) : "memory"); }
 
@@ -101,12 +113,12 @@ __device__ __forceinline__ void row_update(float (&z)[N], int key0, int last_vis
     float c0 = fmaxf(z[0], z[1]), c1 = fmaxf(z[2], z[3]), c2 = fmaxf(z[4], z[5]), c3 = fmaxf(z[6], z[7]);
 #pragma unroll
     for (int j = 8; j < N; j += 8) {
-        c0 = fmaxf(c0, fmaxf(z[j], z[j + 1]));
-        c1 = fmaxf(c1, fmaxf(z[j + 2], z[j + 3]));
-        c2 = fmaxf(c2, fmaxf(z[j + 4], z[j + 5]));
-        c3 = fmaxf(c3, fmaxf(z[j + 6], z[j + 7]));
+        c0 = max3(c0, z[j], z[j + 1]);
+        c1 = max3(c1, z[j + 2], z[j + 3]);
+        c2 = max3(c2, z[j + 4], z[j + 5]);
+        c3 = max3(c3, z[j + 6], z[j + 7]);
     }
-    const float mn = fmaxf(m_raw, fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)));
+    const float mn = fmaxf(max3(m_raw, c0, c1), fmaxf(c2, c3));
     if (mn == -INFINITY) return;
     const float neg = -mn * scale;
     float s0 = 0.f, s1 = 0.f;
@@ -143,17 +155,37 @@ __device__ __forceinline__ ScoreItem score_item(const ScoreLaunch& p, int item, 
     return d;
 }
 
-// WK = window rows handled by one item (16, 32 or 64); the item's local query row of (head h, window
-// row k0 + kk) is h * WK + kk.
-template <int WK>
+// Window rows of one block of the query tile (see the kernel's comment on the row order).
+__host__ __device__ constexpr int score_tc_block_rows(int wk) { return wk == 64 ? 16 : 8; }
+
+// WK = window rows handled by one item (16, 32 or 64).
+//
+// Order of the item's query rows in shared memory (row index of the pass-1 accumulators and of s_c, column index of
+// the pass-2 accumulators): blocks of PW consecutive window rows of one head, the heads of a block of window rows next
+// to each other: row = (wrb * g + h) * PW + jj for window row k0 + wrb * PW + jj of head h. So the columns that a
+// pass-2 thread needs for the max over heads of a few window rows are contiguous and come with few tensor-memory
+// loads, and the rows split into halves by window row, not by head.
+//
+// A turn is one 128 x 128 product (eight instructions) into one of four 128-column accumulators: in pass 1 a row
+// tile (of MT) times a key tile, in pass 2 a key tile times a column chunk (of MT: all the rows, or with more than 128
+// rows the rows of one half of the window). Turn t uses accumulator t % 4; turns of parity 0 belong to issuer 0 and
+// softmax set 0, those of parity 1 to issuer 1 and set 1, so each pair works through its own two accumulators and the
+// pairs share nothing but the K ring and the tensor core. With two row tiles set `rt` always gets row tile `rt` and
+// the column chunk of window half `rt`.
+// LONG: the keys do not fit the shared-memory window sums at once (a prompt of more than kTcChunkKeys tokens).
+template <int WK, bool LONG>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_q, int n_cta, int stages, int q_bufs) {
-    constexpr int HW = WK / kTcGroups;   // window rows one softmax group handles in pass 2
+    constexpr int PW = score_tc_block_rows(WK);      // window rows of a block
+    constexpr int NB = WK / PW;                      // blocks of window rows: 2 or 4
+    constexpr int HB = 32 / PW;                      // heads whose block columns one 32-column tensor-memory load covers
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int R = p.g * WK;                          // query rows of an item, a multiple of 16
-    const int MT = (R + 127) >> 7;                   // 128-row tiles of pass 1
+    const int MT = (R + 127) >> 7;                   // 128-row tiles of pass 1 = column chunks of pass 2 = turns per key tile
+    const int mt_shift = MT - 1;                     // MT is 1 or 2
+    const int N2 = R >> mt_shift;                    // columns of a pass-2 product
     // the rows are loaded twice and the copies split a tile's keys (whole warps per copy: a warp reads one column range)
     const bool dup = 2 * R <= 128 && R % 32 == 0;
     const int q_half = MT * 128 * 128;               // bytes of one d-half of a Q buffer (d-low, then d-high)
@@ -163,13 +195,14 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
     float* s_c = reinterpret_cast<float*>(k_smem + stages * kTcKStageBytes);      // [256] m + log2 l of every local row
     float* s_pm = s_c + kTcMaxRows;                                               // [groups][128] partial row maxima
     float* s_pl = s_pm + kTcGroups * 128;                                         // [groups][128] partial row sums
-    // [2][c_pad] window sums of this item's rows: two groups add into each plane, so every sum has two addends and
-    // the result does not depend on the order in which the groups arrive. Caches hold at most kTcChunkKeys rows and
-    // fit whole; a longer key range (a prompt being compressed) passes through in chunks of kTcChunkKeys keys, each
-    // written out when pass 2, which walks the tiles from the last to the first, leaves it.
+    // [MT][c_pad] window sums of this item's rows: a plane per softmax set that adds to a key (one set with one column
+    // chunk, both with two), and within a plane the set's two groups add, so every sum is a + b (+ c + d in a fixed
+    // order at the end) and the result does not depend on the order in which the groups arrive. Caches hold at most
+    // kTcChunkKeys rows and fit whole; a longer key range (a prompt being compressed) passes through in chunks of
+    // kTcChunkKeys keys, each written out when pass 2, which walks the tiles from the last to the first, leaves it.
     float* s_sum = s_pl + kTcGroups * 128;
     const int c_pad = min((p.C + 63) & ~63, kTcChunkKeys);
-    ScoreTcTail* tail = reinterpret_cast<ScoreTcTail*>(s_sum + 2 * c_pad);
+    ScoreTcTail* tail = reinterpret_cast<ScoreTcTail*>(s_sum + MT * c_pad);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int total_items = p.n_layers * p.batch * p.h_kv * n_cta;
@@ -177,15 +210,18 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
     if (tid == 0) {
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tail->q_full[b]), 1);
-            mbar_init(smem_u32(&tail->q_empty[b]), 1);
+            mbar_init(smem_u32(&tail->q_empty[b]), 2);                        // one commit from either issuer
+        }
+        for (int b = 0; b < 4; ++b) {
             mbar_init(smem_u32(&tail->d_full[b]), 1);
-            mbar_init(smem_u32(&tail->d_empty[b]), kTcSoftmaxThreads / 32);   // one arrival per softmax warp
+            mbar_init(smem_u32(&tail->d_empty[b]), kTcSoftmaxThreads / 64);   // one arrival per warp of the set that reads it
         }
         for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(&tail->k_full[s]), 1);
-            mbar_init(smem_u32(&tail->k_empty[s]), 1);
+            mbar_init(smem_u32(&tail->k_empty[s]), MT);                       // one commit per turn that read the tile
         }
-        mbar_init(smem_u32(&tail->drain), 1);
+        mbar_init(smem_u32(&tail->drain[0]), 1);
+        mbar_init(smem_u32(&tail->drain[1]), 1);
         mbar_init(smem_u32(&tail->chunk_bar), kTcSoftmaxThreads / 32);
         tail->abort_flag = 0;
         tail->issued = 0;
@@ -197,7 +233,7 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
         tmem_relinquish_alloc_permit();
         tmem_fence_before_sync();
     }
-    for (int t = tid; t < 2 * c_pad; t += kTcThreads) s_sum[t] = 0.f;
+    for (int t = tid; t < MT * c_pad; t += kTcThreads) s_sum[t] = 0.f;
     // rows of the Q tiles that no copy fills take part in the pass-1 products: make them zeros (both buffers, once)
     {
         const int filled = dup ? 2 * R : R;
@@ -242,10 +278,12 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                         const int qrow0 = (d.ls * p.h_q + d.head * p.g) * p.w + d.k0;
                         uint8_t* qdst = q_smem + (size_t)qb * q_bytes;
                         for (int c = 0; c < (dup ? 2 : 1); ++c)
-                            for (int h = 0; h < p.g; ++h) {
-                                tma_load_2d(smem_u32(qdst + (size_t)(c * R + h * WK) * 128), &tm_q, 0, qrow0 + h * p.w, qbar);
-                                tma_load_2d(smem_u32(qdst + q_half + (size_t)(c * R + h * WK) * 128), &tm_q, 64, qrow0 + h * p.w, qbar);
-                            }
+                            for (int wrb = 0; wrb < NB; ++wrb)
+                                for (int h = 0; h < p.g; ++h) {
+                                    const uint32_t dst = smem_u32(qdst + (size_t)(c * R + (wrb * p.g + h) * PW) * 128);
+                                    tma_load_2d(dst, &tm_q, 0, qrow0 + h * p.w + wrb * PW, qbar);
+                                    tma_load_2d(dst + q_half, &tm_q, 64, qrow0 + h * p.w + wrb * PW, qbar);
+                                }
                         *(volatile int*)&tail->q_issued = j + 1;
                     }
                     if (i == total) break;
@@ -268,12 +306,20 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == kTcIssuerB) {
+        // ------------------------------------------------------------------ MMA issuers
+        // Two threads, one per turn parity. Issuing the eight instructions of a product, with its two waits before and
+        // its two commits after, takes one thread longer than the tensor core needs for them; with two threads one
+        // product's instructions are queued while the other's execute. The two never touch the same accumulator, and a
+        // commit covers the instructions of the thread that makes it, so a ring slot is released by every turn that read
+        // it (the barrier counts them) and the query buffer by both threads.
         if (lane == 0) {
+            const int me = warp == 1 ? 0 : 1;
             const uint32_t k_lo = umma_desc_lo(smem_u32(k_smem));
-            const uint32_t idesc1 = umma_idesc_bf16_m128(kTcTileKeys), idesc2 = umma_idesc_bf16_m128(R);
-            int s = 0, round = 0, ai = 0;            // ring position and accumulator turn, carried across items
+            const uint32_t idesc1 = umma_idesc_bf16_m128(kTcTileKeys), idesc2 = umma_idesc_bf16_m128(N2);
+            const int lstep = 2 >> mt_shift;            // K tiles between two turns of one issuer: 2 with one turn per tile, else 1
+            int s = (me >> mt_shift) % stages, round = (me >> mt_shift) / stages;   // ring position of this issuer's next turn
+            int t0 = 0;                                 // turn of the item's first product (always even)
             bool ok = true;
             for (int item = blockIdx.x, j = 0; ok && item < total_items; item += gridDim.x, ++j) {
                 const ScoreItem d = score_item(p, item, n_cta, WK);
@@ -283,10 +329,18 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                     break;
                 }
                 const uint32_t q_lo = umma_desc_lo(smem_u32(q_smem + (size_t)qb * q_bytes));
-                const int total = 2 * d.T;
-                for (int i = 0; i < total; ++i, ++ai) {
-                    const int buf = ai & 1;
-                    if (ai >= 2 && !tc_wait(smem_u32(&tail->d_empty[buf]), ((ai >> 1) - 1) & 1, &tail->abort_flag)) {
+                // this issuer's operand of the query tile: pass 1 row tile `me` (of two) or the only one; pass 2 the column
+                // chunk `me` (rows me * N2 ...) or all rows
+                const uint32_t q_off1 = (uint32_t)((MT == 2 ? me * 128 : 0) * 128) >> 4, q_off2 = (uint32_t)((MT == 2 ? me * N2 : 0) * 128) >> 4;
+                uint64_t q_desc[8];
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) q_desc[ks] = umma_desc(q_lo + umma_kstep(ks, q_half));
+                const int half_turns = d.T << mt_shift, total = 2 * half_turns;
+                for (int i = me; i < total; i += 2) {
+                    const int turn = t0 + i;
+                    const int acc = turn & 3, use = turn >> 2;   // accumulator of this turn and how often it has been used
+                    const uint32_t dcol = tmem_base + (uint32_t)(acc * kTcAccCols);
+                    if (use > 0 && !tc_wait(smem_u32(&tail->d_empty[acc]), (use - 1) & 1, &tail->abort_flag)) {
                         tc_abort(tail, p.status, 23);
                         ok = false;
                         break;
@@ -297,87 +351,84 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                         break;
                     }
                     tmem_fence_after_sync();
-                    const uint32_t ks_lo = k_lo + (uint32_t)s * (kTcKStageBytes >> 4);
-                    const uint32_t dcol = tmem_base + (uint32_t)buf * kTcAccCols;
-                    if (i < d.T) {
+                    const uint64_t k_desc = umma_desc(k_lo + (uint32_t)s * (kTcKStageBytes >> 4));
+                    if (i < half_turns) {
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks)
-                            umma_bf16(dcol, umma_desc(q_lo + umma_kstep(ks, q_half)), umma_desc(ks_lo + umma_kstep(ks, kTcKStageBytes / 2)),
-                                      idesc1, ks > 0);
-                        if (MT == 2) {
-#pragma unroll
-                            for (int ks = 0; ks < 8; ++ks)
-                                umma_bf16(dcol + 128, umma_desc(q_lo + ((128 * 128) >> 4) + umma_kstep(ks, q_half)),
-                                          umma_desc(ks_lo + umma_kstep(ks, kTcKStageBytes / 2)), idesc1, ks > 0);
-                        }
+                            umma_bf16(dcol, q_desc[ks] + q_off1, k_desc + umma_kstep(ks, kTcKStageBytes / 2), idesc1, ks > 0);
                     } else {
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks)
-                            umma_bf16(dcol, umma_desc(ks_lo + umma_kstep(ks, kTcKStageBytes / 2)), umma_desc(q_lo + umma_kstep(ks, q_half)),
-                                      idesc2, ks > 0);
+                            umma_bf16(dcol, k_desc + umma_kstep(ks, kTcKStageBytes / 2), q_desc[ks] + q_off2, idesc2, ks > 0);
                     }
                     umma_commit(smem_u32(&tail->k_empty[s]));
-                    umma_commit(smem_u32(&tail->d_full[buf]));
-                    if (++s == stages) { s = 0; ++round; }
+                    umma_commit(smem_u32(&tail->d_full[acc]));
+                    s += lstep;
+                    while (s >= stages) { s -= stages; ++round; }
                 }
-                if (ok) umma_commit(smem_u32(&tail->q_empty[qb]));   // the item's last product has read its queries
+                if (ok) umma_commit(smem_u32(&tail->q_empty[qb]));   // this issuer's last product of the item has read its queries
+                t0 += total;
             }
-            // everything issued has completed before the accumulators are given back
-            umma_commit(smem_u32(&tail->drain));
-            mbar_wait_bounded(smem_u32(&tail->drain), 0);
+            // everything this thread issued has completed before the accumulators are given back
+            umma_commit(smem_u32(&tail->drain[me]));
+            mbar_wait_bounded(smem_u32(&tail->drain[me]), 0);
         }
     } else {
         // ------------------------------------------------------------------ softmax warps
+        // Two sets of two groups: set 0 takes the turns of parity 0, set 1 those of parity 1, so one set's
+        // tensor-memory reads run under the other set's arithmetic.
         const int wg = (warp - 2) >> 2;               // group of four consecutive warps
+        const int set = wg >> 1, sub = wg & 1;
         const int q4 = warp & 3;                      // TMEM lane quarter this warp may touch
         const int L = q4 * 32 + lane;                 // TMEM lane = accumulator row of this thread
         const int stid = (warp - 2) * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q4 * 32) << 16);
         const float scale = p.scale_log2;
         bool ok = true;
-        int ai = 0;                                   // accumulator turn, carried across items
-        uint32_t chunk_phase = 0;
+        int t0 = 0;                                   // turn of the item's first product
+        [[maybe_unused]] uint32_t chunk_phase = 0;
 
-        // pass-1 role of this thread. Two 128-row tiles: two groups per tile, 64 keys each. One tile: all four
-        // groups, 32 keys each; with the rows loaded twice, 16 keys for each copy.
+        // pass-1 role of this thread: a row of the set's row tile, and 64 of a turn's 128 keys (32 for each copy when
+        // the rows are loaded twice)
         const int copy = dup ? (L >= R ? 1 : 0) : 0;
-        const int rl = (MT == 2) ? (wg >> 1) * 128 + L : L - copy * R;                    // local query row
+        const int rl = (MT == 2 ? set * 128 : 0) + L - copy * R;                          // local query row
         const bool valid = (MT == 2) ? rl < R : L < (dup ? 2 * R : R);
-        const int col0 = (MT == 2) ? (wg & 1) * 64 : wg * 32 + copy * 16;
-        const uint32_t t_p1 = t_lane + (uint32_t)((MT == 2) ? (wg >> 1) * 128 + col0 : col0);
+        const int col0 = sub * 64 + copy * 32;
+        const int nch1 = dup ? 1 : 2;                                                     // 32-key pieces per turn
+        const int blk = rl / PW;
+        const int row_k = (blk / p.g) * PW + (rl - blk * PW);                             // window row (within the item) of row rl
+        // pass-2 role: the blocks of window rows whose columns this thread reduces for its key. One column chunk: the set
+        // takes every other key tile and its two groups half of the window each; two chunks: the set takes the chunk of
+        // its half of the window, its two groups a quarter each.
+        const int nb2 = MT == 2 ? 1 : NB / 2;
+        const int wrb0 = MT == 2 ? set * (NB / 2) + sub : sub * (NB / 2);
+        const int colb0 = (MT == 2 ? sub : wrb0) * p.g * PW;                              // column of block wrb0 in the accumulator
+        const int plane = MT == 2 ? set * c_pad : 0;     // this set's plane of the window sums
 
         for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
             const ScoreItem d = score_item(p, item, n_cta, WK);
-            const int n = d.n, T = d.T, k0 = d.k0, total = 2 * T;
-            // ---- pass 1: online (max, sum) of the row this thread owns over its share of the tile's keys
-            const int last_vis = n - p.w + k0 + (rl % WK);    // last key the row's token sees
+            const int n = d.n, T = d.T, k0 = d.k0, half_turns = T << mt_shift, total = 2 * half_turns;
+            // ---- pass 1: online (max, sum) of the row this thread owns over its share of its set's turns
+            const int last_vis = n - p.w + k0 + row_k;        // last key the row's token sees
             float m_raw = -INFINITY, l = 0.f;                 // maximum in unscaled logits, sum relative to it
-            for (int i = 0; i < T; ++i, ++ai) {
-                const int buf = ai & 1;
-                ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (ai >> 1) & 1, &tail->abort_flag));
+            for (int i = set; i < half_turns; i += 2) {
+                const int turn = t0 + i, acc = turn & 3;
+                const uint32_t t_acc = t_lane + (uint32_t)(acc * kTcAccCols);
+                ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[acc]), (turn >> 2) & 1, &tail->abort_flag));
                 if (!ok) { tc_abort(tail, p.status, 25); break; }
                 tmem_fence_after_sync();
-                const int key_base = i * kTcTileKeys + col0;
-                const bool need_mask = i * kTcTileKeys + kTcTileKeys - 1 > n - p.w + k0;
-                if (MT == 2) {
+                const int kt = i >> mt_shift;
+                const int key_base = kt * kTcTileKeys + col0;
+                const bool need_mask = kt * kTcTileKeys + kTcTileKeys - 1 > n - p.w + k0;
 #pragma unroll 1
-                    for (int ch = 0; ch < 2; ++ch) {
-                        float z[32];
-                        tmem_ld<32>(t_p1 + (uint32_t)(buf * kTcAccCols + ch * 32), z);
-                        if (valid) row_update<32>(z, key_base + ch * 32, last_vis, need_mask, scale, m_raw, l);
-                    }
-                } else if (dup) {
-                    float z[16];
-                    tmem_ld<16>(t_p1 + (uint32_t)(buf * kTcAccCols), z);
-                    if (valid) row_update<16>(z, key_base, last_vis, need_mask, scale, m_raw, l);
-                } else {
+                for (int ch = 0; ch < nch1; ++ch) {
                     float z[32];
-                    tmem_ld<32>(t_p1 + (uint32_t)(buf * kTcAccCols), z);
-                    if (valid) row_update<32>(z, key_base, last_vis, need_mask, scale, m_raw, l);
+                    tmem_ld<32>(t_acc + (uint32_t)(col0 + ch * 32), z);
+                    if (valid) row_update<32>(z, key_base + ch * 32, last_vis, need_mask, scale, m_raw, l);
                 }
                 tmem_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&tail->d_empty[buf]));
+                if (lane == 0) mbar_arrive(smem_u32(&tail->d_empty[acc]));
             }
             // (a warp whose wait gave up still walks through every barrier below; all leave together at a point
             // where one thread's view of the abort flag decides for everybody)
@@ -385,8 +436,9 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
             s_pm[wg * 128 + L] = m_raw * scale;
             s_pl[wg * 128 + L] = l;
             softmax_bar_sync();
-            if ((MT == 2) ? (wg & 1) == 0 : (wg == 0 && L < R)) {
-                const int first = (MT == 2) ? wg : 0, count = (MT == 2) ? 2 : kTcGroups;   // groups that shared this row
+            if ((MT == 2) ? sub == 0 : (wg == 0 && L < R)) {
+                // the groups that shared this row: with two row tiles, the two groups of the set; else all four
+                const int first = (MT == 2) ? set * 2 : 0, count = (MT == 2) ? 2 : kTcGroups;
                 float mm = -INFINITY, ll = 0.f;
                 for (int c = 0; c <= (dup ? 1 : 0); ++c)
                     for (int q = first; q < first + count; ++q) mm = fmaxf(mm, s_pm[q * 128 + L + c * R]);
@@ -395,33 +447,39 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                         const float mq = s_pm[q * 128 + L + c * R];
                         ll += (mq == -INFINITY) ? 0.f : s_pl[q * 128 + L + c * R] * fast_exp2(mq - mm);
                     }
-                s_c[(MT == 2) ? rl : L] = mm + log2f(ll);
+                if (rl < R) s_c[rl] = mm + log2f(ll);
             }
             if (stid == 0) tail->abort_seen = *(volatile int*)&tail->abort_flag;
             softmax_bar_sync();
             if (*(volatile int*)&tail->abort_seen) break;
 
-            // ---- pass 2: this thread owns key `tile * 128 + L`; group wg covers window rows k0 + wg*HW .. + HW - 1
-            float* out = p.sacc + (size_t)d.unit * p.C;
+            // ---- pass 2: this thread owns key `tile * 128 + L` of its set's turns
             // window sums of keys [lo, lo + c_pad) leave shared memory (which is zeroed for the next chunk or item)
             auto flush_chunk = [&](int lo) {
+                float* out = p.sacc + (size_t)d.unit * p.C;
                 const int hi = min(lo + c_pad, p.C);
                 for (int t = lo + stid; t < hi; t += kTcSoftmaxThreads) {
-                    const float v = s_sum[t - lo] + s_sum[c_pad + t - lo];
+                    float v = s_sum[t - lo];
                     s_sum[t - lo] = 0.f;
-                    s_sum[c_pad + t - lo] = 0.f;
+                    if (MT == 2) {
+                        v += s_sum[c_pad + t - lo];
+                        s_sum[c_pad + t - lo] = 0.f;
+                    }
                     if (n_cta == 1) out[t] = (t < n) ? v : 0.f;
                     else if (t < n) atomicAdd(&out[t], v);   // buffer zeroed by the host
                 }
             };
-            int chunk_lo = T > 0 ? ((T - 1) * kTcTileKeys / c_pad) * c_pad : 0;
-            for (int i = T; ok && i < total; ++i, ++ai) {
-                const int buf = ai & 1;
-                const int tile_lo = ((total - 1 - i) * kTcTileKeys / c_pad) * c_pad;
+            int chunk_lo = 0;
+            if constexpr (LONG) chunk_lo = T > 0 ? ((T - 1) * kTcTileKeys / c_pad) * c_pad : 0;
+            for (int i = half_turns + ((half_turns ^ set) & 1); ok && i < total; i += 2) {   // this set's turns of pass 2
+                const int turn = t0 + i, acc = turn & 3;
+                const int tile = T - 1 - ((i - half_turns) >> mt_shift);
+                if constexpr (LONG) {
+                const int tile_lo = (tile * kTcTileKeys / c_pad) * c_pad;
                 if (tile_lo != chunk_lo) {
                     // Every softmax warp has added its part of the chunk; then the chunk is written and cleared; then all
                     // go on. mbarrier waits, not bar.sync: a warp that gives up (abort flag) must not leave the others at
-                    // a barrier it will never reach.
+                    // a barrier it will never reach. (A chunk is 64 tiles, so both sets cross every boundary once.)
                     for (int step = 0; ok && step < 2; ++step) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&tail->chunk_bar));
@@ -432,50 +490,73 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                     if (!ok) { tc_abort(tail, p.status, 27); break; }
                     chunk_lo = tile_lo;
                 }
-                ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (ai >> 1) & 1, &tail->abort_flag));
+                }
+                const uint32_t t_acc = t_lane + (uint32_t)(acc * kTcAccCols);
+                ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[acc]), (turn >> 2) & 1, &tail->abort_flag));
                 if (!ok) { tc_abort(tail, p.status, 26); break; }
                 tmem_fence_after_sync();
-                float v[HW];
+                const int key = tile * kTcTileKeys + L;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll 1
+                for (int b = 0; b < nb2; ++b) {
+                    const int wrb = wrb0 + b;
+                    float v[PW];
 #pragma unroll
-                for (int jj = 0; jj < HW; ++jj) v[jj] = -INFINITY;
-                for (int h = 0; h < p.g; ++h) {
-                    float z[HW];
-                    tmem_ld<HW>(t_lane + (uint32_t)(buf * kTcAccCols + h * WK + wg * HW), z);
-                    const float4* c4 = reinterpret_cast<const float4*>(s_c + h * WK + wg * HW);
+                    for (int jj = 0; jj < PW; ++jj) v[jj] = -INFINITY;
+                    for (int h0 = 0; h0 < p.g; h0 += HB) {
+                        float z[32];
+                        tmem_ld<32>(t_acc + (uint32_t)(colb0 + (b * p.g + h0) * PW), z);
+                        const float4* c4 = reinterpret_cast<const float4*>(s_c + (wrb * p.g + h0) * PW);
 #pragma unroll
-                    for (int jj = 0; jj < HW; jj += 4) {
-                        const float4 c = c4[jj >> 2];
-                        v[jj] = fmaxf(v[jj], fmaf(z[jj], scale, -c.x));
-                        v[jj + 1] = fmaxf(v[jj + 1], fmaf(z[jj + 1], scale, -c.y));
-                        v[jj + 2] = fmaxf(v[jj + 2], fmaf(z[jj + 2], scale, -c.z));
-                        v[jj + 3] = fmaxf(v[jj + 3], fmaf(z[jj + 3], scale, -c.w));
+                        for (int hh = 0; hh < HB; hh += 2) {
+                            if (h0 + hh + 1 < p.g) {          // two heads per maximum
+#pragma unroll
+                                for (int jj = 0; jj < PW; jj += 4) {
+                                    const float4 c = c4[(hh * PW + jj) >> 2], e = c4[((hh + 1) * PW + jj) >> 2];
+                                    v[jj] = max3(v[jj], fmaf(z[hh * PW + jj], scale, -c.x), fmaf(z[(hh + 1) * PW + jj], scale, -e.x));
+                                    v[jj + 1] = max3(v[jj + 1], fmaf(z[hh * PW + jj + 1], scale, -c.y), fmaf(z[(hh + 1) * PW + jj + 1], scale, -e.y));
+                                    v[jj + 2] = max3(v[jj + 2], fmaf(z[hh * PW + jj + 2], scale, -c.z), fmaf(z[(hh + 1) * PW + jj + 2], scale, -e.z));
+                                    v[jj + 3] = max3(v[jj + 3], fmaf(z[hh * PW + jj + 3], scale, -c.w), fmaf(z[(hh + 1) * PW + jj + 3], scale, -e.w));
+                                }
+                            } else if (h0 + hh < p.g) {
+#pragma unroll
+                                for (int jj = 0; jj < PW; jj += 4) {
+                                    const float4 c = c4[(hh * PW + jj) >> 2];
+                                    v[jj] = fmaxf(v[jj], fmaf(z[hh * PW + jj], scale, -c.x));
+                                    v[jj + 1] = fmaxf(v[jj + 1], fmaf(z[hh * PW + jj + 1], scale, -c.y));
+                                    v[jj + 2] = fmaxf(v[jj + 2], fmaf(z[hh * PW + jj + 2], scale, -c.z));
+                                    v[jj + 3] = fmaxf(v[jj + 3], fmaf(z[hh * PW + jj + 3], scale, -c.w));
+                                }
+                            }
+                        }
+                    }
+                    if (b == nb2 - 1) {   // the last read of this turn: the accumulator goes back before the exponentials
+                        tmem_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&tail->d_empty[acc]));
+                    }
+                    const int fk = key - (n - p.w) - k0 - wrb * PW;   // rows before it decoded before this key existed
+#pragma unroll
+                    for (int jj = 0; jj < PW; jj += 2) {
+                        s0 += (jj >= fk) ? fast_exp2(v[jj]) : 0.f;
+                        s1 += (jj + 1 >= fk) ? fast_exp2(v[jj + 1]) : 0.f;
                     }
                 }
-                tmem_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&tail->d_empty[buf]));
-                const int key = (total - 1 - i) * kTcTileKeys + L;
-                if (key < n) {
-                    const int first_k = key - (n - p.w) - k0 - wg * HW;   // rows jj < first_k decoded before this key existed
-                    float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-                    for (int jj = 0; jj < HW; jj += 2) {
-                        s0 += (jj >= first_k) ? fast_exp2(v[jj]) : 0.f;
-                        s1 += (jj + 1 >= first_k) ? fast_exp2(v[jj + 1]) : 0.f;
-                    }
-                    atomicAdd(&s_sum[(wg >> 1) * c_pad + key - chunk_lo], s0 + s1);
-                }
+                if (key < n) atomicAdd(&s_sum[plane + key - chunk_lo], s0 + s1);   // two addends per key and plane (the set's two groups)
             }
             softmax_bar_sync();
             if (stid == 0) tail->abort_seen = *(volatile int*)&tail->abort_flag;
             if (ok && !*(volatile int*)&tail->abort_flag) {
                 flush_chunk(chunk_lo);   // the chunk of the first tile, walked last
                 // rows past the chunk that holds the last key were never in shared memory
-                if (n_cta == 1)
+                if (n_cta == 1) {
+                    float* out = p.sacc + (size_t)d.unit * p.C;
                     for (int t = (T > 0 ? ((T - 1) * kTcTileKeys / c_pad + 1) * c_pad : 0) + stid; t < p.C; t += kTcSoftmaxThreads) out[t] = 0.f;
+                }
             }
             softmax_bar_sync();      // the sums are clear and the row constants free before the next item uses them
             if (*(volatile int*)&tail->abort_seen) break;
+            t0 += total;
         }
     }
 
@@ -499,8 +580,11 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
 static size_t score_tc_smem_bytes(int C, int rows, int stages, int q_bufs) {
     const int mt = (rows + 127) >> 7;
     return 1024 + (size_t)q_bufs * mt * 128 * kRowBytes + (size_t)stages * kTcKStageBytes +
-           sizeof(float) * (kTcMaxRows + 2 * kTcGroups * 128 + 2 * min((C + 63) & ~63, kTcChunkKeys)) + sizeof(ScoreTcTail);
+           sizeof(float) * (kTcMaxRows + 2 * kTcGroups * 128 + mt * min((C + 63) & ~63, kTcChunkKeys)) + sizeof(ScoreTcTail);
 }
+
+// Rows of one box of the window-query tensor map (the kernel loads the queries block by block).
+int score_tc_q_box_rows(int wk) { return score_tc_block_rows(wk); }
 
 // Window rows per item for this shape, or 0 when the shape is left to the mma.sync kernel.
 int score_tc_rows_per_cta(int g, int w) {
@@ -511,11 +595,14 @@ int score_tc_rows_per_cta(int g, int w) {
 }
 
 cudaError_t score_tc_kernel_setup() {
-    cudaError_t e = cudaFuncSetAttribute(gkv_score_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(gkv_score_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(gkv_score_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    const void* kernels[6] = {(const void*)gkv_score_tc_kernel<16, false>, (const void*)gkv_score_tc_kernel<32, false>,
+                              (const void*)gkv_score_tc_kernel<64, false>, (const void*)gkv_score_tc_kernel<16, true>,
+                              (const void*)gkv_score_tc_kernel<32, true>,  (const void*)gkv_score_tc_kernel<64, true>};
+    for (const void* k : kernels) {
+        const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s) {
@@ -527,6 +614,10 @@ cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const
     const int q_bufs = score_tc_smem_bytes(p.C, rows, 3, 2) <= 227 * 1024 ? 2 : 1;
     int stages = 2;
     while (stages < kTcMaxStages && score_tc_smem_bytes(p.C, rows, stages + 1, q_bufs) <= 227 * 1024) ++stages;
+    // With one turn per key tile the two issuers take alternate tiles. The ring depth must then be even, so that a ring
+    // slot always belongs to the same issuer: a thread that saw only every other phase of a slot's barrier could pass a
+    // parity wait two phases early. (With two turns per tile both issuers wait for every tile.)
+    if (rows <= 128) stages &= ~1;
     const size_t smem = score_tc_smem_bytes(p.C, rows, stages, q_bufs);
     if (n_cta > 1) {
         const size_t off = (size_t)p.layer0 * p.batch * p.h_kv * p.C;
@@ -540,9 +631,13 @@ cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const
         const int rounds = (items + sm - 1) / sm;
         grid = (items + rounds - 1) / rounds;
     }
-    if (wk == 16) gkv_score_tc_kernel<16><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
-    else if (wk == 32) gkv_score_tc_kernel<32><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
-    else gkv_score_tc_kernel<64><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
+    const bool chunked = p.C > kTcChunkKeys;
+    if (wk == 16 && !chunked) gkv_score_tc_kernel<16, false><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
+    else if (wk == 32 && !chunked) gkv_score_tc_kernel<32, false><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
+    else if (!chunked) gkv_score_tc_kernel<64, false><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
+    else if (wk == 16) gkv_score_tc_kernel<16, true><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
+    else if (wk == 32) gkv_score_tc_kernel<32, true><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
+    else gkv_score_tc_kernel<64, true><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);
     return cudaGetLastError();
 }
 
