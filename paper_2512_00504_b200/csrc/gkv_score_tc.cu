@@ -26,7 +26,7 @@
 // with two accumulators of its own, one pair's waits and loads run under the other's work.
 //
 // Pass 1 is bound by the instructions of the exponentials (one per logit; the special-function unit
-// does 16 a clock and SM): half of them are evaluated on the FMA pipe instead, as
+// does 16 a clock and SM): a quarter of them are evaluated on the FMA pipe instead, as
 // 2^x = 2^round(x) * P(x - round(x)) with a cubic P (relative error < 8e-5; pass 1 only feeds the
 // row sums, and the scores are compared at 1e-3). With at most 64 query rows the rows are loaded
 // twice (lanes 64-127 of the accumulator repeat lanes 0-63) and the two copies split the keys of a
@@ -100,8 +100,8 @@ __device__ __forceinline__ float2 exp2_fma_pair(float xa, float xb) {
 }
 
 // Online (max, sum) of one query row over N more keys whose raw logits are z[0..N): `m_raw` is the running maximum
-// of the unscaled logits, `l` the sum of 2^((z - m_raw) * scale). Half of the exponentials go to the special-function
-// unit, half to the FMA pipe.
+// of the unscaled logits, `l` the sum of 2^((z - m_raw) * scale). Three quarters of the exponentials go to the
+// special-function unit, a quarter to the FMA pipe.
 template <int N>
 __device__ __forceinline__ void row_update(float (&z)[N], int key0, int last_vis, bool need_mask, float scale,
                                            float& m_raw, float& l) {
@@ -125,10 +125,14 @@ __device__ __forceinline__ void row_update(float (&z)[N], int key0, int last_vis
     float2 sp = make_float2(0.f, 0.f);
     const float2 sc2 = make_float2(scale, scale), ng2 = make_float2(neg, neg);
 #pragma unroll
-    for (int j = 0; j < N; j += 4) {
+    for (int j = 0; j < N; j += 8) {
         s0 += fast_exp2(fmaf(z[j], scale, neg));
         s1 += fast_exp2(fmaf(z[j + 1], scale, neg));
-        const float2 a = fma_f32x2(make_float2(z[j + 2], z[j + 3]), sc2, ng2);
+        s0 += fast_exp2(fmaf(z[j + 2], scale, neg));
+        s1 += fast_exp2(fmaf(z[j + 3], scale, neg));
+        s0 += fast_exp2(fmaf(z[j + 4], scale, neg));
+        s1 += fast_exp2(fmaf(z[j + 5], scale, neg));
+        const float2 a = fma_f32x2(make_float2(z[j + 6], z[j + 7]), sc2, ng2);
         const float2 e = exp2_fma_pair(a.x, a.y);
         sp = fma_f32x2(e, make_float2(1.f, 1.f), sp);
     }
