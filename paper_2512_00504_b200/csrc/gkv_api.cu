@@ -102,23 +102,45 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// 2-D view of a buffer of 128-element bf16 rows: [rows][128], boxes of box_rows rows x 64 elements,
-// 128-byte swizzle (K and V: 64-row boxes; the window queries: one box per head slice).
-gkv_status encode_map(CUtensorMap* map, void* base, uint64_t rows, uint32_t box_rows = kTileKeys) {
+// The driver's tensor-map encoder, looked up once (no link-time dependency on libcuda).
+EncodeTiledFn encode_tiled_fn() {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
         void* sym = nullptr;
         cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess || !sym)
-            return GKV_ERR_CUDA;
-        fn = reinterpret_cast<EncodeTiledFn>(sym);
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess && sym)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
     }
+    return fn;
+}
+
+// 2-D view of a buffer of 128-element bf16 rows: [rows][128], boxes of box_rows rows x 64 elements,
+// 128-byte swizzle (K and V: 64-row boxes; 16-row and 128-row boxes for the kernels that want them).
+gkv_status encode_map(CUtensorMap* map, void* base, uint64_t rows, uint32_t box_rows = kTileKeys) {
+    const EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return GKV_ERR_CUDA;
     const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
     const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? GKV_OK : GKV_ERR_CUDA;
+}
+
+// 3-D view of the window queries [heads][w][128] bf16 for the tensor-core scoring kernel: one box = box_rows
+// consecutive window rows of `g` consecutive heads x 64 elements (128-byte swizzle), so a block of window rows of all
+// the heads of a KV head arrives with one copy, head after head.
+gkv_status encode_query_map(CUtensorMap* map, const void* base, uint64_t heads, uint32_t w, uint32_t box_rows, uint32_t g) {
+    const EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return GKV_ERR_CUDA;
+    const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)w, (cuuint64_t)heads};
+    const cuuint64_t strides[2] = {(cuuint64_t)kRowBytes, (cuuint64_t)kRowBytes * w};
+    const cuuint32_t box[3] = {64, box_rows, g};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? GKV_OK : GKV_ERR_CUDA;
@@ -187,14 +209,14 @@ gkv_status launch_redundancy_for(gkv_ctx* ctx, int l0, int nl, cudaStream_t s) {
 }
 
 // tcgen05 kernel for windows that split into 16-, 32- or 64-row slices; the mma.sync kernel covers the rest.
-gkv_status dispatch_score(gkv_ctx* ctx, const ScoreLaunch& sp, const CUtensorMap& tm_k, cudaStream_t s) {
+gkv_status dispatch_score(gkv_ctx* ctx, const ScoreLaunch& sp, const CUtensorMap& tm_k, const CUtensorMap& tm_k128, cudaStream_t s) {
     const gkv_config& c = ctx->cfg;
     const int wk = score_tc_rows_per_cta(ctx->g, c.window);
     if (wk > 0 && (reinterpret_cast<uintptr_t>(sp.q_win) & 15) == 0) {
         CUtensorMap tm_q;
-        const uint64_t q_rows = (uint64_t)sp.n_layers * c.batch * c.n_q_heads * c.window;
-        if (encode_map(&tm_q, const_cast<__nv_bfloat16*>(sp.q_win), q_rows, (uint32_t)score_tc_q_box_rows(wk)) != GKV_OK) return GKV_ERR_CUDA;
-        if (launch_score_tc(sp, tm_k, tm_q, wk, s) != cudaSuccess) return GKV_ERR_CUDA;
+        const uint64_t q_heads = (uint64_t)sp.n_layers * c.batch * c.n_q_heads;
+        if (encode_query_map(&tm_q, sp.q_win, q_heads, (uint32_t)c.window, (uint32_t)score_tc_q_box_rows(wk), (uint32_t)ctx->g) != GKV_OK) return GKV_ERR_CUDA;
+        if (launch_score_tc(sp, tm_k128, tm_q, wk, s) != cudaSuccess) return GKV_ERR_CUDA;
     } else if (sp.C > kMaxPromptShared) {
         return GKV_ERR_INVALID_ARG;   // a long prompt with misaligned window queries: the other kernel holds all sums on chip
     } else if (launch_score(sp, tm_k, s) != cudaSuccess) {
@@ -214,7 +236,7 @@ gkv_status launch_score_for(gkv_ctx* ctx, int l0, int nl, const void* q_window, 
     sp.layer0 = l0; sp.n_layers = nl; sp.batch = c.batch; sp.h_q = c.n_q_heads; sp.h_kv = c.n_kv_heads;
     sp.g = ctx->g; sp.C = ctx->C; sp.w = c.window; sp.sm_count = ctx->sm_count;
     sp.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
-    return dispatch_score(ctx, sp, ctx->tm_k, s);
+    return dispatch_score(ctx, sp, ctx->tm_k, ctx->tm_k128, s);
 }
 
 // Shared validation of an eviction request. Returns GKV_OK with *noop set when len <= b.
@@ -338,7 +360,7 @@ gkv_status gkv_init(gkv_ctx** out, const gkv_config* cfg, const gkv_buffers* b, 
     if (ok) {
         const uint64_t rows = (uint64_t)cfg->n_layers * ctx->units_per_layer * ctx->C;
         ok = encode_map(&ctx->tm_k, b->k, rows) == GKV_OK && encode_map(&ctx->tm_v, b->v, rows) == GKV_OK &&
-             encode_map(&ctx->tm_k16, b->k, rows, 16) == GKV_OK && encode_map(&ctx->tm_v16, b->v, rows, 16) == GKV_OK;
+             encode_map(&ctx->tm_k128, b->k, rows, kScoreTcKeyBoxRows) == GKV_OK && encode_map(&ctx->tm_k16, b->k, rows, 16) == GKV_OK && encode_map(&ctx->tm_v16, b->v, rows, 16) == GKV_OK;
     }
     if (!ok) {
         (void)cudaGetLastError();
@@ -617,9 +639,11 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
     }
     float* sums = ws_ptr<float>(ctx, ctx->ws.prompt_sums);
     if (any_long && scored) {
-        CUtensorMap tm_kp;
+        CUtensorMap tm_kp, tm_kp128;
         const uint64_t rows = (uint64_t)c.batch * c.n_kv_heads * c.max_prompt;
-        if (encode_map(&tm_kp, const_cast<void*>(k_prompt), rows) != GKV_OK) return GKV_ERR_CUDA;
+        if (encode_map(&tm_kp, const_cast<void*>(k_prompt), rows) != GKV_OK ||
+            encode_map(&tm_kp128, const_cast<void*>(k_prompt), rows, kScoreTcKeyBoxRows) != GKV_OK)
+            return GKV_ERR_CUDA;
         ScoreLaunch sp;
         sp.q_win = static_cast<const __nv_bfloat16*>(q_window);
         sp.sacc = sums;
@@ -628,7 +652,7 @@ gkv_status gkv_compress_prompt(gkv_ctx* ctx, int32_t layer, const void* k_prompt
         sp.layer0 = 0; sp.n_layers = 1; sp.batch = c.batch; sp.h_q = c.n_q_heads; sp.h_kv = c.n_kv_heads;
         sp.g = ctx->g; sp.C = c.max_prompt; sp.w = c.window; sp.sm_count = ctx->sm_count;
         sp.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kHeadDim));
-        const gkv_status st = dispatch_score(ctx, sp, tm_kp, s);
+        const gkv_status st = dispatch_score(ctx, sp, tm_kp, tm_kp128, s);
         if (st != GKV_OK) {
             (void)cudaGetLastError();
             return st;

@@ -135,6 +135,7 @@ struct gkv_ctx {
     int device, sm_count;
     CUtensorMap tm_k, tm_v;   // 64-row boxes
     CUtensorMap tm_k16, tm_v16;   // 16-row boxes
+    CUtensorMap tm_k128;          // 128-row boxes (the tensor-core scoring kernel's key tiles)
     std::vector<int32_t> len, n_hist, since_evict, sacc_valid, stage_next, cbar_valid;
     int64_t launches;
     int32_t* evict_log;  // caller's device buffer for the eviction log, or NULL
@@ -156,6 +157,7 @@ cudaError_t launch_score(const ScoreLaunch& p, const CUtensorMap& tm_k, cudaStre
 cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s);
 int score_tc_rows_per_cta(int g, int w);
 int score_tc_q_box_rows(int wk);
+constexpr int kScoreTcKeyBoxRows = 128;   // rows of one box of the key tensor map that launch_score_tc takes
 cudaError_t score_tc_kernel_setup();
 cudaError_t launch_prompt_compress(const PromptLaunch& p, cudaStream_t s);
 cudaError_t launch_keynorm(const RedundancyLaunch& p, cudaStream_t s);

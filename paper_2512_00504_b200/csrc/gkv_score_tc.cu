@@ -205,7 +205,7 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
     // kTcChunkKeys rows and fit whole; a longer key range (a prompt being compressed) passes through in chunks of
     // kTcChunkKeys keys, each written out when pass 2, which walks the tiles from the last to the first, leaves it.
     float* s_sum = s_pl + kTcGroups * 128;
-    const int c_pad = min((p.C + 63) & ~63, kTcChunkKeys);
+    const int c_pad = LONG ? kTcChunkKeys : min((p.C + 63) & ~63, kTcChunkKeys);   // LONG: a chunk is 64 key tiles
     ScoreTcTail* tail = reinterpret_cast<ScoreTcTail*>(s_sum + MT * c_pad);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -279,15 +279,15 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                         }
                         const uint32_t qbar = smem_u32(&tail->q_full[qb]);
                         mbar_arrive_expect_tx(qbar, (uint32_t)(dup ? 2 * R : R) * kRowBytes);
-                        const int qrow0 = (d.ls * p.h_q + d.head * p.g) * p.w + d.k0;
+                        const int qhead0 = d.ls * p.h_q + d.head * p.g;   // first query head of the unit
                         uint8_t* qdst = q_smem + (size_t)qb * q_bytes;
+                        // one box = a block of window rows of all g heads (the query map is [heads][w][d])
                         for (int c = 0; c < (dup ? 2 : 1); ++c)
-                            for (int wrb = 0; wrb < NB; ++wrb)
-                                for (int h = 0; h < p.g; ++h) {
-                                    const uint32_t dst = smem_u32(qdst + (size_t)(c * R + (wrb * p.g + h) * PW) * 128);
-                                    tma_load_2d(dst, &tm_q, 0, qrow0 + h * p.w + wrb * PW, qbar);
-                                    tma_load_2d(dst + q_half, &tm_q, 64, qrow0 + h * p.w + wrb * PW, qbar);
-                                }
+                            for (int wrb = 0; wrb < NB; ++wrb) {
+                                const uint32_t dst = smem_u32(qdst + (size_t)(c * R + wrb * p.g * PW) * 128);
+                                tma_load_3d(dst, &tm_q, 0, d.k0 + wrb * PW, qhead0, qbar);
+                                tma_load_3d(dst + q_half, &tm_q, 64, d.k0 + wrb * PW, qhead0, qbar);
+                            }
                         *(volatile int*)&tail->q_issued = j + 1;
                     }
                     if (i == total) break;
@@ -301,10 +301,8 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                     const uint32_t dst = smem_u32(k_smem + (size_t)s * kTcKStageBytes);
                     const int y = d.row0 + tile * kTcTileKeys;
                     mbar_arrive_expect_tx(bar, kTcKStageBytes);
-                    tma_load_2d(dst, &tm_k, 0, y, bar);
-                    tma_load_2d(dst + kBoxBytes, &tm_k, 0, y + 64, bar);
-                    tma_load_2d(dst + 2 * kBoxBytes, &tm_k, 64, y, bar);
-                    tma_load_2d(dst + 3 * kBoxBytes, &tm_k, 64, y + 64, bar);
+                    tma_load_2d(dst, &tm_k, 0, y, bar);                      // 128-row boxes: d-low half, d-high half
+                    tma_load_2d(dst + kTcKStageBytes / 2, &tm_k, 64, y, bar);
                     *(volatile int*)&tail->issued = ++issued;
                     if (++s == stages) { s = 0; ++round; }
                 }
@@ -474,12 +472,12 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                 }
             };
             int chunk_lo = 0;
-            if constexpr (LONG) chunk_lo = T > 0 ? ((T - 1) * kTcTileKeys / c_pad) * c_pad : 0;
+            if constexpr (LONG) chunk_lo = T > 0 ? (((T - 1) * kTcTileKeys) & ~(kTcChunkKeys - 1)) : 0;
             for (int i = half_turns + ((half_turns ^ set) & 1); ok && i < total; i += 2) {   // this set's turns of pass 2
                 const int turn = t0 + i, acc = turn & 3;
                 const int tile = T - 1 - ((i - half_turns) >> mt_shift);
                 if constexpr (LONG) {
-                const int tile_lo = (tile * kTcTileKeys / c_pad) * c_pad;
+                const int tile_lo = (tile * kTcTileKeys) & ~(kTcChunkKeys - 1);
                 if (tile_lo != chunk_lo) {
                     // Every softmax warp has added its part of the chunk; then the chunk is written and cleared; then all
                     // go on. mbarrier waits, not bar.sync: a warp that gives up (abort flag) must not leave the others at
