@@ -11,8 +11,9 @@
 // Two launches: gkv_keynorm_kernel writes 1 / (|K_t| + eps) per cached row; gkv_redundancy_tc_kernel
 // (one CTA per unit and block of 256 keys) keeps its 256 keys resident in shared memory as the A
 // operand (two 128-row tiles), streams all keys of the unit as 128-key B tiles by TMA, accumulates
-// D[own key][other key] in two 256-column TMEM buffers, and 16 epilogue warps (same roles and
-// barriers as the scoring kernel) scale, threshold and add. The softmax and the max-normalisation
+// D[own key][other key] in two 256-column TMEM buffers (warp 0 copies, one thread of warp 1 issues
+// the tcgen05.mma), and 16 epilogue warps, eight per buffer, scale, threshold and add; every wait is
+// bounded and latches a status word like the scoring kernel's. The softmax and the max-normalisation
 // of the appendix reduce to exp(cbar - max cbar), which the eviction kernel applies.
 #include "gkv_common.cuh"
 #include "gkv_internal.h"
