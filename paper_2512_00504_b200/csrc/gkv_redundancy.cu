@@ -11,9 +11,10 @@
 // Two launches: gkv_keynorm_kernel writes 1 / (|K_t| + eps) per cached row; gkv_redundancy_tc_kernel
 // (one CTA per unit and block of 256 keys) keeps its 256 keys resident in shared memory as the A
 // operand (two 128-row tiles), streams all keys of the unit as 128-key B tiles by TMA, accumulates
-// D[own key][other key] in two 256-column TMEM buffers (warp 0 copies, one thread of warp 1 issues
-// the tcgen05.mma), and 16 epilogue warps, eight per buffer, scale, threshold and add; every wait is
-// bounded and latches a status word like the scoring kernel's. The softmax and the max-normalisation
+// D[own key][other key] in four 128-column TMEM accumulators (warp 0 copies; the 128 x 128 products
+// are issued by two threads, warps 1 and 18, one per turn parity), and 16 epilogue warps in two
+// sets, one per turn parity, scale, threshold and add; every wait is bounded and latches a status
+// word like the scoring kernel's. The softmax and the max-normalisation
 // of the appendix reduce to exp(cbar - max cbar), which the eviction kernel applies.
 #include "gkv_common.cuh"
 #include "gkv_internal.h"
@@ -23,13 +24,14 @@ namespace gkv {
 
 constexpr int kRdGroups = 4;
 constexpr int kRdEpiThreads = kRdGroups * 128;
-constexpr int kRdThreads = 64 + kRdEpiThreads;
+constexpr int kRdIssuerB = 2 + kRdEpiThreads / 32;          // the warp after the epilogue warps: second tcgen05.mma issuer
+constexpr int kRdThreads = 64 + kRdEpiThreads + 32;
 constexpr int kRdTileKeys = 128;
 constexpr int kRdBlockRows = 256;
 constexpr int kRdMaxStages = 4;
 constexpr int kRdStageBytes = kRdTileKeys * kRowBytes;       // 32 KB: d-low half then d-high half
 constexpr int kRdABytes = kRdBlockRows * kRowBytes;          // 64 KB
-constexpr int kRdAccCols = 256;
+constexpr int kRdAccCols = 128;                              // TMEM columns of one accumulator (four of them)
 constexpr uint32_t kRdTmemCols = 512;
 
 // ---------------------------------------------------------------------------------------------
@@ -69,9 +71,9 @@ struct __align__(8) RedundancyTail {
     uint64_t a_full;
     uint64_t k_full[kRdMaxStages];
     uint64_t k_empty[kRdMaxStages];
-    uint64_t d_full[2];
-    uint64_t d_empty[2];
-    uint64_t drain;
+    uint64_t d_full[4];
+    uint64_t d_empty[4];
+    uint64_t drain[2];
     uint32_t tmem_base;
     int abort_flag;
     int issued;
@@ -83,11 +85,9 @@ __device__ __forceinline__ void rd_abort(RedundancyTail* tail, int32_t* status, 
         status[2] = blockIdx.x;
     }
 }
-// 1.0f where a >= b, else 0.0f (also for NaN).
-__device__ __forceinline__ float ge_mask(float a, float b) {
-    float m;
-    asm("set.ge.f32.f32 %0, %1, %2;" : "=f"(m) : "f"(a), "f"(b));
-    return m;
+// s += t where t >= thr (not for NaN).
+__device__ __forceinline__ void add_if_ge(float& s, float t, float thr) {
+    asm("{.reg .pred p; setp.ge.f32 p, %1, %2; @p add.f32 %0, %0, %1;}" : "+f"(s) : "f"(t), "f"(thr));
 }
 __device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kRdEpiThreads) : "memory"); }
 
@@ -117,19 +117,22 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
     if (a0 >= n) return;                              // the whole CTA: no key of the cache in this block
     const int T = (n + kRdTileKeys - 1) / kRdTileKeys;
     const int row0 = (int)(unit * p.C);
-    const int MT = (min(kRdBlockRows, n - a0) + 127) >> 7;
+    const int MT = (min(kRdBlockRows, n - a0) + 127) >> 7;   // row tiles of this block = turns per key tile
+    const int mt_shift = MT - 1;
+    const int total = T << mt_shift;                           // turns: one 128 x 128 product each
 
     if (tid == 0) {
         mbar_init(smem_u32(&tail->a_full), 1);
         for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(&tail->k_full[s]), 1);
-            mbar_init(smem_u32(&tail->k_empty[s]), 1);
+            mbar_init(smem_u32(&tail->k_empty[s]), MT);                   // one commit per turn that read the tile
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < 4; ++b) {
             mbar_init(smem_u32(&tail->d_full[b]), 1);
             mbar_init(smem_u32(&tail->d_empty[b]), kRdEpiThreads / 64);   // the eight warps that read this accumulator
         }
-        mbar_init(smem_u32(&tail->drain), 1);
+        mbar_init(smem_u32(&tail->drain[0]), 1);
+        mbar_init(smem_u32(&tail->drain[1]), 1);
         tail->abort_flag = 0;
         tail->issued = 0;
         fence_mbar_init();
@@ -172,16 +175,32 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
                 if (++s == stages) { s = 0; ++round; }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == kRdIssuerB) {
+        // ------------------------------------------------------------------ MMA issuers
+        // A turn is one 128 x 128 product (a row tile of the block times a key tile, eight instructions) into one of
+        // four 128-column accumulators: turn t uses accumulator t % 4. Turns of parity 0 belong to issuer 0 and epilogue
+        // set 0, those of parity 1 to issuer 1 and set 1, so each pair works through its own two accumulators. One thread
+        // needs longer to get a product out (two waits, the instructions, two commits) than the tensor core to run it;
+        // with two threads one product's instructions are queued while the other's execute, and with two accumulators
+        // per pair a pair's next product runs under its epilogue. A commit covers the instructions of the thread that
+        // makes it, so a ring slot is released by every turn that read it (its barrier counts them). With two row tiles
+        // issuer `rt` always takes row tile `rt`; with one, the issuers take alternate key tiles and the ring depth is
+        // even (see the launch), so that a slot always belongs to the same issuer.
         if (lane == 0) {
+            const int me = warp == 1 ? 0 : 1;
             bool ok = tc_wait(smem_u32(&tail->a_full), 0, &tail->abort_flag);
             if (!ok) rd_abort(tail, p.status, 32);
-            const uint32_t a_lo = umma_desc_lo(smem_u32(a_smem)), k_lo = umma_desc_lo(smem_u32(k_smem));
+            const uint32_t a_lo = umma_desc_lo(smem_u32(a_smem)) + (uint32_t)(MT == 2 ? me * ((128 * 128) >> 4) : 0);
+            const uint32_t k_lo = umma_desc_lo(smem_u32(k_smem));
             const uint32_t idesc = umma_idesc_bf16_m128(kRdTileKeys);
-            for (int i = 0, s = 0, round = 0; ok && i < T; ++i) {
-                const int buf = i & 1;
-                if (i >= 2 && !tc_wait(smem_u32(&tail->d_empty[buf]), ((i >> 1) - 1) & 1, &tail->abort_flag)) {
+            uint64_t a_desc[8];
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) a_desc[ks] = umma_desc(a_lo + umma_kstep(ks, a_half));
+            const int lstep = 2 >> mt_shift;           // key tiles between two turns of one issuer
+            int s = (me >> mt_shift) % stages, round = (me >> mt_shift) / stages;
+            for (int t = me; ok && t < total; t += 2) {
+                const int acc = t & 3, use = t >> 2;
+                if (use > 0 && !tc_wait(smem_u32(&tail->d_empty[acc]), (use - 1) & 1, &tail->abort_flag)) {
                     rd_abort(tail, p.status, 33);
                     break;
                 }
@@ -190,24 +209,18 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
                     break;
                 }
                 tmem_fence_after_sync();
-                const uint32_t ks_lo = k_lo + (uint32_t)s * (kRdStageBytes >> 4);
-                const uint32_t d = tmem_base + (uint32_t)buf * kRdAccCols;
+                const uint64_t k_desc = umma_desc(k_lo + (uint32_t)s * (kRdStageBytes >> 4));
+                const uint32_t d = tmem_base + (uint32_t)(acc * kRdAccCols);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    umma_bf16(d, umma_desc(a_lo + umma_kstep(ks, a_half)), umma_desc(ks_lo + umma_kstep(ks, kRdStageBytes / 2)),
-                              idesc, ks > 0);
-                if (MT == 2) {
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        umma_bf16(d + 128, umma_desc(a_lo + ((128 * 128) >> 4) + umma_kstep(ks, a_half)),
-                                  umma_desc(ks_lo + umma_kstep(ks, kRdStageBytes / 2)), idesc, ks > 0);
-                }
+                    umma_bf16(d, a_desc[ks], k_desc + umma_kstep(ks, kRdStageBytes / 2), idesc, ks > 0);
                 umma_commit(smem_u32(&tail->k_empty[s]));
-                umma_commit(smem_u32(&tail->d_full[buf]));
-                if (++s == stages) { s = 0; ++round; }
+                umma_commit(smem_u32(&tail->d_full[acc]));
+                s += lstep;
+                while (s >= stages) { s -= stages; ++round; }
             }
-            umma_commit(smem_u32(&tail->drain));     // everything issued has completed before TMEM is given back
-            mbar_wait_bounded(smem_u32(&tail->drain), 0);
+            umma_commit(smem_u32(&tail->drain[me]));     // everything this thread issued has completed before TMEM is given back
+            mbar_wait_bounded(smem_u32(&tail->drain[me]), 0);
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
@@ -215,27 +228,25 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
         const int q4 = warp & 3;
         const int L = q4 * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q4 * 32) << 16);
-        // Groups 0, 1 take the even key tiles (accumulator 0), groups 2, 3 the odd ones (accumulator 1), so two tiles
-        // are in the epilogue at any time and one pair's TMEM loads overlap the other pair's arithmetic. Within a
-        // pair: two row tiles -> one each, all 128 columns; one row tile -> 64 columns each.
-        const int parity = wg >> 1, sub = wg & 1;
-        const int rl = (MT == 2) ? sub * 128 + L : L;
-        const int col0 = (MT == 2) ? 0 : sub * 64;
-        const int nch = (MT == 2) ? 4 : 2;
-        const uint32_t t_p = t_lane + (uint32_t)((MT == 2) ? sub * 128 : col0);
+        // Two sets of two groups: set 0 reads the turns of parity 0, set 1 those of parity 1, so one set's TMEM loads
+        // run under the other's arithmetic. With two row tiles a set always has row tile `set`; with one, the sets take
+        // alternate key tiles. The two groups of a set take 64 of a turn's 128 columns each.
+        const int set = wg >> 1, sub = wg & 1;
+        const int rl = (MT == 2) ? set * 128 + L : L;
+        const int col0 = sub * 64;
         const int row = a0 + rl;                       // the key this thread sums for
         const float inv_r = (row < n) ? (LONG ? ginv[row] : s_inv[row]) : 0.f;
         const float thr = (row < n) ? __fdiv_rn(p.tau, inv_r) : INFINITY;   // Cm >= tau  <=>  G * inv_col >= tau / inv_row
         float sum = 0.f;
         bool ok = true;
-        for (int i = parity; i < T; i += 2) {
-            const int buf = parity;
-            ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (i >> 1) & 1, &tail->abort_flag));
+        for (int t = set; t < total; t += 2) {
+            const int i = t >> mt_shift, buf = t & 3;   // key tile and accumulator of this turn
+            ok = __all_sync(0xffffffffu, ok && tc_wait(smem_u32(&tail->d_full[buf]), (t >> 2) & 1, &tail->abort_flag));
             if (!ok) { rd_abort(tail, p.status, 35); break; }
             tmem_fence_after_sync();
-            for (int ch = 0; ch < nch; ++ch) {
+            for (int ch = 0; ch < 2; ++ch) {
                 float gacc[32];
-                tmem_ld<32>(t_p + (uint32_t)(buf * kRdAccCols + ch * 32), gacc);
+                tmem_ld<32>(t_lane + (uint32_t)(buf * kRdAccCols + col0 + ch * 32), gacc);
                 const int colbase = i * kRdTileKeys + col0 + ch * 32;
                 float4 ivl[8];
                 const float4* iv = LONG ? ivl : reinterpret_cast<const float4*>(s_inv + colbase);
@@ -249,18 +260,16 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
                 }
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
                 if (i + 1 < T) {
-                    // per element one compare (1.0 / 0.0) and half a packed multiply and half a packed multiply-add: a
-                    // compare + select pair would put two instructions per element on the ALU pipe, which throttles first
-                    float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
+                    // per element a multiply, a compare into a predicate and an add under it (one instruction on the ALU
+                    // pipe, two on the FMA pipe; a compare + select + add would put two on the ALU pipe, which throttles first)
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
                         const float4 c = iv[j >> 2];
-                        const float2 ta = mul_f32x2(make_float2(gacc[j], gacc[j + 1]), make_float2(c.x, c.y));
-                        const float2 tb = mul_f32x2(make_float2(gacc[j + 2], gacc[j + 3]), make_float2(c.z, c.w));
-                        sa = fma_f32x2(ta, make_float2(ge_mask(ta.x, thr), ge_mask(ta.y, thr)), sa);
-                        sb = fma_f32x2(tb, make_float2(ge_mask(tb.x, thr), ge_mask(tb.y, thr)), sb);
+                        add_if_ge(s0, gacc[j] * c.x, thr);
+                        add_if_ge(s1, gacc[j + 1] * c.y, thr);
+                        add_if_ge(s2, gacc[j + 2] * c.z, thr);
+                        add_if_ge(s3, gacc[j + 3] * c.w, thr);
                     }
-                    s0 = sa.x; s1 = sa.y; s2 = sb.x; s3 = sb.y;
                 } else {
                     // last tile: columns past the end of the cache hold whatever the rows beyond it contain (possibly
                     // NaN or Inf bit patterns); their inverse norm is 0 and a select drops them whatever the product is
@@ -282,9 +291,9 @@ gkv_redundancy_tc_kernel(const RedundancyLaunch p, const __grid_constant__ CUten
         }
         s_part[wg * 128 + L] = sum;
         epilogue_bar_sync();
-        if (!*(volatile int*)&tail->abort_flag && ((MT == 2) ? parity == 0 : wg == 0) && row < n) {
-            float tot;   // even-tile and odd-tile partials (and, with one row tile, the two column halves), fixed order
-            if (MT == 2) tot = s_part[sub * 128 + L] + s_part[(2 + sub) * 128 + L];
+        if (!*(volatile int*)&tail->abort_flag && ((MT == 2) ? sub == 0 : wg == 0) && row < n) {
+            float tot;   // the partials of the groups that shared this row (two column halves; with one row tile also the two sets), fixed order
+            if (MT == 2) tot = s_part[(2 * set) * 128 + L] + s_part[(2 * set + 1) * 128 + L];
             else tot = (s_part[L] + s_part[128 + L]) + (s_part[256 + L] + s_part[384 + L]);
             p.cbar[(size_t)unit * p.C + row] = (row < n - p.recent) ? tot * inv_r : 0.f;   // recent tokens: column zeroed
         }
@@ -327,6 +336,7 @@ cudaError_t launch_redundancy(const RedundancyLaunch& p, const CUtensorMap& tm_k
     const int blocks_per_unit = (p.C + kRdBlockRows - 1) / kRdBlockRows;
     int stages = 2;
     while (stages < kRdMaxStages && redundancy_smem_bytes(p.C, stages + 1) <= 227 * 1024) ++stages;
+    stages &= ~1;   // a block with one row tile has its issuers take alternate key tiles: a ring slot must stay with one of them
     if (p.C > kRdMaxShared)
         gkv_redundancy_tc_kernel<true><<<units * blocks_per_unit, kRdThreads, redundancy_smem_bytes(p.C, stages), s>>>(
             p, tm_k, blocks_per_unit, stages);
