@@ -258,14 +258,7 @@ __device__ __forceinline__ void bulk_wait() {
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// Packed fp32 pairs (one instruction for two lanes of arithmetic): d = a * b, d = a * b + c.
-__device__ __forceinline__ float2 mul_f32x2(float2 a, float2 b) {
-    float2 d;
-    asm("{ .reg .b64 ra, rb, rd;\n\t mov.b64 ra, {%2, %3};\n\t mov.b64 rb, {%4, %5};\n\t mul.f32x2 rd, ra, rb;\n\t"
-        " mov.b64 {%0, %1}, rd; }"
-        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-    return d;
-}
+// Packed fp32 pairs (one instruction for two lanes of arithmetic): d = a * b + c.
 __device__ __forceinline__ float2 fma_f32x2(float2 a, float2 b, float2 c) {
     float2 d;
     asm("{ .reg .b64 ra, rb, rc, rd;\n\t mov.b64 ra, {%2, %3};\n\t mov.b64 rb, {%4, %5};\n\t mov.b64 rc, {%6, %7};\n\t"
