@@ -191,6 +191,13 @@ def test_evict_large_window_and_group8():
     (dict(batch=2, h_q=8, h_kv=8, b=40, buffer=24, w=16, s=24), None),       # g = 1, a single ragged 128-key tile
     (dict(batch=1, h_q=16, h_kv=2, b=1000, buffer=153, w=64, s=153), None),  # g = 8, two CTAs per unit, last tile holds one key
     (dict(batch=1, h_q=32, h_kv=8, b=500, buffer=140, w=64, s=140), 601),    # g = 4, 256 rows in one CTA, cache not full
+    (dict(batch=2, h_q=3, h_kv=1, b=400, buffer=100, w=64, s=100), None),    # g = 3: 192 rows, two column chunks of 96
+    (dict(batch=2, h_q=10, h_kv=2, b=300, buffer=70, w=32, s=70), 333),      # g = 5: 160 rows, second row tile a quarter full
+    (dict(batch=2, h_q=12, h_kv=2, b=260, buffer=64, w=32, s=64), None),     # g = 6: 192 rows with 8-row blocks
+    (dict(batch=3, h_q=2, h_kv=2, b=700, buffer=80, w=64, s=80), None),      # g = 1, w = 64: 64 rows loaded twice, 16-row blocks
+    (dict(batch=3, h_q=4, h_kv=2, b=290, buffer=40, w=32, s=40), 301),       # g = 2, w = 32: 64 rows loaded twice, 8-row blocks
+    (dict(batch=2, h_q=4, h_kv=4, b=150, buffer=90, w=32, s=90), None),      # g = 1, w = 32: 32 rows loaded twice, half the lanes idle
+    (dict(batch=1, h_q=8, h_kv=1, b=1500, buffer=130, w=128, s=130), None),  # w = 128: four items of 32 window rows per unit add into the sums
 ])
 def test_score_tensor_core_shapes(shape, l):
     """Window shapes that take the tcgen05 scoring kernel (w a multiple of 16), full eviction step from the
