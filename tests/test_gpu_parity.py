@@ -810,3 +810,31 @@ def test_decode_random_shapes(i):
         S = oracle.window_mean(oracle.group_max(oracle.window_attention(synth.bits(q_win[n]), K[n], l_end), H))
         np.testing.assert_allclose(sacc[n][:, :l_end] / w, S, rtol=SCORE_RTOL, atol=SCORE_ATOL)
         assert not sacc[n][:, l_end:].any()
+
+
+def test_recompute_eviction_of_all_layers_and_of_one_inner_layer():
+    """The window queries of several layers in one call (leading [n_layers] dimension), and of one layer that is not
+    the first: every layer's step against the oracle on its own inputs."""
+    shape = dict(batch=2, h_q=16, h_kv=4, b=300, buffer=84, w=32, s=84)          # g = 4, 128 query rows per unit
+    L, B, H, b = 3, shape["batch"], shape["h_kv"], shape["b"]
+    kw = {k: shape[k] for k in ("batch", "h_q", "h_kv", "b", "buffer", "w")}
+    for layers in (-1, 1):
+        cfg = gkv.make_config(n_layers=L, **shape, fuse_window_scores=False, track_positions=True)
+        cache = gkv.GKVCache(cfg, DEV)
+        cases = [synth.eviction_case(synth.BASE_SEED + 4000 + i, **kw, l=370, n_planted=8, device=DEV) for i in range(L)]
+        for i, case in enumerate(cases):
+            load_case(cache, case, i)
+        which = list(range(L)) if layers < 0 else [layers]
+        snaps = {i: snapshot(cache, i, range(B)) for i in which}
+        kept = torch.full((len(which), B, H, b), -1, dtype=torch.int32, device=DEV)
+        q_win = torch.stack([cases[i].q_win for i in which]).contiguous()            # [layers][B][h_q][w][d]
+        cache.evict(layers, q_win if layers < 0 else q_win[0], kept if layers < 0 else kept[0])
+        cache.poll()
+        kk = kept.cpu().numpy()
+        for j, i in enumerate(which):
+            assert cache.state(i) == (b, b - shape["w"], 0)
+            check_evict_against_oracle(cache, i, range(B), snaps[i], kk[j], l=cases[i].l, n_h=cases[i].n_h,
+                                       q_win=[synth.bits(cases[i].q_win[n]) for n in range(B)])
+        for i in set(range(L)) - set(which):                                         # the other layers are untouched
+            assert cache.state(i) == (cases[i].l, cases[i].n_h, cfg.interval)
+            assert (synth.bits(cache.k[i]) == synth.bits(cases[i].k)).all()
