@@ -388,7 +388,6 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
         const float scale = p.scale_log2;
         bool ok = true;
         int t0 = 0;                                   // turn of the item's first product
-        [[maybe_unused]] uint32_t chunk_phase = 0;
 
         // pass-1 role of this thread: a row of the set's row tile, and 64 of a turn's 128 keys (32 for each copy when
         // the rows are loaded twice)
@@ -485,8 +484,8 @@ gkv_score_tc_kernel(const ScoreLaunch p, const __grid_constant__ CUtensorMap tm_
                     for (int step = 0; ok && step < 2; ++step) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&tail->chunk_bar));
-                        ok = __all_sync(0xffffffffu, tc_wait(smem_u32(&tail->chunk_bar), chunk_phase & 1, &tail->abort_flag));
-                        ++chunk_phase;
+                        // two phases of the barrier per boundary: its parity is `step` every time
+                        ok = __all_sync(0xffffffffu, tc_wait(smem_u32(&tail->chunk_bar), (uint32_t)step, &tail->abort_flag));
                         if (ok && step == 0) flush_chunk(chunk_lo);
                     }
                     if (!ok) { tc_abort(tail, p.status, 27); break; }
