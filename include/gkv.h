@@ -299,6 +299,17 @@ gkv_status gkv_decode_launch_plan(const gkv_config* cfg, int32_t n_layers_in_lau
 typedef struct { int32_t grid, stages, ctas_per_sm, smem_bytes; } gkv_evict_plan_t;
 gkv_status gkv_evict_launch_plan(const gkv_config* cfg, int32_t n_layers_in_launch, int32_t sm_count, gkv_evict_plan_t* out);
 
+/* How the recompute path would launch its tensor-core scoring kernel on the cache (no paper counterpart; host
+ * arithmetic, for capacity planning and tests without a GPU). tensor_core = 0 when the window is not a multiple of 16
+ * (the other scoring kernel runs; the remaining fields are 0). items = work items (a unit and up to 64 window rows of
+ * all its heads), rows_per_item = query rows of an item, grid = CTAs launched (persistent, one per SM at most, rounds
+ * filled equally), stages = depth of the ring of 128-key tiles, query_buffers = 1 or 2, smem_bytes = dynamic shared
+ * memory per CTA. With at most 128 query rows per item the ring depth is even (the kernel's two issuing threads then
+ * take alternate tiles, and a ring slot must stay with one of them).
+ * Errors: as gkv_query_sizes; INVALID_ARG for a layer count other than 1 or cfg->n_layers. */
+typedef struct { int32_t tensor_core, grid, items, rows_per_item, stages, query_buffers, smem_bytes; } gkv_score_plan_t;
+gkv_status gkv_score_launch_plan(const gkv_config* cfg, int32_t n_layers_in_launch, int32_t sm_count, gkv_score_plan_t* out);
+
 /* Memory model of the paper's appendix "Memory Analysis": bytes of the full KV cache at
  * seq_len tokens, of the compressed cache ((b + s) rows instead of seq_len), and of the score
  * cache F (b - w entries per head), for `elem_bytes`-wide elements, over all layers and the

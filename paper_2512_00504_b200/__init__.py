@@ -64,6 +64,11 @@ class gkv_evict_plan_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("grid", "stages", "ctas_per_sm", "smem_bytes")]
 
 
+class gkv_score_plan_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("tensor_core", "grid", "items", "rows_per_item", "stages", "query_buffers",
+                                              "smem_bytes")]
+
+
 class gkv_memory_model_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint64) for n in ("full_kv", "compressed_kv", "score_cache")]
 
@@ -125,6 +130,8 @@ def lib() -> ctypes.CDLL:
         L.gkv_decode_launch_plan.argtypes = [P(gkv_config), i32, i32, i32, P(gkv_decode_plan_t)]
         L.gkv_evict_launch_plan.argtypes = [P(gkv_config), i32, i32, P(gkv_evict_plan_t)]
         L.gkv_evict_launch_plan.restype = ctypes.c_int
+        L.gkv_score_launch_plan.argtypes = [P(gkv_config), i32, i32, P(gkv_score_plan_t)]
+        L.gkv_score_launch_plan.restype = ctypes.c_int
         L.gkv_strerror.argtypes = [ctypes.c_int]
         L.gkv_strerror.restype = ctypes.c_char_p
         L.gkv_destroy.argtypes = [vp]
@@ -184,6 +191,13 @@ def gkv_decode_launch_plan(cfg: gkv_config, n_layers_in_launch: int, window_step
     out = gkv_decode_plan_t()
     _check(lib().gkv_decode_launch_plan(ctypes.byref(cfg), int(n_layers_in_launch), int(bool(window_step)), int(sm_count),
                                         ctypes.byref(out)), "gkv_decode_launch_plan")
+    return out
+
+
+def gkv_score_launch_plan(cfg: gkv_config, n_layers_in_launch: int, sm_count: int = 148) -> gkv_score_plan_t:
+    out = gkv_score_plan_t()
+    _check(lib().gkv_score_launch_plan(ctypes.byref(cfg), int(n_layers_in_launch), int(sm_count), ctypes.byref(out)),
+           "gkv_score_launch_plan")
     return out
 
 

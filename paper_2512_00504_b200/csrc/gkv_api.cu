@@ -793,6 +793,25 @@ gkv_status gkv_evict_launch_plan(const gkv_config* cfg, int32_t n_layers_in_laun
     return GKV_OK;
 }
 
+gkv_status gkv_score_launch_plan(const gkv_config* cfg, int32_t n_layers_in_launch, int32_t sm_count, gkv_score_plan_t* out) {
+    if (!out) return GKV_ERR_INVALID_ARG;
+    const gkv_status st = check_config(cfg);
+    if (st != GKV_OK) return st;
+    if (n_layers_in_launch != 1 && n_layers_in_launch != cfg->n_layers) return GKV_ERR_INVALID_ARG;
+    const int g = cfg->n_q_heads / cfg->n_kv_heads;
+    const int wk = score_tc_rows_per_cta(g, cfg->window);
+    *out = {};
+    if (wk == 0) return GKV_OK;   // this window goes to the other scoring kernel: tensor_core stays 0
+    ScoreLaunch p = {};
+    p.n_layers = n_layers_in_launch; p.batch = cfg->batch; p.h_q = cfg->n_q_heads; p.h_kv = cfg->n_kv_heads;
+    p.g = g; p.C = cfg->budget + cfg->buffer; p.w = cfg->window; p.sm_count = sm_count;
+    ScoreTcPlan plan;
+    score_tc_plan(p, wk, &plan);
+    out->tensor_core = 1; out->grid = plan.grid; out->items = plan.items; out->rows_per_item = plan.rows;
+    out->stages = plan.stages; out->query_buffers = plan.q_bufs; out->smem_bytes = (int32_t)plan.smem;
+    return GKV_OK;
+}
+
 gkv_status gkv_memory_model(const gkv_config* cfg, int64_t seq_len, int32_t elem_bytes, gkv_memory_model_t* out) {
     if (!cfg || !out || seq_len <= 0 || elem_bytes <= 0) return GKV_ERR_INVALID_ARG;
     if (cfg->n_layers <= 0 || cfg->batch <= 0 || cfg->n_kv_heads <= 0 || cfg->head_dim <= 0 || cfg->budget <= 0 ||

@@ -156,6 +156,8 @@ cudaError_t launch_evict_compact(const EvictLaunch& p, int sm_count, cudaStream_
 cudaError_t launch_score(const ScoreLaunch& p, const CUtensorMap& tm_k, cudaStream_t s);
 cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s);
 int score_tc_rows_per_cta(int g, int w);
+struct ScoreTcPlan { int items, items_per_unit, rows, q_bufs, stages, grid; size_t smem; };
+void score_tc_plan(const ScoreLaunch& p, int wk, ScoreTcPlan* out);
 int score_tc_q_box_rows(int wk);
 constexpr int kScoreTcKeyBoxRows = 128;   // rows of one box of the key tensor map that launch_score_tc takes
 cudaError_t score_tc_kernel_setup();

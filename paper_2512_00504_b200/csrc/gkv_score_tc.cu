@@ -606,7 +606,9 @@ cudaError_t score_tc_kernel_setup() {
     return cudaSuccess;
 }
 
-cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s) {
+// Launch shape of the kernel for window rows per item `wk`: items, query rows per item, query buffers, ring depth,
+// shared memory and grid.
+void score_tc_plan(const ScoreLaunch& p, int wk, ScoreTcPlan* out) {
     const int n_cta = p.w / wk;
     const int units = p.n_layers * p.batch * p.h_kv;
     const int items = units * n_cta;
@@ -619,18 +621,27 @@ cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const
     // slot always belongs to the same issuer: a thread that saw only every other phase of a slot's barrier could pass a
     // parity wait two phases early. (With two turns per tile both issuers wait for every tile.)
     if (rows <= 128) stages &= ~1;
-    const size_t smem = score_tc_smem_bytes(p.C, rows, stages, q_bufs);
-    if (n_cta > 1) {
-        const size_t off = (size_t)p.layer0 * p.batch * p.h_kv * p.C;
-        cudaError_t e = cudaMemsetAsync(p.sacc + off, 0, sizeof(float) * (size_t)units * p.C, s);
-        if (e != cudaSuccess) return e;
-    }
     // persistent: one CTA per SM (shared memory and tensor memory allow no more), rounds filled equally
     const int sm = p.sm_count > 0 ? p.sm_count : 148;
     int grid = items < sm ? items : sm;
     if (items > sm) {
         const int rounds = (items + sm - 1) / sm;
         grid = (items + rounds - 1) / rounds;
+    }
+    out->items = items; out->items_per_unit = n_cta; out->rows = rows; out->q_bufs = q_bufs; out->stages = stages;
+    out->grid = grid; out->smem = score_tc_smem_bytes(p.C, rows, stages, q_bufs);
+}
+
+cudaError_t launch_score_tc(const ScoreLaunch& p, const CUtensorMap& tm_k, const CUtensorMap& tm_q, int wk, cudaStream_t s) {
+    ScoreTcPlan plan;
+    score_tc_plan(p, wk, &plan);
+    const int n_cta = plan.items_per_unit, units = p.n_layers * p.batch * p.h_kv, stages = plan.stages, q_bufs = plan.q_bufs;
+    const int grid = plan.grid;
+    const size_t smem = plan.smem;
+    if (n_cta > 1) {
+        const size_t off = (size_t)p.layer0 * p.batch * p.h_kv * p.C;
+        cudaError_t e = cudaMemsetAsync(p.sacc + off, 0, sizeof(float) * (size_t)units * p.C, s);
+        if (e != cudaSuccess) return e;
     }
     const bool chunked = p.C > kTcChunkKeys;
     if (wk == 16 && !chunked) gkv_score_tc_kernel<16, false><<<grid, kTcThreads, smem, s>>>(p, tm_k, tm_q, n_cta, stages, q_bufs);

@@ -170,6 +170,37 @@ def test_evict_launch_plan_invariants(sm_count):
     assert (p.grid, p.stages, p.ctas_per_sm) == (256, 6, 2)
 
 
+def test_score_launch_plan_invariants():
+    """Host-side planning of the tensor-core scoring launch: shared memory within a CTA's 227 KB, a persistent grid of at
+    most one CTA per SM with equally filled rounds, and the rule its two issuing threads rely on: with at most 128 query
+    rows per item (one product per key tile, taken by the issuers in turn) the ring depth is even, so that a ring slot
+    always stays with the same thread."""
+    seen_small = seen_large = 0
+    for h_q, h_kv in ((4, 4), (8, 4), (12, 4), (16, 4), (28, 4), (32, 8), (64, 8), (16, 2)):
+        for w in (16, 32, 48, 64, 128):
+            for b, buffer in ((256, 128), (1024, 128), (2048, 256), (3800, 296)):
+                for batch in (1, 64, 256):
+                    cfg = base(batch=batch, n_layers=1, h_q=h_q, h_kv=h_kv, w=w, b=b, buffer=max(buffer, w), s=max(buffer, w))
+                    p = gkv.gkv_score_launch_plan(cfg, 1, 148)
+                    assert p.tensor_core == 1
+                    g = h_q // h_kv
+                    assert p.rows_per_item % (16 * g) == 0 and p.rows_per_item <= 256
+                    assert p.items == batch * h_kv * (w * g // p.rows_per_item)
+                    assert 2 <= p.stages <= 6 and p.query_buffers in (1, 2) and p.smem_bytes <= 227 * 1024
+                    assert 1 <= p.grid <= min(p.items, 148)
+                    if p.items > 148:
+                        assert p.grid == -(-p.items // -(-p.items // 148))
+                    if p.rows_per_item <= 128:
+                        assert p.stages % 2 == 0
+                        seen_small += 1
+                    else:
+                        seen_large += 1
+    assert seen_small and seen_large
+    # windows that are not a multiple of 16 go to the other scoring kernel
+    p = gkv.gkv_score_launch_plan(base(w=20, buffer=128, s=128), 1, 148)
+    assert (p.tensor_core, p.grid, p.stages) == (0, 0, 0)
+
+
 def test_memory_model_reproduces_the_papers_appendix():
     """Appendix "Memory Analysis": 28 layers, d = 128, 2 KV heads, bf16, 16k tokens -> ~0.44 GB per
     sequence and 56 GB at batch 128; with s = 128 and b = 512 / 1024 / 2048 the compressed cache
