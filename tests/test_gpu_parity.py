@@ -760,13 +760,13 @@ def _random_eviction_setup(i):
     return shape, kw
 
 
-@pytest.mark.parametrize("i", range(24))
+@pytest.mark.parametrize("i", range(48))
 def test_evict_random_shapes(i):
     shape, kw = _random_eviction_setup(i)
     run_single_eviction(shape, synth.BASE_SEED + 2000 + i, **kw)
 
 
-@pytest.mark.parametrize("i", range(12))
+@pytest.mark.parametrize("i", range(24))
 def test_decode_random_shapes(i):
     """Seeded sweep of decode shapes: a few plain steps, then the w window steps before a compression, at a random
     cache length; every step's output and the accumulated window sums against the oracle."""
